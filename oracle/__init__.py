@@ -1,0 +1,251 @@
+"""ctypes front end of the CPU oracle (``srq_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the bench's CPU
+baseline leg import this; the product package never does, and this module
+never imports the product package.  All arithmetic lives in the C file; this
+module only builds it with gcc and marshals numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "srq_oracle.c")
+_LIB = os.path.join(_HERE, "libsrq_oracle.so")
+
+PER_TENSOR, PER_ROW = 0, 1
+SR, RTN = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fused multiply-add, OpenMP over rows)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+               "-fPIC", "-shared", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+class _QSpec(ctypes.Structure):
+    _fields_ = [("bits", ctypes.c_int32), ("scale_mode", ctypes.c_int32),
+                ("round_mode", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("seed", ctypes.c_uint64), ("tensor_id", ctypes.c_uint64),
+                ("index_offset", ctypes.c_uint64)]
+
+
+@dataclass
+class QSpec:
+    """One quantization point: the (Delta rule, eps) pair of one operand."""
+    bits: int = 8
+    scale_mode: int = PER_TENSOR
+    round_mode: int = SR
+    seed: int = 0
+    tensor_id: int = 0
+    index_offset: int = 0
+
+    def c(self) -> _QSpec:
+        return _QSpec(self.bits, self.scale_mode, self.round_mode, 0, self.seed, self.tensor_id,
+                      self.index_offset)
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        L = _lib
+        u32p = ctypes.POINTER(ctypes.c_uint32)
+        L.orc_philox4x32_10.argtypes = [u32p, u32p, u32p]
+        L.orc_philox4x32_10.restype = None
+        L.orc_threshold_u24.argtypes = [ctypes.c_uint64] * 3
+        L.orc_threshold_u24.restype = ctypes.c_uint32
+        L.orc_scale_from_absmax.argtypes = [ctypes.c_float, ctypes.c_int,
+                                            ctypes.POINTER(ctypes.c_float),
+                                            ctypes.POINTER(ctypes.c_float)]
+        L.orc_scale_from_absmax.restype = None
+        L.orc_quantize_scalar.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_int,
+                                          ctypes.c_int, ctypes.c_uint32]
+        L.orc_quantize_scalar.restype = ctypes.c_int
+        vp = ctypes.c_void_p
+        i64 = ctypes.c_int64
+        L.orc_sum_sr_codes_over_all_thresholds.argtypes = [ctypes.c_float, ctypes.c_float,
+                                                          ctypes.c_int]
+        L.orc_sum_sr_codes_over_all_thresholds.restype = i64
+        for name in ("orc_absmax_tensor", "orc_absmax_rows", "orc_absmax_cols"):
+            getattr(L, name).argtypes = [vp, i64, i64, i64, vp]
+            getattr(L, name).restype = None
+        L.orc_sr_quantize.argtypes = [vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                      ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64,
+                                      vp, vp, vp, vp]
+        L.orc_sr_quantize.restype = ctypes.c_int
+        L.orc_gemm_i8_nt.argtypes = [vp, vp, i64, i64, i64, vp]
+        L.orc_gemm_i8_nt.restype = i64
+        L.orc_dequant.argtypes = [vp, i64, i64, vp, ctypes.c_int, vp, ctypes.c_int, vp]
+        L.orc_dequant.restype = None
+        qp = ctypes.POINTER(_QSpec)
+        for name in ("orc_qlinear_fwd", "orc_qlinear_bwd_input", "orc_qlinear_bwd_weight"):
+            getattr(L, name).argtypes = [vp, vp, i64, i64, i64, qp, qp, vp, vp, vp, vp, vp, vp]
+            getattr(L, name).restype = i64
+        L.orc_num_threads.argtypes = []
+        L.orc_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32_2d(x) -> np.ndarray:
+    x = np.asarray(x)
+    if x.dtype != np.float32 or x.ndim != 2:
+        raise TypeError("oracle takes 2-D float32 arrays (widen bfloat16 first)")
+    if x.strides[1] != 4 or x.strides[0] % 4 != 0:
+        x = np.ascontiguousarray(x)
+    return x
+
+
+def num_threads() -> int:
+    return int(lib().orc_num_threads())
+
+
+def philox4x32_10(ctr, key):
+    c = (ctypes.c_uint32 * 4)(*[int(v) & 0xFFFFFFFF for v in ctr])
+    k = (ctypes.c_uint32 * 2)(*[int(v) & 0xFFFFFFFF for v in key])
+    o = (ctypes.c_uint32 * 4)()
+    lib().orc_philox4x32_10(c, k, o)
+    return [int(v) for v in o]
+
+
+def threshold_u24(seed: int, tensor_id: int, i: int) -> int:
+    return int(lib().orc_threshold_u24(seed, tensor_id, i))
+
+
+def scale_from_absmax(m: float, bits: int):
+    d, inv = ctypes.c_float(), ctypes.c_float()
+    lib().orc_scale_from_absmax(ctypes.c_float(m), bits, ctypes.byref(d), ctypes.byref(inv))
+    return np.float32(d.value), np.float32(inv.value)
+
+
+def quantize_scalar(x: float, inv: float, bits: int, round_mode: int, u24: int = 0) -> int:
+    return int(lib().orc_quantize_scalar(ctypes.c_float(x), ctypes.c_float(inv), bits, round_mode,
+                                         u24))
+
+
+def sum_sr_codes_over_all_thresholds(x: float, inv: float, bits: int) -> int:
+    return int(lib().orc_sum_sr_codes_over_all_thresholds(ctypes.c_float(x), ctypes.c_float(inv),
+                                                         bits))
+
+
+def absmax(x, mode: str) -> np.ndarray:
+    x = _f32_2d(x)
+    rows, cols = x.shape
+    ld = x.strides[0] // 4
+    n = {"tensor": 1, "rows": rows, "cols": cols}[mode]
+    m = np.zeros(n, dtype=np.float32)
+    getattr(lib(), "orc_absmax_" + mode)(_ptr(x), rows, cols, ld, _ptr(m))
+    return m
+
+
+def sr_quantize(x, q: QSpec, want_rm: bool = True, want_tr: bool = False):
+    """Returns (codes_rm, scale_rm, codes_tr, scale_tr); unrequested pairs are None."""
+    x = _f32_2d(x)
+    rows, cols = x.shape
+    ld = x.strides[0] // 4
+    per_row = q.scale_mode == PER_ROW
+    crm = srm = ctr = strr = None
+    if want_rm:
+        crm = np.zeros((rows, cols), dtype=np.int8)
+        srm = np.zeros(rows if per_row else 1, dtype=np.float32)
+    if want_tr:
+        ctr = np.zeros((cols, rows), dtype=np.int8)
+        strr = np.zeros(cols if per_row else 1, dtype=np.float32)
+    rc = lib().orc_sr_quantize(_ptr(x), rows, cols, ld, q.bits, q.scale_mode, q.round_mode,
+                               q.seed, q.tensor_id, q.index_offset,
+                               _ptr(crm), _ptr(srm), _ptr(ctr), _ptr(strr))
+    if rc != 0:
+        raise ValueError("oracle: bits outside 2..8")
+    return crm, srm, ctr, strr
+
+
+def gemm_i8_nt(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """acc[i,j] = sum_k a[i,k] b[j,k] for int8 codes; raises if a sum leaves int32."""
+    a = np.ascontiguousarray(a, dtype=np.int8)
+    b = np.ascontiguousarray(b, dtype=np.int8)
+    M, Kc = a.shape
+    N, Kb = b.shape
+    assert Kc == Kb
+    acc = np.zeros((M, N), dtype=np.int32)
+    ov = lib().orc_gemm_i8_nt(_ptr(a), _ptr(b), M, N, Kc, _ptr(acc))
+    if ov:
+        raise OverflowError(f"{ov} accumulators do not fit in int32")
+    return acc
+
+
+def dequant(acc: np.ndarray, s_row: np.ndarray, s_col: np.ndarray) -> np.ndarray:
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    s_row = np.ascontiguousarray(s_row, dtype=np.float32)
+    s_col = np.ascontiguousarray(s_col, dtype=np.float32)
+    M, N = acc.shape
+    assert s_row.size in (1, M) and s_col.size in (1, N)
+    out = np.zeros((M, N), dtype=np.float32)
+    lib().orc_dequant(_ptr(acc), M, N, _ptr(s_row), int(s_row.size != 1),
+                      _ptr(s_col), int(s_col.size != 1), _ptr(out))
+    return out
+
+
+@dataclass
+class LinearResult:
+    out: np.ndarray
+    acc: np.ndarray
+    codes_a: np.ndarray
+    scale_a: np.ndarray
+    codes_b: np.ndarray
+    scale_b: np.ndarray
+
+
+def _qlinear(fn, X0, X1, T, N, K, q0: QSpec, q1: QSpec, shape0, shape1, out_shape):
+    X0 = np.ascontiguousarray(X0, dtype=np.float32)
+    X1 = np.ascontiguousarray(X1, dtype=np.float32)
+    c0 = np.zeros(shape0, dtype=np.int8)
+    c1 = np.zeros(shape1, dtype=np.int8)
+    s0 = np.zeros(shape0[0] if q0.scale_mode == PER_ROW else 1, dtype=np.float32)
+    s1 = np.zeros(shape1[0] if q1.scale_mode == PER_ROW else 1, dtype=np.float32)
+    acc = np.zeros(out_shape, dtype=np.int32)
+    out = np.zeros(out_shape, dtype=np.float32)
+    c_q0, c_q1 = q0.c(), q1.c()
+    ov = fn(_ptr(X0), _ptr(X1), T, N, K, ctypes.byref(c_q0), ctypes.byref(c_q1),
+            _ptr(c0), _ptr(s0), _ptr(c1), _ptr(s1), _ptr(acc), _ptr(out))
+    if ov:
+        raise OverflowError(f"{ov} accumulators do not fit in int32")
+    return LinearResult(out, acc, c0, s0, c1, s1)
+
+
+def qlinear_fwd(A, W, qa: QSpec, qw: QSpec) -> LinearResult:
+    """Alg. 1: Y[T,N] = Q(A[T,K]) Q(W[N,K])^T."""
+    T, K = A.shape
+    N, K2 = W.shape
+    assert K == K2
+    return _qlinear(lib().orc_qlinear_fwd, A, W, T, N, K, qa, qw, (T, K), (N, K), (T, N))
+
+
+def qlinear_bwd_input(dY, W, qdy: QSpec, qw: QSpec) -> LinearResult:
+    """Alg. 2: dA[T,K] = Q(dY[T,N]) Q(W[N,K]); codes_b is the [K,N] layout of Q(W)."""
+    T, N = dY.shape
+    N2, K = W.shape
+    assert N == N2
+    return _qlinear(lib().orc_qlinear_bwd_input, dY, W, T, N, K, qdy, qw, (T, N), (K, N), (T, K))
+
+
+def qlinear_bwd_weight(dY, A, qdy: QSpec, qa: QSpec) -> LinearResult:
+    """Alg. 2: dW[N,K] = Q(dY[T,N])^T Q(A[T,K]); both code sets are transposed layouts."""
+    T, N = dY.shape
+    T2, K = A.shape
+    assert T == T2
+    return _qlinear(lib().orc_qlinear_bwd_weight, dY, A, T, N, K, qdy, qa, (N, T), (K, T), (N, K))

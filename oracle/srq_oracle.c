@@ -1,0 +1,408 @@
+/*
+ * CPU oracle for the stochastically-rounded quantized linear layer.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what
+ * the method computes; it exists so that the CUDA library can be checked
+ * against it element by element.  It shares no code, header, table or
+ * constant generator with the CUDA path, and the product never calls it.
+ *
+ * Every function follows one passage of the paper ("Training with Fewer
+ * Bits: Unlocking Edge LLMs Training with Stochastic Rounding"):
+ *   - Def. 1  threshold quantizer  Q_D(x, eps)
+ *   - Def. 2  round-to-nearest     eps = 1/2, ties toward +infinity
+ *   - Def. 3  stochastic rounding  eps ~ U[0,1], independent per element
+ *   - Sec. 2.2.2  mixed-precision matmul = exact product of the two
+ *                 quantized matrices (low-precision multiply, wide accumulate)
+ *   - Alg. 1  forward   A_out = Q(A_in) Q(W)
+ *   - Alg. 2  backward  dA_in = Q(dA_out) Q(W)^T,  dW = Q(A_in)^T Q(dA_out)
+ *
+ * Storage convention (the usual deep-learning one, transposed with respect
+ * to the paper's W[in,out]):  A[T,K], W[N,K], dY[T,N];  Y[T,N] = A W^T,
+ * dA[T,K] = dY W,  dW[N,K] = dY^T A.
+ *
+ * Floating point: the rounding decision is taken in IEEE binary32 with
+ * round-to-nearest and no fused multiply-add (compile with
+ * -ffp-contract=off), because the decision yields an integer code and both
+ * sides of a parity test must take it in the same precision.  bfloat16
+ * inputs are widened to binary32 (exactly) by the caller.
+ *
+ * The step size D of a group g of elements is not fixed by the paper (D is
+ * a free "precision level" in Def. 1); it is the symmetric absmax rule
+ * D_g = max_g|x| / qmax,  qmax = 2^(bits-1) - 1,  codes in [-qmax, qmax].
+ *
+ * Pins for every function here live in tests/test_oracle_*.py.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORC_PER_TENSOR 0
+#define ORC_PER_ROW 1
+#define ORC_SR 0
+#define ORC_RTN 1
+
+/* ---------------------------------------------------------------------- */
+/* Thresholds eps (Def. 3): counter-based Philox4x32-10                     */
+/* (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as       */
+/* 1, 2, 3", SC'11).  A 128-bit counter and a 64-bit key give four 32-bit  */
+/* words after ten rounds; the key is bumped by the Weyl constants between */
+/* rounds.                                                                 */
+/* ---------------------------------------------------------------------- */
+void orc_philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr_in[0], c1 = ctr_in[1], c2 = ctr_in[2], c3 = ctr_in[3];
+    uint32_t k0 = key_in[0], k1 = key_in[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) {
+            k0 += 0x9E3779B9u;
+            k1 += 0xBB67AE85u;
+        }
+        uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+        uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+        uint32_t n0 = hi1 ^ c1 ^ k0;
+        uint32_t n1 = lo1;
+        uint32_t n2 = hi0 ^ c3 ^ k1;
+        uint32_t n3 = lo0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/*
+ * The 24-bit threshold of the element with flat index i (row-major index of
+ * the SOURCE tensor plus index_offset): Philox block j = i >> 2 with counter
+ * {lo(j), hi(j), lo(tensor_id), hi(tensor_id)} and key {lo(seed), hi(seed)};
+ * the element takes word i & 3, and its top 24 bits u24 stand for
+ * eps = u24 * 2^-24 in [0, 1).
+ */
+uint32_t orc_threshold_u24(uint64_t seed, uint64_t tensor_id, uint64_t i)
+{
+    uint64_t j = i >> 2;
+    uint32_t ctr[4] = { (uint32_t)j, (uint32_t)(j >> 32),
+                        (uint32_t)tensor_id, (uint32_t)(tensor_id >> 32) };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    return out[i & 3] >> 8;
+}
+
+/* ---------------------------------------------------------------------- */
+/* Step size (absmax rule)                                                  */
+/* ---------------------------------------------------------------------- */
+static int orc_qmax(int bits) { return (1 << (bits - 1)) - 1; }
+
+/*
+ * D = m / qmax and the reciprocal 1/D actually multiplied in, inv = qmax / m,
+ * both one binary32 division.  m = 0 is Def. 1's D = 0 case (Q_0 is the
+ * identity, and the group is all zeros, so codes 0 with scale 0 reproduce
+ * it).  A group whose absmax is so small that qmax / m overflows binary32
+ * (m below about 4e-37) is treated the same way.
+ */
+void orc_scale_from_absmax(float m, int bits, float *delta, float *inv)
+{
+    float qmax = (float)orc_qmax(bits);
+    float r = (m == 0.0f) ? 0.0f : qmax / m;
+    if (isinf(r) || r != r) r = 0.0f;
+    *inv = r;
+    *delta = (r == 0.0f) ? 0.0f : m / qmax;
+}
+
+/* ---------------------------------------------------------------------- */
+/* Def. 1-3: one element                                                    */
+/* ---------------------------------------------------------------------- */
+/*
+ * Code q such that Q_D(x, eps) = q * D, with x/D evaluated as x * inv:
+ *   t = x * inv;  f = floor(t);  p = t - f   (the fractional part)
+ *   SR : round up  iff  eps < p   (strict, so grid-exact x never moves;
+ *        Def. 1 rounds down when p < eps, up otherwise; with eps on a
+ *        2^-24 lattice the strict form keeps P(up) within 2^-24 of p)
+ *   RTN: round up  iff  p >= 1/2  (Def. 1 with eps = 1/2; a tie goes up,
+ *        i.e. toward +infinity, Def. 2)
+ *   q = f + up, clamped to [-qmax, qmax] (the rounded product t can exceed
+ *   qmax by one ulp at the extreme element).
+ */
+int orc_quantize_scalar(float x, float inv, int bits, int round_mode, uint32_t u24)
+{
+    int qmax = orc_qmax(bits);
+    float t = x * inv;
+    float f = floorf(t);
+    float p = t - f;
+    int up;
+    if (round_mode == ORC_SR) {
+        float eps = (float)u24 * 0x1p-24f; /* exact: 24-bit integer times a power of two */
+        up = (eps < p);
+    } else {
+        up = (p >= 0.5f);
+    }
+    int q = (int)f + up;
+    if (q > qmax) q = qmax;
+    if (q < -qmax) q = -qmax;
+    return q;
+}
+
+/*
+ * Sum of the SR codes of x over all 2^24 possible thresholds.  With eps
+ * uniform on the lattice (Def. 3), E[q] = sum / 2^24 exactly; the tests use
+ * it to check P(round up) without sampling.
+ */
+int64_t orc_sum_sr_codes_over_all_thresholds(float x, float inv, int bits)
+{
+    int64_t sum = 0;
+    for (uint32_t u = 0; u < (1u << 24); ++u)
+        sum += orc_quantize_scalar(x, inv, bits, ORC_SR, u);
+    return sum;
+}
+
+/* ---------------------------------------------------------------------- */
+/* absmax over the three kinds of group                                     */
+/* ---------------------------------------------------------------------- */
+void orc_absmax_tensor(const float *x, int64_t rows, int64_t cols, int64_t ld, float *m)
+{
+    float best = 0.0f;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < cols; ++c) {
+            float a = fabsf(x[r * ld + c]);
+            if (a > best) best = a;
+        }
+    m[0] = best;
+}
+
+void orc_absmax_rows(const float *x, int64_t rows, int64_t cols, int64_t ld, float *m)
+{
+    for (int64_t r = 0; r < rows; ++r) {
+        float best = 0.0f;
+        for (int64_t c = 0; c < cols; ++c) {
+            float a = fabsf(x[r * ld + c]);
+            if (a > best) best = a;
+        }
+        m[r] = best;
+    }
+}
+
+void orc_absmax_cols(const float *x, int64_t rows, int64_t cols, int64_t ld, float *m)
+{
+    for (int64_t c = 0; c < cols; ++c) m[c] = 0.0f;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < cols; ++c) {
+            float a = fabsf(x[r * ld + c]);
+            if (a > m[c]) m[c] = a;
+        }
+}
+
+/* ---------------------------------------------------------------------- */
+/* Matrix quantizer (Def. 3, "matrix stochastic rounding is element-wise") */
+/* ---------------------------------------------------------------------- */
+/*
+ * x[rows, cols] (row pitch ld) -> int8 codes in either or both layouts.
+ *
+ *   codes_rm[rows, cols] with scale_rm: [1] (per tensor) or [rows] (one step
+ *       size per row);
+ *   codes_tr[cols, rows] (the transpose) with scale_tr: [1] or [cols] (one
+ *       step size per COLUMN of x, i.e. per row of the transposed view).
+ *
+ * A step size can be pulled out of a matrix product only if it is constant
+ * along the contracted axis, which is the contiguous axis of each layout;
+ * hence "per row" always means per row of the layout being written.  Per
+ * tensor, both layouts hold the same codes.  Either way the element x[r,c]
+ * uses ONE threshold, that of flat index index_offset + r*cols + c, for both
+ * layouts (one eps per element per quantization point, Alg. 2).
+ *
+ * Any output pointer pair may be NULL.  Returns 0, or 1 if bits is outside
+ * 2..8.
+ */
+int orc_sr_quantize(const float *x, int64_t rows, int64_t cols, int64_t ld,
+                    int bits, int scale_mode, int round_mode,
+                    uint64_t seed, uint64_t tensor_id, uint64_t index_offset,
+                    int8_t *codes_rm, float *scale_rm,
+                    int8_t *codes_tr, float *scale_tr)
+{
+    if (bits < 2 || bits > 8) return 1;
+    float m_tensor = 0.0f;
+    if (scale_mode == ORC_PER_TENSOR) orc_absmax_tensor(x, rows, cols, ld, &m_tensor);
+
+    if (codes_rm) {
+        if (scale_mode == ORC_PER_TENSOR) {
+            float delta, inv;
+            orc_scale_from_absmax(m_tensor, bits, &delta, &inv);
+            scale_rm[0] = delta;
+        } else {
+            orc_absmax_rows(x, rows, cols, ld, scale_rm); /* holds absmax for now */
+        }
+#pragma omp parallel for schedule(static)
+        for (int64_t r = 0; r < rows; ++r) {
+            float delta, inv;
+            if (scale_mode == ORC_PER_TENSOR) {
+                orc_scale_from_absmax(m_tensor, bits, &delta, &inv);
+            } else {
+                orc_scale_from_absmax(scale_rm[r], bits, &delta, &inv);
+                scale_rm[r] = delta;
+            }
+            for (int64_t c = 0; c < cols; ++c) {
+                uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
+                uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, i) : 0u;
+                codes_rm[r * cols + c] =
+                    (int8_t)orc_quantize_scalar(x[r * ld + c], inv, bits, round_mode, u24);
+            }
+        }
+    }
+
+    if (codes_tr) {
+        if (scale_mode == ORC_PER_TENSOR) {
+            float delta, inv;
+            orc_scale_from_absmax(m_tensor, bits, &delta, &inv);
+            scale_tr[0] = delta;
+        } else {
+            orc_absmax_cols(x, rows, cols, ld, scale_tr);
+        }
+#pragma omp parallel for schedule(static)
+        for (int64_t c = 0; c < cols; ++c) {
+            float delta, inv;
+            if (scale_mode == ORC_PER_TENSOR) {
+                orc_scale_from_absmax(m_tensor, bits, &delta, &inv);
+            } else {
+                orc_scale_from_absmax(scale_tr[c], bits, &delta, &inv);
+                scale_tr[c] = delta;
+            }
+            for (int64_t r = 0; r < rows; ++r) {
+                uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
+                uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, i) : 0u;
+                codes_tr[c * rows + r] =
+                    (int8_t)orc_quantize_scalar(x[r * ld + c], inv, bits, round_mode, u24);
+            }
+        }
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------------- */
+/* Sec. 2.2.2: product of two code matrices, both stored with the           */
+/* contracted axis contiguous:  acc[i,j] = sum_k a[i,k] * b[j,k].           */
+/* The sum is formed in 64 bits; the return value counts entries that do    */
+/* not fit in 32 bits (a caller precondition, 0 in every valid use).        */
+/* ---------------------------------------------------------------------- */
+int64_t orc_gemm_i8_nt(const int8_t *a, const int8_t *b, int64_t M, int64_t N, int64_t Kc,
+                       int32_t *acc)
+{
+    int64_t overflow = 0;
+#pragma omp parallel for schedule(static) reduction(+ : overflow)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            int64_t s = 0;
+            for (int64_t k = 0; k < Kc; ++k)
+                s += (int64_t)a[i * Kc + k] * (int64_t)b[j * Kc + k];
+            if (s > INT32_MAX || s < INT32_MIN) overflow += 1;
+            acc[i * N + j] = (int32_t)s;
+        }
+    return overflow;
+}
+
+/*
+ * Value of the product of the two quantized matrices: the integer sum times
+ * the two step sizes,  out[i,j] = float(acc[i,j]) * (s_row[i] * s_col[j]),
+ * each operation one binary32 rounding, the scale product formed first.
+ * row_stride / col_stride are 0 for a per-tensor scale and 1 for per-row.
+ */
+void orc_dequant(const int32_t *acc, int64_t M, int64_t N,
+                 const float *s_row, int row_stride, const float *s_col, int col_stride,
+                 float *out)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            float s = s_row[i * row_stride] * s_col[j * col_stride];
+            out[i * N + j] = (float)acc[i * N + j] * s;
+        }
+}
+
+/* ---------------------------------------------------------------------- */
+/* One quantization point = (bits, scale mode, rounding mode, seed, id,    */
+/* index offset): the paper's (Delta, eps) for one operand.                 */
+/* ---------------------------------------------------------------------- */
+typedef struct {
+    int32_t bits;
+    int32_t scale_mode;
+    int32_t round_mode;
+    int32_t reserved;
+    uint64_t seed;
+    uint64_t tensor_id;
+    uint64_t index_offset;
+} orc_qspec;
+
+/*
+ * Alg. 1:  Y[T,N] = Q(A) Q(W)^T.  Caller provides scratch for the codes,
+ * scales (T and N floats, of which one is used per tensor) and accumulators,
+ * which are outputs too.  Returns the overflow count of the product.
+ */
+int64_t orc_qlinear_fwd(const float *A, const float *W, int64_t T, int64_t N, int64_t K,
+                        const orc_qspec *qa, const orc_qspec *qw,
+                        int8_t *codes_a /*[T,K]*/, float *scale_a,
+                        int8_t *codes_w /*[N,K]*/, float *scale_w,
+                        int32_t *acc /*[T,N]*/, float *Y /*[T,N]*/)
+{
+    orc_sr_quantize(A, T, K, K, qa->bits, qa->scale_mode, qa->round_mode, qa->seed, qa->tensor_id,
+                    qa->index_offset, codes_a, scale_a, NULL, NULL);
+    orc_sr_quantize(W, N, K, K, qw->bits, qw->scale_mode, qw->round_mode, qw->seed, qw->tensor_id,
+                    qw->index_offset, codes_w, scale_w, NULL, NULL);
+    int64_t ov = orc_gemm_i8_nt(codes_a, codes_w, T, N, K, acc);
+    orc_dequant(acc, T, N, scale_a, qa->scale_mode == ORC_PER_ROW, scale_w,
+                qw->scale_mode == ORC_PER_ROW, Y);
+    return ov;
+}
+
+/*
+ * Alg. 2, input gradient:  dA[T,K] = Q(dY) Q(W).  The contraction runs over
+ * N, so W is taken in its transposed layout W^T[K,N] (per-row scale = one
+ * per input feature k).
+ */
+int64_t orc_qlinear_bwd_input(const float *dY, const float *W, int64_t T, int64_t N, int64_t K,
+                              const orc_qspec *qdy, const orc_qspec *qw,
+                              int8_t *codes_dy /*[T,N]*/, float *scale_dy,
+                              int8_t *codes_wt /*[K,N]*/, float *scale_wt,
+                              int32_t *acc /*[T,K]*/, float *dA /*[T,K]*/)
+{
+    orc_sr_quantize(dY, T, N, N, qdy->bits, qdy->scale_mode, qdy->round_mode, qdy->seed,
+                    qdy->tensor_id, qdy->index_offset, codes_dy, scale_dy, NULL, NULL);
+    orc_sr_quantize(W, N, K, K, qw->bits, qw->scale_mode, qw->round_mode, qw->seed, qw->tensor_id,
+                    qw->index_offset, NULL, NULL, codes_wt, scale_wt);
+    int64_t ov = orc_gemm_i8_nt(codes_dy, codes_wt, T, K, N, acc);
+    orc_dequant(acc, T, K, scale_dy, qdy->scale_mode == ORC_PER_ROW, scale_wt,
+                qw->scale_mode == ORC_PER_ROW, dA);
+    return ov;
+}
+
+/*
+ * Alg. 2, weight gradient:  dW[N,K] = Q(dY)^T Q(A).  The contraction runs
+ * over the T samples (the axis along which the SR noise averages out), so
+ * both operands are taken in their transposed layouts dY^T[N,T], A^T[K,T].
+ */
+int64_t orc_qlinear_bwd_weight(const float *dY, const float *A, int64_t T, int64_t N, int64_t K,
+                               const orc_qspec *qdy, const orc_qspec *qa,
+                               int8_t *codes_dyt /*[N,T]*/, float *scale_dyt,
+                               int8_t *codes_at /*[K,T]*/, float *scale_at,
+                               int32_t *acc /*[N,K]*/, float *dW /*[N,K]*/)
+{
+    orc_sr_quantize(dY, T, N, N, qdy->bits, qdy->scale_mode, qdy->round_mode, qdy->seed,
+                    qdy->tensor_id, qdy->index_offset, NULL, NULL, codes_dyt, scale_dyt);
+    orc_sr_quantize(A, T, K, K, qa->bits, qa->scale_mode, qa->round_mode, qa->seed, qa->tensor_id,
+                    qa->index_offset, NULL, NULL, codes_at, scale_at);
+    int64_t ov = orc_gemm_i8_nt(codes_dyt, codes_at, N, K, T, acc);
+    orc_dequant(acc, N, K, scale_dyt, qdy->scale_mode == ORC_PER_ROW, scale_at,
+                qa->scale_mode == ORC_PER_ROW, dW);
+    return ov;
+}
+
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
