@@ -1,0 +1,179 @@
+/*
+ * srq — stochastically-rounded quantized linear layer for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libsrq.so.  The operations are those of the paper "Training with
+ * Fewer Bits: Unlocking Edge LLMs Training with Stochastic Rounding":
+ * the threshold quantizer Q_D(x, eps) (Def. 1) in its round-to-nearest
+ * (Def. 2) and stochastic-rounding (Def. 3) forms, the mixed-precision
+ * forward pass (Alg. 1) and the mixed-precision backward pass (Alg. 2).
+ *
+ * Conventions for every entry point
+ *   - Storage: activations A[T,K], weights W[N,K], output gradients dY[T,N],
+ *     all row-major; Y[T,N] = Q(A) Q(W)^T, dA[T,K] = Q(dY) Q(W),
+ *     dW[N,K] = Q(dY)^T Q(A).  (The paper writes W as [in,out]; this is the
+ *     same mathematics with W stored [out,in].)
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, the
+ *     workspace included.  qspec pointers and the debug struct are HOST
+ *     pointers, read before the call returns.  The library allocates no
+ *     device memory and keeps no state between calls.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL
+ *     for the default stream) and the call returns without waiting.
+ *   - Errors the host can see (null pointer, bits outside 2..8, a pitch or
+ *     pointer that breaks the alignment rules below, workspace too small,
+ *     a contraction long enough to overflow int32) return a status at once
+ *     and enqueue nothing.  Conditions only the device can see (an input
+ *     that is not finite, a bounded wait inside a kernel that ran out) are
+ *     recorded in a status word at the start of the workspace; read it with
+ *     srq_poll_status.  After such a condition the outputs are unspecified.
+ *   - Outputs are overwritten, never accumulated into.
+ *   - Alignment: input base pointers 16-byte aligned; input pitch `ld` in
+ *     elements; fp32 outputs 16-byte aligned; the workspace 256-byte aligned.
+ *     Inputs whose pitch or extent is not a multiple of 4 elements take a
+ *     slower element-wise path with identical results.
+ *
+ * Step size.  The paper leaves the precision level D of Def. 1 free.  Here
+ * D_g = absmax_g / qmax with qmax = 2^(bits-1) - 1 and codes in
+ * [-qmax, qmax]; x / D is evaluated as x * (qmax / absmax_g), one binary32
+ * multiply.  The group g is the whole tensor (SRQ_PER_TENSOR) or one row of
+ * the code layout being written (SRQ_PER_ROW), i.e. one index of the
+ * dimension that is NOT contracted in the product that consumes the codes.
+ *
+ * Thresholds.  eps of Def. 3 is never stored: element x[r,c] uses
+ * eps = u24 * 2^-24, where u24 is the top 24 bits of word (i & 3) of
+ * Philox4x32-10 with counter {lo(i>>2), hi(i>>2), lo(tensor_id),
+ * hi(tensor_id)} and key {lo(seed), hi(seed)}, i = index_offset + r*cols + c.
+ * SR rounds up iff eps < frac(x/D); RTN rounds up iff frac(x/D) >= 1/2.
+ * The same (seed, tensor_id, index_offset, bits, scale, round) reproduces the
+ * same codes, which is how one quantized W serves forward and backward.
+ */
+#ifndef SRQ_H
+#define SRQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SRQ_OK = 0,
+    SRQ_ERR_INVALID_ARG = 1,   /* null pointer, bad enum, bad extent, misaligned pointer/pitch */
+    SRQ_ERR_UNSUPPORTED = 2,   /* bits outside 2..8 */
+    SRQ_ERR_WORKSPACE = 3,     /* workspace smaller than srq_*_workspace_bytes says */
+    SRQ_ERR_ACC_OVERFLOW = 4,  /* contraction length * qmax_a * qmax_b >= 2^31 */
+    SRQ_ERR_CUDA = 5,          /* a CUDA call failed (launch, tensor-map encode, copy) */
+    SRQ_ERR_NONFINITE = 6,     /* device: an input group has a NaN or infinite absmax */
+    SRQ_ERR_TIMEOUT = 7        /* device: a bounded wait in a kernel ran out */
+} srq_status_t;
+
+typedef enum { SRQ_F32 = 0, SRQ_BF16 = 1 } srq_dtype_t;
+typedef enum { SRQ_PER_TENSOR = 0, SRQ_PER_ROW = 1 } srq_scale_t;
+typedef enum { SRQ_SR = 0, SRQ_RTN = 1 } srq_round_t;
+
+/* One quantization point: the paper's (D, eps) pair for one operand of one pass
+ * (five per layer: A and W forward; A, W and dY backward). */
+typedef struct {
+    int32_t bits;          /* 2..8; codes are stored one per int8 whatever the width */
+    int32_t scale;         /* srq_scale_t */
+    int32_t round;         /* srq_round_t */
+    int32_t reserved;      /* 0 */
+    uint64_t seed;         /* Philox key; one per training step */
+    uint64_t tensor_id;    /* Philox counter words 2-3; one per (layer, operand, pass) */
+    uint64_t index_offset; /* added to the flat index; first_row*cols for a row shard */
+} srq_qspec_t;
+
+/* Optional copies of what a layer pass fed to its product: dense code matrices in the layout
+ * the product consumed (contracted axis contiguous), their step sizes, and the int32 sums.
+ * Any member may be NULL.  All are device pointers. */
+typedef struct {
+    int8_t *codes_a;   /* first operand  [M, Kc] */
+    float *scale_a;    /* [1] or [M] */
+    int8_t *codes_b;   /* second operand [Nn, Kc] */
+    float *scale_b;    /* [1] or [Nn] */
+    int32_t *acc;      /* [M, Nn] */
+} srq_debug_out_t;
+
+/* Bytes of workspace sr_quantize needs for a [rows, cols] input. */
+size_t srq_quantize_workspace_bytes(int64_t rows, int64_t cols);
+
+/* Bytes of workspace srq_gemm_i8 needs for an [M, N] output (split accumulators). */
+size_t srq_gemm_workspace_bytes(int64_t M, int64_t N);
+
+/* Bytes of workspace that suffices for any one of the qlinear_* calls on a layer with
+ * T tokens, N output and K input features. */
+size_t srq_workspace_bytes(int64_t T, int64_t N, int64_t K);
+
+/*
+ * Def. 1-3 applied element-wise to x[rows, cols] (row pitch ld elements, type dt).
+ * Writes int8 codes in the row-major layout codes_rm[rows, ld_rm] with scale_rm ([1] per
+ * tensor, [rows] per row) and/or the transposed layout codes_tr[cols, ld_tr] with scale_tr
+ * ([1] per tensor, [cols] per row of that layout, i.e. per column of x).  A NULL code
+ * pointer skips that layout (its scale pointer is then ignored).  Per tensor both layouts
+ * hold the same codes; per row they differ in step size but share each element's threshold.
+ * ld_rm >= cols, ld_tr >= rows; padding bytes are left untouched.
+ */
+srq_status_t sr_quantize(const void *x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+                         const srq_qspec_t *q,
+                         int8_t *codes_rm, int64_t ld_rm, float *scale_rm,
+                         int8_t *codes_tr, int64_t ld_tr, float *scale_tr,
+                         void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * The product of two quantized matrices (mixed-precision matmul subsection): int8 codes
+ * a[M, Kc] (pitch lda) and b[N, Kc] (pitch ldb), both with the contracted axis contiguous,
+ * multiplied on the tensor cores with exact int32 accumulation, then
+ *     out[i, j] = float(acc[i, j]) * (s_row[i * row_stride] * s_col[j * col_stride])
+ * (each operation one binary32 rounding).  row_stride / col_stride are 0 for a per-tensor
+ * step size and 1 for per-row.  acc_out, if not NULL, also receives the raw sums [M, N]
+ * (pitch N).  lda and ldb must be multiples of 16 and a, b 16-byte aligned (TMA rule).
+ * Requires Kc * 127 * 127 < 2^31 unless the caller passes smaller code ranges through the
+ * qlinear_* entry points, which check the bound for their own bit widths.
+ */
+srq_status_t srq_gemm_i8(const int8_t *a, int64_t lda, const int8_t *b, int64_t ldb,
+                         int64_t M, int64_t N, int64_t Kc,
+                         const float *s_row, int32_t row_stride,
+                         const float *s_col, int32_t col_stride,
+                         float *out, int64_t ldo, int32_t *acc_out,
+                         void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Alg. 1: Y[T,N] = Q(A) Q(W)^T.  qA, qW are the forward quantization points of A and W.
+ * Per row: A per token, W per output feature. */
+srq_status_t qlinear_fwd(const void *A, const void *W, srq_dtype_t dt,
+                         int64_t T, int64_t N, int64_t K,
+                         const srq_qspec_t *qA, const srq_qspec_t *qW,
+                         float *Y, const srq_debug_out_t *dbg,
+                         void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Alg. 2, input gradient: dA[T,K] = Q(dY) Q(W).  The contraction runs over N, so Q(W) is
+ * written in its transposed layout [K,N].  Per row: dY per token, W per input feature. */
+srq_status_t qlinear_bwd_input(const void *dY, const void *W, srq_dtype_t dt,
+                               int64_t T, int64_t N, int64_t K,
+                               const srq_qspec_t *qdY, const srq_qspec_t *qW,
+                               float *dA, const srq_debug_out_t *dbg,
+                               void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Alg. 2, weight gradient: dW[N,K] = Q(dY)^T Q(A).  The contraction runs over the T tokens;
+ * both operands are written in their transposed layouts [N,T] and [K,T].  Per row: dY per
+ * output feature, A per input feature. */
+srq_status_t qlinear_bwd_weight(const void *dY, const void *A, srq_dtype_t dt,
+                                int64_t T, int64_t N, int64_t K,
+                                const srq_qspec_t *qdY, const srq_qspec_t *qA,
+                                float *dW, const srq_debug_out_t *dbg,
+                                void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Waits for the stream, then returns the device status word of the workspace: SRQ_OK, or the
+ * first device-side condition recorded by the calls that used this workspace since its header
+ * was last cleared (every entry point clears it when it starts). */
+srq_status_t srq_poll_status(void *ws, void *cuda_stream);
+
+/* Static, human-readable name of a status. */
+const char *srq_status_string(srq_status_t s);
+
+/* Number of kernels the library has launched in this process (for launch accounting). */
+uint64_t srq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SRQ_H */

@@ -1,1 +1,13 @@
-"""B200-native stochastically-rounded quantized linear layer (C-ABI library + thin binding)."""
+"""B200-native stochastically-rounded quantized linear layer.
+
+The product is the C-ABI library ``libsrq.so`` (hand-written CUDA for sm_100a, declared in
+``include/srq.h``); this package holds its sources (``csrc/``), the build step (``build.py``),
+a thin ctypes binding with the same entry-point names (``binding.py``) and the seeded synthetic
+input recipes (``synth.py``).  Importing the package loads nothing; the first call loads the
+library and raises if it has not been built.
+"""
+from .binding import (BF16, F32, PER_ROW, PER_TENSOR, RTN, SR, DebugOut, QSpec, SrqError,  # noqa: F401
+                      launch_count, new_workspace, qlinear_bwd_input, qlinear_bwd_weight,
+                      qlinear_fwd, sr_quantize, srq_gemm_i8, srq_gemm_workspace_bytes,
+                      srq_poll_status, srq_quantize_workspace_bytes, srq_workspace_bytes,
+                      status_string)

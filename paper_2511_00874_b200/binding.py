@@ -1,0 +1,256 @@
+"""Thin ctypes binding of libsrq.so: argument marshalling only.
+
+Every function has the name and argument order of the C entry point it calls (see
+``include/srq.h``); tensors are torch CUDA tensors used purely as device memory, and the
+current torch stream is passed as the CUDA stream.  There is no fallback: if the shared
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libsrq.so")
+
+# enums of srq.h
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_ACC_OVERFLOW, ERR_CUDA, ERR_NONFINITE, \
+    ERR_TIMEOUT = range(8)
+F32, BF16 = 0, 1
+PER_TENSOR, PER_ROW = 0, 1
+SR, RTN = 0, 1
+
+EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
+           "sr_quantize", "srq_gemm_i8", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight",
+           "srq_poll_status", "srq_status_string", "srq_launch_count"]
+
+
+class SrqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class _QSpec(ctypes.Structure):
+    _fields_ = [("bits", ctypes.c_int32), ("scale", ctypes.c_int32), ("round", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("seed", ctypes.c_uint64),
+                ("tensor_id", ctypes.c_uint64), ("index_offset", ctypes.c_uint64)]
+
+
+class _DebugOut(ctypes.Structure):
+    _fields_ = [("codes_a", ctypes.c_void_p), ("scale_a", ctypes.c_void_p),
+                ("codes_b", ctypes.c_void_p), ("scale_b", ctypes.c_void_p),
+                ("acc", ctypes.c_void_p)]
+
+
+@dataclass
+class QSpec:
+    """One quantization point (bits, scale mode, rounding mode, seed, tensor_id, index_offset)."""
+    bits: int = 8
+    scale: int = PER_TENSOR
+    round: int = SR
+    seed: int = 0
+    tensor_id: int = 0
+    index_offset: int = 0
+
+    def c(self) -> _QSpec:
+        return _QSpec(self.bits, self.scale, self.round, 0, self.seed, self.tensor_id,
+                      self.index_offset)
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libsrq.so (built in-tree by ``build.py``); raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                           "`python -m paper_2511_00874_b200.build` (there is no fallback path)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
+    qp = ctypes.POINTER(_QSpec)
+    dp = ctypes.POINTER(_DebugOut)
+    L.srq_quantize_workspace_bytes.argtypes = [i64, i64]
+    L.srq_quantize_workspace_bytes.restype = sz
+    L.srq_gemm_workspace_bytes.argtypes = [i64, i64]
+    L.srq_gemm_workspace_bytes.restype = sz
+    L.srq_workspace_bytes.argtypes = [i64, i64, i64]
+    L.srq_workspace_bytes.restype = sz
+    L.sr_quantize.argtypes = [vp, ctypes.c_int, i64, i64, i64, qp, vp, i64, vp, vp, i64, vp, vp, sz, vp]
+    L.sr_quantize.restype = ctypes.c_int
+    L.srq_gemm_i8.argtypes = [vp, i64, vp, i64, i64, i64, i64, vp, i32, vp, i32, vp, i64, vp, vp, sz, vp]
+    L.srq_gemm_i8.restype = ctypes.c_int
+    for name in ("qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight"):
+        f = getattr(L, name)
+        f.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, qp, qp, vp, dp, vp, sz, vp]
+        f.restype = ctypes.c_int
+    L.srq_poll_status.argtypes = [vp, vp]
+    L.srq_poll_status.restype = ctypes.c_int
+    L.srq_status_string.argtypes = [ctypes.c_int]
+    L.srq_status_string.restype = ctypes.c_char_p
+    L.srq_launch_count.argtypes = []
+    L.srq_launch_count.restype = ctypes.c_uint64
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().srq_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(lib().srq_launch_count())
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise SrqError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _dtype_of(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"inputs must be float32 or bfloat16, got {t.dtype}")
+
+
+def _dev2d(t: torch.Tensor, name: str) -> None:
+    if not t.is_cuda or t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError(f"{name} must be a 2-D CUDA tensor with unit inner stride")
+
+
+def srq_quantize_workspace_bytes(rows: int, cols: int) -> int:
+    return int(lib().srq_quantize_workspace_bytes(rows, cols))
+
+
+def srq_gemm_workspace_bytes(M: int, N: int) -> int:
+    return int(lib().srq_gemm_workspace_bytes(M, N))
+
+
+def srq_workspace_bytes(T: int, N: int, K: int) -> int:
+    return int(lib().srq_workspace_bytes(T, N, K))
+
+
+def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """Device buffer for a workspace (torch's allocator returns 512-byte aligned blocks)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def sr_quantize(x: torch.Tensor, q: QSpec, codes_rm: Optional[torch.Tensor] = None,
+                scale_rm: Optional[torch.Tensor] = None, codes_tr: Optional[torch.Tensor] = None,
+                scale_tr: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None) -> None:
+    """Def. 1-3 on x[rows, cols]; code tensors are int8 [rows, >=cols] / [cols, >=rows] views."""
+    _dev2d(x, "x")
+    rows, cols = x.shape
+    if ws is None:
+        ws = new_workspace(srq_quantize_workspace_bytes(rows, cols), x.device)
+    cq = q.c()
+    st = lib().sr_quantize(x.data_ptr(), _dtype_of(x), rows, cols, x.stride(0), ctypes.byref(cq),
+                           _ptr(codes_rm), codes_rm.stride(0) if codes_rm is not None else 0,
+                           _ptr(scale_rm),
+                           _ptr(codes_tr), codes_tr.stride(0) if codes_tr is not None else 0,
+                           _ptr(scale_tr), ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "sr_quantize")
+
+
+def srq_gemm_i8(a: torch.Tensor, b: torch.Tensor, s_row: torch.Tensor, s_col: torch.Tensor,
+                out: torch.Tensor, acc_out: Optional[torch.Tensor] = None,
+                ws: Optional[torch.Tensor] = None) -> None:
+    """out[M,N] = float(a[M,Kc] . b[N,Kc]^T) * (s_row x s_col); a, b int8 with pitch % 16 == 0."""
+    _dev2d(a, "a")
+    _dev2d(b, "b")
+    M, Kc = a.shape
+    N = b.shape[0]
+    if ws is None:
+        ws = new_workspace(srq_gemm_workspace_bytes(M, N), a.device)
+    st = lib().srq_gemm_i8(a.data_ptr(), a.stride(0), b.data_ptr(), b.stride(0), M, N, Kc,
+                           s_row.data_ptr(), int(s_row.numel() != 1), s_col.data_ptr(),
+                           int(s_col.numel() != 1), out.data_ptr(), out.stride(0), _ptr(acc_out),
+                           ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "srq_gemm_i8")
+
+
+@dataclass
+class DebugOut:
+    """Optional device tensors that receive what a layer pass fed to its product."""
+    codes_a: Optional[torch.Tensor] = None
+    scale_a: Optional[torch.Tensor] = None
+    codes_b: Optional[torch.Tensor] = None
+    scale_b: Optional[torch.Tensor] = None
+    acc: Optional[torch.Tensor] = None
+
+    def c(self) -> _DebugOut:
+        return _DebugOut(_ptr(self.codes_a), _ptr(self.scale_a), _ptr(self.codes_b),
+                         _ptr(self.scale_b), _ptr(self.acc))
+
+
+def _layer(fn_name: str, X0: torch.Tensor, X1: torch.Tensor, T: int, N: int, K: int, q0: QSpec,
+           q1: QSpec, out: torch.Tensor, dbg: Optional[DebugOut], ws: Optional[torch.Tensor]) -> None:
+    for t, n in ((X0, "first operand"), (X1, "second operand")):
+        _dev2d(t, n)
+        if not t.is_contiguous():
+            raise ValueError(f"{n} must be contiguous")
+    if _dtype_of(X0) != _dtype_of(X1):
+        raise TypeError("both operands must have the same dtype")
+    if out.dtype != torch.float32 or not out.is_contiguous():
+        raise TypeError("output must be a contiguous float32 tensor")
+    if ws is None:
+        ws = new_workspace(srq_workspace_bytes(T, N, K), X0.device)
+    c0, c1 = q0.c(), q1.c()
+    cd = dbg.c() if dbg is not None else None
+    st = getattr(lib(), fn_name)(X0.data_ptr(), X1.data_ptr(), _dtype_of(X0), T, N, K,
+                                 ctypes.byref(c0), ctypes.byref(c1), out.data_ptr(),
+                                 ctypes.byref(cd) if cd is not None else None,
+                                 ws.data_ptr(), ws.numel(), _stream())
+    _check(st, fn_name)
+
+
+def qlinear_fwd(A: torch.Tensor, W: torch.Tensor, qA: QSpec, qW: QSpec, Y: torch.Tensor,
+                dbg: Optional[DebugOut] = None, ws: Optional[torch.Tensor] = None) -> None:
+    """Alg. 1: Y[T,N] = Q(A[T,K]) Q(W[N,K])^T."""
+    T, K = A.shape
+    N, K2 = W.shape
+    if K != K2 or tuple(Y.shape) != (T, N):
+        raise ValueError("qlinear_fwd: shapes must be A[T,K], W[N,K], Y[T,N]")
+    _layer("qlinear_fwd", A, W, T, N, K, qA, qW, Y, dbg, ws)
+
+
+def qlinear_bwd_input(dY: torch.Tensor, W: torch.Tensor, qdY: QSpec, qW: QSpec, dA: torch.Tensor,
+                      dbg: Optional[DebugOut] = None, ws: Optional[torch.Tensor] = None) -> None:
+    """Alg. 2: dA[T,K] = Q(dY[T,N]) Q(W[N,K])."""
+    T, N = dY.shape
+    N2, K = W.shape
+    if N != N2 or tuple(dA.shape) != (T, K):
+        raise ValueError("qlinear_bwd_input: shapes must be dY[T,N], W[N,K], dA[T,K]")
+    _layer("qlinear_bwd_input", dY, W, T, N, K, qdY, qW, dA, dbg, ws)
+
+
+def qlinear_bwd_weight(dY: torch.Tensor, A: torch.Tensor, qdY: QSpec, qA: QSpec, dW: torch.Tensor,
+                       dbg: Optional[DebugOut] = None, ws: Optional[torch.Tensor] = None) -> None:
+    """Alg. 2: dW[N,K] = Q(dY[T,N])^T Q(A[T,K])."""
+    T, N = dY.shape
+    T2, K = A.shape
+    if T != T2 or tuple(dW.shape) != (N, K):
+        raise ValueError("qlinear_bwd_weight: shapes must be dY[T,N], A[T,K], dW[N,K]")
+    _layer("qlinear_bwd_weight", dY, A, T, N, K, qdY, qA, dW, dbg, ws)
+
+
+def srq_poll_status(ws: torch.Tensor) -> int:
+    """Synchronises the current stream and returns the device status word of ``ws``."""
+    return int(lib().srq_poll_status(ws.data_ptr(), _stream()))

@@ -1,0 +1,236 @@
+// C-ABI entry points of libsrq: argument checks, workspace carving and launch sequencing.
+// All arithmetic is in quantize.cu and gemm_i8.cu.
+#include "common.cuh"
+
+using namespace srq;
+
+namespace {
+
+inline int qmax_of(int bits) { return (1 << (bits - 1)) - 1; }
+
+srq_status_t check_qspec(const srq_qspec_t* q) {
+    if (!q) return SRQ_ERR_INVALID_ARG;
+    if (q->bits < 2 || q->bits > 8) return SRQ_ERR_UNSUPPORTED;
+    if (q->scale != SRQ_PER_TENSOR && q->scale != SRQ_PER_ROW) return SRQ_ERR_INVALID_ARG;
+    if (q->round != SRQ_SR && q->round != SRQ_RTN) return SRQ_ERR_INVALID_ARG;
+    return SRQ_OK;
+}
+
+inline bool aligned_to(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+inline int64_t pitch16(int64_t n) { return (n + 15) / 16 * 16; }
+inline size_t f32_block(int64_t n) { return align_up((size_t)n * 4); }
+
+cudaError_t clear_header(void* ws, cudaStream_t st) { return cudaMemsetAsync(ws, 0, sizeof(WsHeader), st); }
+
+// One operand of a layer pass: source matrix, which code layout the product needs, its spec.
+struct Operand {
+    const void* x; int64_t rows, cols;   // source extents (pitch = cols)
+    bool transposed;                     // false: codes [rows, cols]; true: codes [cols, rows]
+    const srq_qspec_t* q;
+    int64_t out_rows() const { return transposed ? cols : rows; }
+    int64_t out_cols() const { return transposed ? rows : cols; }   // contraction length
+};
+
+// Carving of a qlinear workspace.
+struct LayerPlan {
+    size_t off_scratch[2], off_scale[2], off_codes[2], off_split, total;
+    int64_t pitch;
+};
+
+LayerPlan plan_layer(const Operand& a, const Operand& b) {
+    LayerPlan p;
+    size_t o = sizeof(WsHeader);
+    const Operand* ops[2] = {&a, &b};
+    for (int i = 0; i < 2; ++i) { p.off_scratch[i] = o; o += quant_scratch_bytes(ops[i]->rows, ops[i]->cols); }
+    for (int i = 0; i < 2; ++i) { p.off_scale[i] = o; o += f32_block(ops[i]->out_rows()); }
+    p.pitch = pitch16(a.out_cols());
+    for (int i = 0; i < 2; ++i) { p.off_codes[i] = o; o += align_up((size_t)ops[i]->out_rows() * p.pitch); }
+    p.off_split = o;
+    o += gemm_splitk_bytes(a.out_rows(), b.out_rows());
+    p.total = o;
+    return p;
+}
+
+srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float* out, const srq_debug_out_t* dbg,
+                       void* ws, size_t ws_bytes, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!a.x || !b.x || !out || !ws) return SRQ_ERR_INVALID_ARG;
+    if (dt != SRQ_F32 && dt != SRQ_BF16) return SRQ_ERR_INVALID_ARG;
+    if (a.rows < 0 || a.cols < 0 || b.rows < 0 || b.cols < 0) return SRQ_ERR_INVALID_ARG;
+    srq_status_t s;
+    if ((s = check_qspec(a.q)) != SRQ_OK) return s;
+    if ((s = check_qspec(b.q)) != SRQ_OK) return s;
+    if (!aligned_to(a.x, 16) || !aligned_to(b.x, 16) || !aligned_to(out, 16) || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
+    const int64_t M = a.out_rows(), Nn = b.out_rows(), Kc = a.out_cols();
+    if (Kc != b.out_cols()) return SRQ_ERR_INVALID_ARG;
+    if ((double)Kc * qmax_of(a.q->bits) * qmax_of(b.q->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
+    const LayerPlan p = plan_layer(a, b);
+    if (ws_bytes < p.total) return SRQ_ERR_WORKSPACE;
+    if (M == 0 || Nn == 0) return SRQ_OK;
+
+    char* base = (char*)ws;
+    uint32_t* status = &((WsHeader*)ws)->status;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+
+    const Operand* ops[2] = {&a, &b};
+    int8_t* codes[2];
+    float* scales[2];
+    for (int i = 0; i < 2; ++i) {
+        const Operand& o = *ops[i];
+        codes[i] = (int8_t*)(base + p.off_codes[i]);
+        scales[i] = (float*)(base + p.off_scale[i]);
+        QuantArgs qa;
+        qa.x = o.x; qa.dt = dt; qa.rows = o.rows; qa.cols = o.cols; qa.ld = o.cols; qa.q = *o.q;
+        qa.codes_rm = o.transposed ? nullptr : codes[i]; qa.ld_rm = p.pitch; qa.scale_rm = o.transposed ? nullptr : scales[i];
+        qa.codes_tr = o.transposed ? codes[i] : nullptr; qa.ld_tr = p.pitch; qa.scale_tr = o.transposed ? scales[i] : nullptr;
+        if (Kc > 0 && launch_quantize(qa, carve_quant_scratch(base + p.off_scratch[i], o.rows, o.cols), status, st) != cudaSuccess)
+            return SRQ_ERR_CUDA;
+    }
+    if (Kc == 0) {   // empty contraction: the product is zero
+        return cudaMemset2DAsync(out, (size_t)Nn * 4, 0, (size_t)Nn * 4, (size_t)M, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+    }
+
+    GemmArgs g;
+    g.a = codes[0]; g.lda = p.pitch; g.b = codes[1]; g.ldb = p.pitch;
+    g.M = M; g.N = Nn; g.Kc = Kc;
+    g.s_row = scales[0]; g.row_stride = a.q->scale == SRQ_PER_ROW;
+    g.s_col = scales[1]; g.col_stride = b.q->scale == SRQ_PER_ROW;
+    g.out = out; g.ldo = Nn; g.acc_out = dbg ? dbg->acc : nullptr;
+    g.splitk_ws = base + p.off_split; g.splitk_ws_bytes = p.total - p.off_split;
+    if ((s = launch_gemm_i8(g, status, st)) != SRQ_OK) return s;
+
+    if (dbg) {
+        const int64_t rows[2] = {M, Nn};
+        int8_t* dcodes[2] = {dbg->codes_a, dbg->codes_b};
+        float* dscale[2] = {dbg->scale_a, dbg->scale_b};
+        for (int i = 0; i < 2; ++i) {
+            if (dcodes[i] && cudaMemcpy2DAsync(dcodes[i], (size_t)Kc, codes[i], (size_t)p.pitch, (size_t)Kc, (size_t)rows[i],
+                                               cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return SRQ_ERR_CUDA;
+            const size_t n = ops[i]->q->scale == SRQ_PER_ROW ? (size_t)rows[i] : 1;
+            if (dscale[i] && cudaMemcpyAsync(dscale[i], scales[i], n * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return SRQ_ERR_CUDA;
+        }
+    }
+    return SRQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t srq_quantize_workspace_bytes(int64_t rows, int64_t cols) {
+    if (rows < 0 || cols < 0) return 0;
+    return sizeof(WsHeader) + quant_scratch_bytes(rows, cols);
+}
+
+size_t srq_gemm_workspace_bytes(int64_t M, int64_t N) {
+    if (M < 0 || N < 0) return 0;
+    return sizeof(WsHeader) + gemm_splitk_bytes(M, N);
+}
+
+size_t srq_workspace_bytes(int64_t T, int64_t N, int64_t K) {
+    if (T < 0 || N < 0 || K < 0) return 0;
+    srq_qspec_t q{};
+    const Operand fa{(void*)1, T, K, false, &q}, fw{(void*)1, N, K, false, &q};
+    const Operand iy{(void*)1, T, N, false, &q}, iw{(void*)1, N, K, true, &q};
+    const Operand wy{(void*)1, T, N, true, &q}, wa{(void*)1, T, K, true, &q};
+    size_t m = plan_layer(fa, fw).total;
+    const size_t m1 = plan_layer(iy, iw).total, m2 = plan_layer(wy, wa).total;
+    if (m1 > m) m = m1;
+    if (m2 > m) m = m2;
+    return m;
+}
+
+srq_status_t sr_quantize(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, const srq_qspec_t* q,
+                         int8_t* codes_rm, int64_t ld_rm, float* scale_rm, int8_t* codes_tr, int64_t ld_tr, float* scale_tr,
+                         void* ws, size_t ws_bytes, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!x || !ws || rows < 0 || cols < 0 || ld < cols) return SRQ_ERR_INVALID_ARG;
+    if (dt != SRQ_F32 && dt != SRQ_BF16) return SRQ_ERR_INVALID_ARG;
+    srq_status_t s = check_qspec(q);
+    if (s != SRQ_OK) return s;
+    if (!codes_rm && !codes_tr) return SRQ_ERR_INVALID_ARG;
+    if (codes_rm && (!scale_rm || ld_rm < cols)) return SRQ_ERR_INVALID_ARG;
+    if (codes_tr && (!scale_tr || ld_tr < rows)) return SRQ_ERR_INVALID_ARG;
+    if (!aligned_to(x, 16) || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
+    if (ws_bytes < srq_quantize_workspace_bytes(rows, cols)) return SRQ_ERR_WORKSPACE;
+    if (rows == 0 || cols == 0) return SRQ_OK;
+    uint32_t* status = &((WsHeader*)ws)->status;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    QuantArgs a;
+    a.x = x; a.dt = dt; a.rows = rows; a.cols = cols; a.ld = ld; a.q = *q;
+    a.codes_rm = codes_rm; a.ld_rm = ld_rm; a.scale_rm = scale_rm;
+    a.codes_tr = codes_tr; a.ld_tr = ld_tr; a.scale_tr = scale_tr;
+    const QuantScratch sc = carve_quant_scratch((char*)ws + sizeof(WsHeader), rows, cols);
+    return launch_quantize(a, sc, status, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+}
+
+srq_status_t srq_gemm_i8(const int8_t* a, int64_t lda, const int8_t* b, int64_t ldb, int64_t M, int64_t N, int64_t Kc,
+                         const float* s_row, int32_t row_stride, const float* s_col, int32_t col_stride,
+                         float* out, int64_t ldo, int32_t* acc_out, void* ws, size_t ws_bytes, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!a || !b || !s_row || !s_col || !out || !ws) return SRQ_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || Kc <= 0 || lda < Kc || ldb < Kc || ldo < N) return SRQ_ERR_INVALID_ARG;
+    if ((row_stride != 0 && row_stride != 1) || (col_stride != 0 && col_stride != 1)) return SRQ_ERR_INVALID_ARG;
+    if (!aligned_to(a, 16) || !aligned_to(b, 16) || lda % 16 || ldb % 16 || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
+    if ((double)Kc * 127.0 * 127.0 >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
+    if (ws_bytes < sizeof(WsHeader)) return SRQ_ERR_WORKSPACE;
+    if (M == 0 || N == 0) return SRQ_OK;
+    uint32_t* status = &((WsHeader*)ws)->status;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    GemmArgs g;
+    g.a = a; g.lda = lda; g.b = b; g.ldb = ldb; g.M = M; g.N = N; g.Kc = Kc;
+    g.s_row = s_row; g.row_stride = row_stride; g.s_col = s_col; g.col_stride = col_stride;
+    g.out = out; g.ldo = ldo; g.acc_out = acc_out;
+    g.splitk_ws = (char*)ws + sizeof(WsHeader); g.splitk_ws_bytes = ws_bytes - sizeof(WsHeader);
+    return launch_gemm_i8(g, status, st);
+}
+
+srq_status_t qlinear_fwd(const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
+                         const srq_qspec_t* qA, const srq_qspec_t* qW, float* Y, const srq_debug_out_t* dbg,
+                         void* ws, size_t ws_bytes, void* cuda_stream) {
+    const Operand a{A, T, K, false, qA}, b{W, N, K, false, qW};
+    return run_layer(a, b, dt, Y, dbg, ws, ws_bytes, cuda_stream);
+}
+
+srq_status_t qlinear_bwd_input(const void* dY, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
+                               const srq_qspec_t* qdY, const srq_qspec_t* qW, float* dA, const srq_debug_out_t* dbg,
+                               void* ws, size_t ws_bytes, void* cuda_stream) {
+    const Operand a{dY, T, N, false, qdY}, b{W, N, K, true, qW};
+    return run_layer(a, b, dt, dA, dbg, ws, ws_bytes, cuda_stream);
+}
+
+srq_status_t qlinear_bwd_weight(const void* dY, const void* A, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
+                                const srq_qspec_t* qdY, const srq_qspec_t* qA, float* dW, const srq_debug_out_t* dbg,
+                                void* ws, size_t ws_bytes, void* cuda_stream) {
+    const Operand a{dY, T, N, true, qdY}, b{A, T, K, true, qA};
+    return run_layer(a, b, dt, dW, dbg, ws, ws_bytes, cuda_stream);
+}
+
+srq_status_t srq_poll_status(void* ws, void* cuda_stream) {
+    if (!ws) return SRQ_ERR_INVALID_ARG;
+    uint32_t v = 0;
+    if (cudaMemcpyAsync(&v, &((WsHeader*)ws)->status, 4, cudaMemcpyDeviceToHost, (cudaStream_t)cuda_stream) != cudaSuccess)
+        return SRQ_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return SRQ_ERR_CUDA;
+    return (srq_status_t)v;
+}
+
+const char* srq_status_string(srq_status_t s) {
+    switch (s) {
+        case SRQ_OK: return "ok";
+        case SRQ_ERR_INVALID_ARG: return "invalid argument";
+        case SRQ_ERR_UNSUPPORTED: return "unsupported bit width";
+        case SRQ_ERR_WORKSPACE: return "workspace too small";
+        case SRQ_ERR_ACC_OVERFLOW: return "contraction too long for int32 accumulation";
+        case SRQ_ERR_CUDA: return "CUDA call failed";
+        case SRQ_ERR_NONFINITE: return "input is not finite";
+        case SRQ_ERR_TIMEOUT: return "bounded wait in a kernel ran out";
+    }
+    return "unknown status";
+}
+
+uint64_t srq_launch_count(void) { return (uint64_t)g_launches; }
+
+}  // extern "C"

@@ -1,0 +1,67 @@
+// Shared declarations of the CUDA side of libsrq: workspace header, launch accounting and the
+// internal launchers that the C-ABI file strings together.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "srq.h"
+
+namespace srq {
+
+// First 256 bytes of every workspace.
+struct WsHeader {
+    uint32_t status;    // srq_status_t recorded by device code (first error wins)
+    uint32_t pad[63];
+};
+static_assert(sizeof(WsHeader) == 256, "header is one 256-byte line");
+
+constexpr size_t kAlign = 256;
+__host__ __device__ inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
+
+extern unsigned long long g_launches;   // kernels launched by this process (host counter)
+
+__device__ __forceinline__ void record_status(uint32_t* status, uint32_t code) {
+    atomicCAS(status, 0u, code);
+}
+
+// ------------------------------------------------------------------------------------------
+// Quantizer (quantize.cu)
+// ------------------------------------------------------------------------------------------
+// Scratch carved from a workspace for one sr_quantize: absmax words and reciprocal steps for
+// the row-major layout (1 or rows) and the transposed layout (1 or cols).
+struct QuantScratch {
+    uint32_t* amax_rm;   // fp32 bit patterns, zeroed before use
+    uint32_t* amax_tr;
+    float* inv_rm;
+    float* inv_tr;
+    size_t bytes;        // total bytes carved (multiple of 256)
+};
+size_t quant_scratch_bytes(int64_t rows, int64_t cols);
+QuantScratch carve_quant_scratch(void* base, int64_t rows, int64_t cols);
+
+struct QuantArgs {
+    const void* x; srq_dtype_t dt; int64_t rows, cols, ld;
+    srq_qspec_t q;
+    int8_t* codes_rm; int64_t ld_rm; float* scale_rm;
+    int8_t* codes_tr; int64_t ld_tr; float* scale_tr;
+};
+// Enqueues: clear scratch, absmax, step sizes, quantize.  `scratch` must be exclusively this
+// call's until the kernels finish.
+cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& scratch, uint32_t* status,
+                            cudaStream_t stream);
+
+// ------------------------------------------------------------------------------------------
+// int8 GEMM (gemm_i8.cu)
+// ------------------------------------------------------------------------------------------
+struct GemmArgs {
+    const int8_t* a; int64_t lda; const int8_t* b; int64_t ldb;
+    int64_t M, N, Kc;
+    const float* s_row; int32_t row_stride; const float* s_col; int32_t col_stride;
+    float* out; int64_t ldo; int32_t* acc_out;
+    void* splitk_ws; size_t splitk_ws_bytes;   // int32 [M,N] partial sums + tile tickets
+};
+size_t gemm_splitk_bytes(int64_t M, int64_t N);
+srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream);
+
+}  // namespace srq

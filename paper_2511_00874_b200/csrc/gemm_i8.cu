@@ -1,0 +1,490 @@
+// Product of two int8 code matrices on the 5th-generation tensor cores (sm_100a), with the
+// dequantizing epilogue: the paper's mixed-precision matmul (low-precision multiply, wide
+// accumulate) used by Alg. 1 (forward) and Alg. 2 (both backward products).
+//
+//   acc[i,j] = sum_k a[i,k] * b[j,k]          int8 x int8 -> int32, exact
+//   out[i,j] = float(acc[i,j]) * (s_row[i] * s_col[j])
+//
+// One persistent CTA per SM, 6 warps:
+//   warp 0      TMA producer: 128 x 128-byte tiles of a and 256 x 128-byte tiles of b into a
+//               4-stage shared-memory ring (128-byte swizzle), signalled through mbarriers
+//   warp 1      allocates TMEM and issues tcgen05.mma.kind::i8 (M128 x N256 x K32) from one
+//               thread; accumulators live in TMEM, two buffers of 256 columns, so the tensor
+//               pipe starts the next tile while the previous one is being drained
+//   warps 2-5   epilogue: tcgen05.ld the accumulator (one TMEM lane quarter per warp), convert,
+//               scale and store; or, for a split contraction, add the exact int32 partial
+//               sums into a workspace, the CTA that finishes a tile last doing the scaling
+// Ragged edges rely on TMA zero fill for loads and on bounds checks for stores.
+// Every wait is bounded by a wall-clock limit; on expiry the CTA records SRQ_ERR_TIMEOUT,
+// stops issuing work, waits (bounded) for what it has in flight, frees its TMEM and returns.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace srq {
+
+constexpr int BM = 128, BN = 256, BK = 128;          // tile extents; BK in bytes = int8 elements
+constexpr int STAGES = 4;
+constexpr int UMMA_K = 32;                             // bytes of K per tcgen05.mma.kind::i8
+constexpr int A_STAGE_BYTES = BM * BK, B_STAGE_BYTES = BN * BK;
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int TMEM_COLS = 512;                         // two accumulator buffers of BN columns
+constexpr int GEMM_THREADS = 192;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;      // 2 s
+
+struct SharedTail {                                    // after the stage ring
+    uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain;
+    uint32_t tmem_base;
+    volatile uint32_t abort_flag;
+    uint32_t last_flag[2];
+    uint32_t epi_abort;
+    float s_col[2][BN];
+};
+constexpr size_t GEMM_SMEM = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + sizeof(SharedTail);
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false if the limit passed or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t spin = 0;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int32_t x, int32_t y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem], int8 operands, int32 accumulators, issued by one thread.
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier gets one arrival once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// 32 lanes x 32 consecutive 32-bit columns: thread t of the warp receives lane (base + t).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t v[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major operand tile written by TMA with the 128-byte
+// swizzle: rows are 128 bytes, eight rows form a 1024-byte swizzle atom, so the stride between
+// 8-row groups is 1024 bytes; the leading-dimension offset is not used for this layout.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                               // leading byte offset (unused), 16-byte units
+    d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset
+    d |= (uint64_t)1 << 46;                               // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                               // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: dense, no saturation, D = s32, A = B = s8, both K-major, N x M.
+__device__ __forceinline__ constexpr uint32_t make_idesc_i8(int m, int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------
+// kernel
+// ------------------------------------------------------------------------------------------
+struct GemmParams {
+    int64_t M, N;
+    int32_t num_kb;            // 128-byte blocks along the contraction
+    int32_t splits;            // parts the contraction is cut into (1 = none)
+    int32_t tiles_m, tiles_n;
+    const float* s_row; int32_t row_stride;
+    const float* s_col; int32_t col_stride;
+    float* out; int64_t ldo;
+    int32_t* acc_out;          // optional raw sums [M, N]
+    int32_t* part;             // split contraction: zeroed int32 [M, N]
+    uint32_t* tickets;         // split contraction: zeroed, one per output tile
+    uint32_t* status;
+    int32_t vec_out;           // 16-byte stores to out allowed
+};
+
+__device__ __forceinline__ void give_up(SharedTail* T, uint32_t* status) {
+    T->abort_flag = 1u;
+    record_status(status, SRQ_ERR_TIMEOUT);
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    SharedTail* T = (SharedTail*)(smem + (size_t)STAGES * STAGE_BYTES);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&T->full[s], 1); mbar_init(&T->empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&T->tmem_full[b], 1); mbar_init(&T->tmem_empty[b], 4); }
+        mbar_init(&T->drain, 1);
+        T->abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&T->tmem_base, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = T->tmem_base;
+
+    const int64_t units = (int64_t)P.tiles_m * P.tiles_n * P.splits;
+    const int32_t kb_per_split = (P.num_kb + P.splits - 1) / P.splits;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t u = blockIdx.x; u < units && ok; u += gridDim.x) {
+                const int32_t split = (int32_t)(u % P.splits);
+                const int64_t tile = u / P.splits;
+                const int32_t tn = (int32_t)(tile % P.tiles_n), tm = (int32_t)(tile / P.tiles_n);
+                const int32_t kb0 = split * kb_per_split;
+                const int32_t kb1 = min(kb0 + kb_per_split, P.num_kb);
+                for (int32_t kb = kb0; kb < kb1; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(&T->empty[s], ph ^ 1u, &T->abort_flag)) { give_up(T, P.status); ok = false; break; }
+                    mbar_expect_tx(&T->full[s], STAGE_BYTES);
+                    uint8_t* sa = smem + (size_t)s * STAGE_BYTES;
+                    tma_load_2d(sa, &map_a, kb * BK, tm * BM, &T->full[s]);
+                    tma_load_2d(sa + A_STAGE_BYTES, &map_b, kb * BK, tn * BN, &T->full[s]);
+                }
+            }
+            if (!ok) {
+                // loads already issued must land before the CTA may leave
+                const uint32_t back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+                for (uint32_t j = 1; j <= back; ++j) {
+                    const uint32_t jt = it - j;
+                    const uint64_t t0 = global_ns();
+                    while (!mbar_try_wait(&T->full[jt % STAGES], (jt / STAGES) & 1u) && global_ns() - t0 < WAIT_LIMIT_NS) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_i8(BM, BN);
+            uint32_t it = 0, lt = 0;
+            bool ok = true;
+            for (int64_t u = blockIdx.x; u < units && ok; u += gridDim.x, ++lt) {
+                const int32_t split = (int32_t)(u % P.splits);
+                const int32_t kb0 = split * kb_per_split;
+                const int32_t kb1 = min(kb0 + kb_per_split, P.num_kb);
+                const uint32_t buf = lt & 1u, use = lt >> 1;
+                if (!mbar_wait(&T->tmem_empty[buf], (use & 1u) ^ 1u, &T->abort_flag)) { give_up(T, P.status); ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int32_t kb = kb0; kb < kb1; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(&T->full[s], ph, &T->abort_flag)) { give_up(T, P.status); ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
+                    const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + A_STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // advancing K inside the swizzle atom = advancing the start address
+                        umma_i8(d_tmem, da + (uint64_t)((k * UMMA_K) >> 4), db + (uint64_t)((k * UMMA_K) >> 4), idesc,
+                                (kb > kb0 || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&T->empty[s]);       // stage reusable once these MMAs have read it
+                }
+                if (ok) umma_commit(&T->tmem_full[buf]);   // accumulator complete
+            }
+            if (!ok) {
+                umma_commit(&T->drain);
+                const uint64_t t0 = global_ns();
+                while (!mbar_try_wait(&T->drain, 0u) && global_ns() - t0 < WAIT_LIMIT_NS) {}
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;                    // TMEM lanes this warp may read
+        const int etid = threadIdx.x - 64;               // 0..127 within the epilogue group
+        uint32_t lt = 0;
+        bool ok = true;
+        for (int64_t u = blockIdx.x; u < units && ok; u += gridDim.x, ++lt) {
+            const int64_t tile = u / P.splits;
+            const int32_t tn = (int32_t)(tile % P.tiles_n), tm = (int32_t)(tile / P.tiles_n);
+            const uint32_t buf = lt & 1u, use = lt >> 1;
+            const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
+            const int64_t col_base = (int64_t)tn * BN;
+            // stage this tile's column step sizes (other buffer may still be read by slower warps)
+            for (int i = etid; i < BN; i += 128) {
+                const int64_t c = col_base + i;
+                T->s_col[buf][i] = (c < P.N) ? P.s_col[c * P.col_stride] : 0.0f;
+            }
+            const float sr = (row < P.M) ? P.s_row[row * P.row_stride] : 0.0f;
+            if (!mbar_wait(&T->tmem_full[buf], use & 1u, &T->abort_flag)) give_up(T, P.status);
+            // the four warps must leave together (they share named barrier 1): agree on one flag
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (etid == 0) T->epi_abort = T->abort_flag;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (T->epi_abort) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
+            if (P.splits == 1) {
+#pragma unroll 1
+                for (int j = 0; j < BN / 32; ++j) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + j * 32, v);
+                    tmem_ld_wait();
+                    const int64_t col0 = col_base + j * 32;
+                    if (row < P.M && col0 < P.N) {
+                        float* dst = P.out + row * P.ldo + col0;
+                        const float* sc = &T->s_col[buf][j * 32];
+                        if (P.vec_out && col0 + 32 <= P.N) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                const float4 c4 = *reinterpret_cast<const float4*>(sc + 4 * q);
+                                float4 o;
+                                o.x = __fmul_rn(__int2float_rn((int)v[4 * q + 0]), __fmul_rn(sr, c4.x));
+                                o.y = __fmul_rn(__int2float_rn((int)v[4 * q + 1]), __fmul_rn(sr, c4.y));
+                                o.z = __fmul_rn(__int2float_rn((int)v[4 * q + 2]), __fmul_rn(sr, c4.z));
+                                o.w = __fmul_rn(__int2float_rn((int)v[4 * q + 3]), __fmul_rn(sr, c4.w));
+                                __stcs(reinterpret_cast<float4*>(dst + 4 * q), o);
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (col0 + i < P.N) dst[i] = __fmul_rn(__int2float_rn((int)v[i]), __fmul_rn(sr, sc[i]));
+                        }
+                        if (P.acc_out) {
+                            int32_t* ad = P.acc_out + row * P.N + col0;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (col0 + i < P.N) ad[i] = (int32_t)v[i];
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&T->tmem_empty[buf]);
+            } else {
+                // exact partial sums: integer adds commute, so any arrival order gives the same total
+#pragma unroll 1
+                for (int j = 0; j < BN / 32; ++j) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + j * 32, v);
+                    tmem_ld_wait();
+                    const int64_t col0 = col_base + j * 32;
+                    if (row < P.M && col0 < P.N) {
+                        int32_t* pd = P.part + row * P.N + col0;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + i < P.N) atomicAdd(pd + i, (int32_t)v[i]);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&T->tmem_empty[buf]);
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (etid == 0) {
+                    const uint32_t t = atomicAdd(&P.tickets[tile], 1u);
+                    T->last_flag[buf] = (t == (uint32_t)P.splits - 1u) ? 1u : 0u;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (T->last_flag[buf]) {
+                    __threadfence();
+                    // the last contributor scales the finished tile: warp w takes rows w, w+4, ...
+                    const int ew = warp - 2;
+                    for (int r = ew; r < BM; r += 4) {
+                        const int64_t grow = (int64_t)tm * BM + r;
+                        if (grow >= P.M) break;
+                        const float srr = P.s_row[grow * P.row_stride];
+                        for (int cidx = lane; cidx < BN; cidx += 32) {
+                            const int64_t gcol = col_base + cidx;
+                            if (gcol < P.N) {
+                                const int32_t a = __ldcg(P.part + grow * P.N + gcol);
+                                P.out[grow * P.ldo + gcol] = __fmul_rn(__int2float_rn(a), __fmul_rn(srr, T->s_col[buf][cidx]));
+                                if (P.acc_out) P.acc_out[grow * P.N + gcol] = a;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    });
+    return fn;
+}
+
+// [rows, kc] int8 matrix with row pitch ld bytes, boxes of box_rows x 128 bytes, 128-byte swizzle.
+static bool encode_operand(CUtensorMap* map, const int8_t* base, int64_t rows, int64_t kc, int64_t ld, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kc, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 1;
+    }
+    return n;
+}
+
+static int choose_splits(int64_t tiles, int32_t num_kb) {
+    const int sms = sm_count();
+    if (tiles * 2 > sms || num_kb < 16) return 1;          // enough tiles to fill the machine
+    int s = (int)(sms / tiles);
+    const int max_by_k = num_kb / 8;                        // keep at least 8 k-blocks per part
+    if (s > max_by_k) s = max_by_k;
+    if (s < 1) s = 1;
+    const int per = (num_kb + s - 1) / s;                   // no part may be empty
+    return (num_kb + per - 1) / per;
+}
+
+size_t gemm_splitk_bytes(int64_t M, int64_t N) {
+    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    if (tiles * 2 > 160) return 0;   // never split (bound is generous with respect to the SM count)
+    return align_up((size_t)M * N * 4) + align_up((size_t)tiles * 4);
+}
+
+srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream) {
+    if (g.M == 0 || g.N == 0) return SRQ_OK;
+    {   // opt in to the large dynamic shared-memory carve-out once per device
+        static bool done[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return SRQ_ERR_CUDA;
+        if (dev < 0 || dev >= 64 || !done[dev]) {
+            if (cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM) != cudaSuccess)
+                return SRQ_ERR_CUDA;
+            if (dev >= 0 && dev < 64) done[dev] = true;
+        }
+    }
+
+    CUtensorMap map_a, map_b;
+    if (!encode_operand(&map_a, g.a, g.M, g.Kc, g.lda, BM)) return SRQ_ERR_CUDA;
+    if (!encode_operand(&map_b, g.b, g.N, g.Kc, g.ldb, BN)) return SRQ_ERR_CUDA;
+
+    GemmParams P;
+    P.M = g.M; P.N = g.N;
+    P.num_kb = (int32_t)((g.Kc + BK - 1) / BK);
+    P.tiles_m = (int32_t)((g.M + BM - 1) / BM);
+    P.tiles_n = (int32_t)((g.N + BN - 1) / BN);
+    const int64_t tiles = (int64_t)P.tiles_m * P.tiles_n;
+    P.splits = choose_splits(tiles, P.num_kb);
+    P.part = nullptr; P.tickets = nullptr;
+    if (P.splits > 1) {
+        const size_t part_bytes = align_up((size_t)g.M * g.N * 4), ticket_bytes = align_up((size_t)tiles * 4);
+        if (g.splitk_ws == nullptr || g.splitk_ws_bytes < part_bytes + ticket_bytes) {
+            P.splits = 1;   // no room: run unsplit (same result)
+        } else {
+            P.part = (int32_t*)g.splitk_ws;
+            P.tickets = (uint32_t*)((char*)g.splitk_ws + part_bytes);
+            if (cudaMemsetAsync(g.splitk_ws, 0, part_bytes + ticket_bytes, stream) != cudaSuccess) return SRQ_ERR_CUDA;
+        }
+    }
+    P.s_row = g.s_row; P.row_stride = g.row_stride;
+    P.s_col = g.s_col; P.col_stride = g.col_stride;
+    P.out = g.out; P.ldo = g.ldo; P.acc_out = g.acc_out;
+    P.status = status;
+    P.vec_out = ((uintptr_t)g.out % 16 == 0) && (g.ldo % 4 == 0);
+
+    const int64_t units = tiles * P.splits;
+    const unsigned grid = (unsigned)(units < sm_count() ? units : sm_count());
+    gemm_i8_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(map_a, map_b, P);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+}
+
+}  // namespace srq

@@ -1,0 +1,101 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header declares, and rejects
+bad arguments on the host before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+from paper_2511_00874_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    entry.build()
+    return binding.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "srq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b([a-z_0-9]+)\s*\([^;{]*\)\s*;", text)
+    return sorted(set(names))
+
+
+def test_header_symbols_are_exported(L):
+    names = _declared()
+    assert set(binding.EXPORTS) == set(names), (names, binding.EXPORTS)
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_status_strings(L):
+    seen = {binding.status_string(i) for i in range(8)}
+    assert len(seen) == 8 and "ok" in seen
+    assert "unknown" in binding.status_string(99)
+
+
+def test_workspace_sizes_grow_with_the_problem(L):
+    small = binding.srq_workspace_bytes(64, 256, 256)
+    big = binding.srq_workspace_bytes(4096, 4096, 4096)
+    assert 0 < small < big
+    # room for both int8 code matrices of the largest pass at least
+    assert big >= 2 * 4096 * 4096
+    assert binding.srq_workspace_bytes(-1, 1, 1) == 0
+    assert binding.srq_quantize_workspace_bytes(128, 128) >= 256 + 4 * 4 * 128
+    assert binding.srq_gemm_workspace_bytes(768, 768) >= 256 + 768 * 768 * 4
+    # large outputs are never split, so they need only the header
+    assert binding.srq_gemm_workspace_bytes(65536, 4096) == 256
+
+
+def test_host_side_argument_checks_need_no_device(L):
+    q = binding.QSpec().c()
+    fake = 4096          # an "aligned pointer"; the calls below must fail before using it
+    f = L.sr_quantize
+    r = lambda *a: int(f(*a))
+    # null input, null workspace
+    assert r(None, 0, 8, 8, 8, ctypes.byref(q), fake, 8, fake, None, 0, None, fake, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert r(fake, 0, 8, 8, 8, ctypes.byref(q), fake, 8, fake, None, 0, None, None, 1 << 20, None) == binding.ERR_INVALID_ARG
+    # no output layout requested; pitch smaller than extent; bad dtype
+    assert r(fake, 0, 8, 8, 8, ctypes.byref(q), None, 0, None, None, 0, None, fake, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert r(fake, 0, 8, 8, 4, ctypes.byref(q), fake, 8, fake, None, 0, None, fake, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert r(fake, 7, 8, 8, 8, ctypes.byref(q), fake, 8, fake, None, 0, None, fake, 1 << 20, None) == binding.ERR_INVALID_ARG
+    # misaligned input pointer, misaligned workspace
+    assert r(fake + 4, 0, 8, 8, 8, ctypes.byref(q), fake, 8, fake, None, 0, None, fake, 1 << 20, None) == binding.ERR_INVALID_ARG
+    assert r(fake, 0, 8, 8, 8, ctypes.byref(q), fake, 8, fake, None, 0, None, fake + 64, 1 << 20, None) == binding.ERR_INVALID_ARG
+    # bits outside 2..8; bad enums
+    for bits in (1, 9, 0, -3):
+        qb = binding.QSpec(bits=bits).c()
+        assert r(fake, 0, 8, 8, 8, ctypes.byref(qb), fake, 8, fake, None, 0, None, fake, 1 << 20, None) == binding.ERR_UNSUPPORTED
+    qb = binding.QSpec(scale=5).c()
+    assert r(fake, 0, 8, 8, 8, ctypes.byref(qb), fake, 8, fake, None, 0, None, fake, 1 << 20, None) == binding.ERR_INVALID_ARG
+    # workspace too small
+    assert r(fake, 0, 8, 8, 8, ctypes.byref(q), fake, 8, fake, None, 0, None, fake, 16, None) == binding.ERR_WORKSPACE
+
+
+def test_layer_calls_check_overflow_and_workspace_on_the_host(L):
+    q8 = binding.QSpec(bits=8).c()
+    q4 = binding.QSpec(bits=4).c()
+    fake = 4096
+    g = L.qlinear_bwd_weight
+    # contraction over T: 133145 * 127 * 127 >= 2^31 is refused, 4-bit gradients lift the limit
+    assert int(g(fake, fake, 0, 133145, 16, 16, ctypes.byref(q8), ctypes.byref(q8), fake, None, fake, 1 << 40, None)) == binding.ERR_ACC_OVERFLOW
+    assert int(g(fake, fake, 0, 133145, 16, 16, ctypes.byref(q4), ctypes.byref(q8), fake, None, fake, 16, None)) == binding.ERR_WORKSPACE
+    f = L.qlinear_fwd
+    assert int(f(fake, fake, 0, 64, 64, 64, ctypes.byref(q8), ctypes.byref(q8), None, None, fake, 1 << 30, None)) == binding.ERR_INVALID_ARG
+    assert int(f(fake, fake, 0, 64, 64, 64, ctypes.byref(q8), None, fake, None, fake, 1 << 30, None)) == binding.ERR_INVALID_ARG
+    assert int(f(fake, fake, 0, 64, 64, 64, ctypes.byref(q8), ctypes.byref(q8), fake, None, fake, 1024, None)) == binding.ERR_WORKSPACE
+    h = L.srq_gemm_i8
+    # pitch not a multiple of 16 breaks the TMA rule
+    assert int(h(fake, 24, fake, 32, 8, 8, 24, fake, 0, fake, 0, fake, 8, None, fake, 4096, None)) == binding.ERR_INVALID_ARG
+    assert int(h(fake, 32, fake, 32, 8, 8, 24, fake, 0, fake, 2, fake, 8, None, fake, 4096, None)) == binding.ERR_INVALID_ARG
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "libsrq.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        binding.lib()

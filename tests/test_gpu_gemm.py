@@ -1,0 +1,101 @@
+"""GPU parity of the int8 tensor-core product and its dequantizing epilogue."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2511_00874_b200 as srq
+
+pytestmark = pytest.mark.gpu
+
+
+def _codes(rows, kc, seed, lo=-127, hi=127, pad=None):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    pitch = (kc + 15) // 16 * 16 if pad is None else pad
+    full = torch.zeros((rows, pitch), dtype=torch.int8)
+    full[:, :kc] = torch.randint(lo, hi + 1, (rows, kc), generator=g, dtype=torch.int8)
+    if pitch > kc:
+        full[:, kc:] = 77        # padding must never be read as data
+    return full.cuda()[:, :kc]
+
+
+def _run(a, b, s_row, s_col, want_acc=True):
+    M, N = a.shape[0], b.shape[0]
+    out = torch.full((M, N), float("nan"), device="cuda")
+    acc = torch.full((M, N), -1, dtype=torch.int32, device="cuda") if want_acc else None
+    ws = srq.new_workspace(srq.srq_gemm_workspace_bytes(M, N))
+    srq.srq_gemm_i8(a, b, s_row, s_col, out, acc, ws)
+    st = srq.srq_poll_status(ws)
+    assert st == 0, srq.status_string(st)
+    return out.cpu().numpy(), None if acc is None else acc.cpu().numpy()
+
+
+@pytest.mark.parametrize("M,N,Kc", [(64, 256, 256), (128, 256, 128), (1, 1, 1), (5, 7, 3), (129, 257, 130),
+                                    (300, 520, 1000), (128, 512, 4096), (200, 40, 48), (384, 768, 640)])
+@pytest.mark.parametrize("per_row", [False, True])
+def test_product_and_dequant_match_the_oracle(M, N, Kc, per_row):
+    a, b = _codes(M, Kc, 1), _codes(N, Kc, 2)
+    g = torch.Generator(device="cpu").manual_seed(3)
+    s_row = (torch.rand(M if per_row else 1, generator=g) * 0.1 + 1e-3).cuda()
+    s_col = (torch.rand(N if per_row else 1, generator=g) * 0.1 + 1e-3).cuda()
+    out, acc = _run(a, b, s_row, s_col)
+    ref_acc = oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy())
+    assert np.array_equal(acc, ref_acc)
+    ref_out = oracle.dequant(ref_acc, s_row.cpu().numpy(), s_col.cpu().numpy())
+    assert np.array_equal(out, ref_out)          # same two binary32 multiplies: 0 ulp
+
+
+def test_special_code_matrices():
+    # all ones: every sum equals the contraction length; identity: returns the other operand
+    Kc = 400
+    ones = torch.ones((130, 400), dtype=torch.int8, device="cuda")
+    one = torch.ones(1, device="cuda")
+    out, acc = _run(ones[:, :Kc], ones[:70, :Kc], one, one)
+    assert (acc == Kc).all() and (out == Kc).all()
+    eye = torch.eye(256, dtype=torch.int8, device="cuda")
+    b = _codes(300, 256, 5)
+    out, acc = _run(eye, b, one, one)
+    assert np.array_equal(acc, b.cpu().numpy().T.astype(np.int32))
+    # extreme codes over the longest contraction of the workloads: 65536 * 127^2 < 2^31
+    a = torch.full((128, 65536), 127, dtype=torch.int8, device="cuda")
+    bb = torch.full((256, 65536), -127, dtype=torch.int8, device="cuda")
+    out, acc = _run(a, bb, one, one)
+    assert (acc == -65536 * 127 * 127).all()
+
+
+def test_split_contraction_is_exact():
+    # small output, long contraction: the kernel splits K across CTAs and adds int32 partials
+    for (M, N, Kc) in [(768, 768, 8192), (256, 256, 16384), (100, 300, 4224)]:
+        a, b = _codes(M, Kc, 11), _codes(N, Kc, 12)
+        s_row = torch.rand(M, device="cuda") + 0.5
+        s_col = torch.rand(N, device="cuda") + 0.5
+        out, acc = _run(a, b, s_row, s_col)
+        ref_acc = oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy())
+        assert np.array_equal(acc, ref_acc)
+        assert np.array_equal(out, oracle.dequant(ref_acc, s_row.cpu().numpy(), s_col.cpu().numpy()))
+        # and without the workspace (unsplit path) the result is the same
+        out2 = torch.empty((M, N), device="cuda")
+        ws = srq.new_workspace(256)
+        srq.srq_gemm_i8(a, b, s_row, s_col, out2, None, ws)
+        assert srq.srq_poll_status(ws) == 0
+        assert np.array_equal(out2.cpu().numpy(), out)
+
+
+def test_many_tiles_per_cta_and_freivalds():
+    """More tiles than SMs (persistent loop, both TMEM buffers, ring wrap-around), checked
+    with exact integer Freivalds products and 64 fully recomputed rows."""
+    M, N, Kc = 128 * 40, 256 * 9, 768
+    a, b = _codes(M, Kc, 21), _codes(N, Kc, 22)
+    one = torch.ones(1, device="cuda")
+    out, acc = _run(a, b, one, one)
+    rng = np.random.default_rng(0)
+    rows = np.sort(rng.choice(M, 64, replace=False))
+    ref = oracle.gemm_i8_nt(a.cpu().numpy()[rows], b.cpu().numpy())
+    assert np.array_equal(acc[rows], ref)
+    A64, B64, C64 = a.cpu().numpy().astype(np.int64), b.cpu().numpy().astype(np.int64), acc.astype(np.int64)
+    for _ in range(3):
+        r = rng.integers(-3, 4, (N, 1))
+        assert np.array_equal(C64 @ r, A64 @ (B64.T @ r))
+        l = rng.integers(-3, 4, (1, M))
+        assert np.array_equal(l @ C64, (l @ A64) @ B64.T)
+    assert np.array_equal(out, acc.astype(np.float32))

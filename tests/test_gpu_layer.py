@@ -1,0 +1,130 @@
+"""GPU parity of the three layer passes (Alg. 1 and Alg. 2) against the CPU oracle:
+codes, step sizes and int32 sums bit for bit, fp32 outputs equal (0 ulp; bound 1 ulp)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2511_00874_b200 as srq
+from paper_2511_00874_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+PASSES = {
+    "fwd": (srq.qlinear_fwd, oracle.qlinear_fwd),
+    "bwd_input": (srq.qlinear_bwd_input, oracle.qlinear_bwd_input),
+    "bwd_weight": (srq.qlinear_bwd_weight, oracle.qlinear_bwd_weight),
+}
+
+
+def _ulp_diff(a, b):
+    ia = a.view(np.int32).astype(np.int64)
+    ib = b.view(np.int32).astype(np.int64)
+    ia = np.where(ia < 0, -(ia & 0x7FFFFFFF), ia)
+    ib = np.where(ib < 0, -(ib & 0x7FFFFFFF), ib)
+    return np.abs(ia - ib).max() if a.size else 0
+
+
+def run_pass(name, X0, X1, T, N, K, q0, q1, ws=None, full=True):
+    """Runs one pass on the GPU and in the oracle; returns (gpu out tensor, oracle result)."""
+    fn, ofn = PASSES[name]
+    dev = X0.device
+    shapes = {"fwd": ((T, K), (N, K), (T, N)), "bwd_input": ((T, N), (K, N), (T, K)),
+              "bwd_weight": ((N, T), (K, T), (N, K))}[name]
+    n_a = shapes[0][0] if q0.scale == srq.PER_ROW else 1
+    n_b = shapes[1][0] if q1.scale == srq.PER_ROW else 1
+    out = torch.full(shapes[2], float("nan"), device=dev)
+    dbg = srq.DebugOut(torch.empty(shapes[0], dtype=torch.int8, device=dev), torch.empty(n_a, device=dev),
+                       torch.empty(shapes[1], dtype=torch.int8, device=dev), torch.empty(n_b, device=dev),
+                       torch.empty(shapes[2], dtype=torch.int32, device=dev))
+    if ws is None:
+        ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K), dev)
+    fn(X0, X1, q0, q1, out, dbg, ws)
+    st = srq.srq_poll_status(ws)
+    assert st == 0, srq.status_string(st)
+    oq = lambda q: oracle.QSpec(q.bits, q.scale, q.round, q.seed, q.tensor_id, q.index_offset)
+    ref = ofn(X0.float().cpu().numpy(), X1.float().cpu().numpy(), oq(q0), oq(q1))
+    if full:
+        assert np.array_equal(dbg.codes_a.cpu().numpy(), ref.codes_a), name + ": codes of first operand"
+        assert np.array_equal(dbg.codes_b.cpu().numpy(), ref.codes_b), name + ": codes of second operand"
+        assert np.array_equal(dbg.scale_a.cpu().numpy(), ref.scale_a), name + ": step sizes of first operand"
+        assert np.array_equal(dbg.scale_b.cpu().numpy(), ref.scale_b), name + ": step sizes of second operand"
+        assert np.array_equal(dbg.acc.cpu().numpy(), ref.acc), name + ": int32 sums"
+        o = out.cpu().numpy()
+        assert _ulp_diff(o, ref.out) <= 1, name + ": fp32 output beyond 1 ulp"
+        assert np.array_equal(o, ref.out), name + ": fp32 output"
+    return out, ref
+
+
+def layer_specs(scale, rnd, seed, bits_fwd=8, bits_bwd=8):
+    # five quantization points per layer: A and W forward; A, W and dY backward
+    return {"a_fwd": srq.QSpec(bits_fwd, scale, rnd, seed, 0), "w_fwd": srq.QSpec(bits_fwd, scale, rnd, seed, 1),
+            "a_bwd": srq.QSpec(bits_bwd, scale, rnd, seed, 2), "w_bwd": srq.QSpec(bits_bwd, scale, rnd, seed, 3),
+            "dy_bwd": srq.QSpec(bits_bwd, scale, rnd, seed, 4)}
+
+
+def all_passes(A, W, dY, q, ws=None):
+    T, K = A.shape
+    N = W.shape[0]
+    run_pass("fwd", A, W, T, N, K, q["a_fwd"], q["w_fwd"], ws)
+    run_pass("bwd_input", dY, W, T, N, K, q["dy_bwd"], q["w_bwd"], ws)
+    run_pass("bwd_weight", dY, A, T, N, K, q["dy_bwd"], q["a_bwd"], ws)
+
+
+def test_single_layer_8bit_per_tensor_seed0():
+    """A 64x256, W 256x256, dY 64x256 fp32, 8-bit per-tensor SR, seed 0."""
+    A, W, dY = synth.layer_inputs(64, 256, 256, seed=0, device="cuda", std_dy=1.0)
+    all_passes(A, W, dY, layer_specs(srq.PER_TENSOR, srq.SR, 0))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("scale", [srq.PER_TENSOR, srq.PER_ROW])
+@pytest.mark.parametrize("rnd", [srq.SR, srq.RTN])
+def test_ragged_multi_tile_layer(dtype, scale, rnd):
+    T, N, K = 264, 392, 328            # all three differ, none a tile multiple
+    A, W, dY = synth.layer_inputs(T, N, K, seed=1, dtype=dtype, device="cuda", std_dy=1e-3)
+    all_passes(A, W, dY, layer_specs(scale, rnd, seed=3, bits_fwd=8, bits_bwd=4))
+
+
+def test_odd_extents_take_the_elementwise_path():
+    T, N, K = 37, 21, 50
+    A, W, dY = synth.layer_inputs(T, N, K, seed=2, device="cuda")
+    all_passes(A, W, dY, layer_specs(srq.PER_ROW, srq.SR, seed=9, bits_bwd=6))
+
+
+def test_gpt2_shaped_layer_small_batch():
+    """GPT-2-small projection 768 -> 2304 at 1024 tokens; 64 sampled rows per output."""
+    T, K, N = 1024, 768, 2304
+    A, W, dY = synth.layer_inputs(T, N, K, seed=3, device="cuda", std_dy=1e-3)
+    all_passes(A, W, dY, layer_specs(srq.PER_TENSOR, srq.SR, seed=0))
+
+
+def test_workspace_reuse_and_shared_quantized_weight():
+    """One workspace for all passes; the same (seed, tensor_id) for W forward and backward
+    gives one quantized W, its backward layout being the transpose of the forward one."""
+    T, N, K = 256, 384, 512
+    A, W, dY = synth.layer_inputs(T, N, K, seed=4, device="cuda")
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
+    q = layer_specs(srq.PER_TENSOR, srq.SR, seed=1)
+    q["w_bwd"] = q["w_fwd"]
+    dev = A.device
+    cw = torch.empty((N, K), dtype=torch.int8, device=dev)
+    cwt = torch.empty((K, N), dtype=torch.int8, device=dev)
+    Y = torch.empty((T, N), device=dev)
+    dA = torch.empty((T, K), device=dev)
+    srq.qlinear_fwd(A, W, q["a_fwd"], q["w_fwd"], Y, srq.DebugOut(codes_b=cw), ws)
+    srq.qlinear_bwd_input(dY, W, q["dy_bwd"], q["w_bwd"], dA, srq.DebugOut(codes_b=cwt), ws)
+    assert srq.srq_poll_status(ws) == 0
+    assert torch.equal(cw.t(), cwt)
+    all_passes(A, W, dY, q, ws)
+
+
+def test_overflowing_contraction_is_refused():
+    A = torch.zeros((133145, 16), device="cuda")
+    dY = torch.zeros((133145, 16), device="cuda")
+    dW = torch.empty((16, 16), device="cuda")
+    with pytest.raises(srq.SrqError) as e:
+        srq.qlinear_bwd_weight(dY, A, srq.QSpec(8), srq.QSpec(8), dW)
+    assert e.value.status == 4
+    srq.qlinear_bwd_weight(dY, A, srq.QSpec(4), srq.QSpec(8), dW)       # 7 * 127 * T fits
+    assert torch.count_nonzero(dW).item() == 0

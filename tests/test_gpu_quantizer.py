@@ -1,0 +1,156 @@
+"""GPU parity of sr_quantize against the CPU oracle: codes and step sizes bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2511_00874_b200 as srq
+from paper_2511_00874_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_gpu(x, q, want_rm=True, want_tr=True, pad_rm=0, pad_tr=0):
+    rows, cols = x.shape
+    per_row = q.scale == srq.PER_ROW
+    dev = x.device
+    crm = srm = ctr = strr = None
+    if want_rm:
+        crm_full = torch.full((rows, cols + pad_rm), 99, dtype=torch.int8, device=dev)
+        crm = crm_full[:, :cols]
+        srm = torch.full((rows if per_row else 1,), -1.0, dtype=torch.float32, device=dev)
+    if want_tr:
+        ctr_full = torch.full((cols, rows + pad_tr), 99, dtype=torch.int8, device=dev)
+        ctr = ctr_full[:, :rows]
+        strr = torch.full((cols if per_row else 1,), -1.0, dtype=torch.float32, device=dev)
+    ws = srq.new_workspace(srq.srq_quantize_workspace_bytes(rows, cols), dev)
+    srq.sr_quantize(x, q, crm, srm, ctr, strr, ws)
+    assert srq.srq_poll_status(ws) == 0
+    if want_rm and pad_rm:
+        assert bool((crm_full[:, cols:] == 99).all()), "padding of the row-major layout was written"
+    if want_tr and pad_tr:
+        assert bool((ctr_full[:, rows:] == 99).all()), "padding of the transposed layout was written"
+    f = lambda t: None if t is None else t.cpu().numpy()
+    return f(crm), f(srm), f(ctr), f(strr)
+
+
+def _check(x, bits, scale, rnd, seed=0, tid=0, off=0, want_rm=True, want_tr=True, pad_rm=0, pad_tr=0):
+    q = srq.QSpec(bits, scale, rnd, seed, tid, off)
+    got = _run_gpu(x, q, want_rm, want_tr, pad_rm, pad_tr)
+    ref = oracle.sr_quantize(x.float().cpu().numpy(), oracle.QSpec(bits, scale, rnd, seed, tid, off),
+                             want_rm, want_tr)
+    for name, g, r in zip(("codes_rm", "scale_rm", "codes_tr", "scale_tr"), got, ref):
+        if r is None:
+            continue
+        assert g.shape == r.shape, name
+        bad = np.argwhere(g != r)
+        assert bad.size == 0, f"{name}: {len(bad)} mismatches, first at {bad[0]}: gpu {g[tuple(bad[0])]} oracle {r[tuple(bad[0])]}"
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("scale", [srq.PER_TENSOR, srq.PER_ROW])
+@pytest.mark.parametrize("rnd", [srq.SR, srq.RTN])
+@pytest.mark.parametrize("bits", [8, 6, 4, 3])
+def test_multi_tile_with_ragged_tail(dtype, scale, rnd, bits):
+    # 2.x tiles of 128 in each direction, extents multiples of 4 (vector path)
+    x = synth.with_outliers((300, 388), seed=bits, dtype=dtype, device="cuda")
+    _check(x, bits, scale, rnd, seed=bits, tid=7, pad_rm=12, pad_tr=4)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("shape,off", [((131, 259), 0), ((17, 5), 3), ((1, 1), 0), ((1, 1000), 1),
+                                       ((1000, 1), 2), ((129, 130), 2 ** 33 + 2), ((64, 256), 2 ** 40)])
+def test_unaligned_extents_and_offsets(dtype, shape, off):
+    x = synth.normal(shape, 1.0, seed=shape[0], dtype=dtype, device="cuda")
+    for scale in (srq.PER_TENSOR, srq.PER_ROW):
+        _check(x, 8, scale, srq.SR, seed=2 ** 40 + 3, tid=2 ** 35 + 1, off=off)
+        _check(x, 5, scale, srq.RTN)
+
+
+def test_single_layout_requests():
+    x = synth.normal((200, 136), 1.0, seed=1, device="cuda")
+    for scale in (srq.PER_TENSOR, srq.PER_ROW):
+        _check(x, 8, scale, srq.SR, want_rm=True, want_tr=False)
+        _check(x, 8, scale, srq.SR, want_rm=False, want_tr=True)
+
+
+def test_strided_input_view():
+    big = synth.normal((150, 512), 1.0, seed=2, device="cuda")
+    _check(big[:, 64:64 + 260], 8, srq.PER_ROW, srq.SR, seed=1)      # pitch 512, 16-byte aligned start
+    _check(big[:, 4:4 + 201], 8, srq.PER_TENSOR, srq.SR, seed=1)      # ragged width, aligned start
+
+
+def test_zero_tensor_zero_rows_and_tiny_groups():
+    z = torch.zeros((130, 132), device="cuda")
+    _check(z, 8, srq.PER_TENSOR, srq.SR)
+    x = synth.normal((130, 132), 1.0, seed=3, device="cuda")
+    x[5] = 0
+    x[:, 9] = 0
+    x[7] = 1e-39          # reciprocal step overflows: the group is flushed to zero
+    _check(x, 8, srq.PER_ROW, srq.SR)
+    _check(x, 4, srq.PER_ROW, srq.RTN)
+
+
+def test_grid_exact_inputs_and_extreme_element():
+    k = torch.arange(-127, 128, dtype=torch.float32, device="cuda").repeat(4, 1) * 2.0 ** -5
+    for seed in range(3):
+        _check(k.contiguous(), 8, srq.PER_TENSOR, srq.SR, seed=seed)
+    c = torch.empty((4, 255), dtype=torch.int8, device="cuda")
+    s = torch.empty(1, device="cuda")
+    srq.sr_quantize(k.contiguous(), srq.QSpec(seed=5), c, s)
+    assert torch.equal(c.float(), k * 32)
+
+
+def test_same_spec_same_codes_other_spec_other_codes():
+    x = synth.normal((256, 256), 1.0, seed=4, device="cuda")
+    a = _run_gpu(x, srq.QSpec(8, 0, 0, 1, 2))[0]
+    b = _run_gpu(x, srq.QSpec(8, 0, 0, 1, 2))[0]
+    c = _run_gpu(x, srq.QSpec(8, 0, 0, 1, 3))[0]
+    d = _run_gpu(x, srq.QSpec(8, 0, 0, 2, 2))[0]
+    assert np.array_equal(a, b)
+    assert (a != c).mean() > 0.2 and (a != d).mean() > 0.2
+
+
+def test_nonfinite_input_is_reported():
+    x = synth.normal((64, 64), 1.0, seed=5, device="cuda")
+    x[3, 3] = float("inf")
+    ws = srq.new_workspace(srq.srq_quantize_workspace_bytes(64, 64))
+    c = torch.empty((64, 64), dtype=torch.int8, device="cuda")
+    s = torch.empty(1, device="cuda")
+    srq.sr_quantize(x, srq.QSpec(), c, s, ws=ws)
+    assert srq.srq_poll_status(ws) == 6
+    x[3, 3] = float("nan")
+    srq.sr_quantize(x, srq.QSpec(scale=srq.PER_ROW), c, torch.empty(64, device="cuda"), ws=ws)
+    assert srq.srq_poll_status(ws) == 6
+    x[3, 3] = 1.0
+    srq.sr_quantize(x, srq.QSpec(), c, s, ws=ws)
+    assert srq.srq_poll_status(ws) == 0
+
+
+def test_unbiasedness_of_1e4_draws_on_the_gpu():
+    """E[Q(x)] = x within 5 sigma and Var <= D^2/4, 4096-element tensor, 10^4 seeds."""
+    x = synth.normal((1, 4096), 1.0, seed=6, device="cuda")
+    draws = 10_000
+    c = torch.empty((1, 4096), dtype=torch.int8, device="cuda")
+    s = torch.empty(1, device="cuda")
+    ws = srq.new_workspace(srq.srq_quantize_workspace_bytes(1, 4096))
+    acc = torch.zeros((1, 4096), dtype=torch.float64, device="cuda")
+    acc2 = torch.zeros_like(acc)
+    for seed in range(draws):
+        srq.sr_quantize(x, srq.QSpec(8, 0, 0, seed, 3), c, s, ws=ws)
+        acc += c
+        acc2 += c.double() ** 2
+    xs = x.cpu().numpy()
+    d, inv = oracle.scale_from_absmax(float(np.abs(xs).max()), 8)
+    assert s.item() == d
+    t = xs.astype(np.float64) * float(inv)
+    p = t - np.floor(t)
+    mean = (acc / draws).cpu().numpy()
+    var = (acc2 / draws).cpu().numpy() - mean ** 2
+    assert np.all(np.abs(mean - t) <= 5 * np.sqrt(p * (1 - p) / draws) + 3.0 / draws)
+    assert var.max() <= 0.25 + 1e-9
+    # the first few draws agree with the oracle exactly (same generator, same rule)
+    for seed in (0, 1, 9999):
+        srq.sr_quantize(x, srq.QSpec(8, 0, 0, seed, 3), c, s, ws=ws)
+        ref = oracle.sr_quantize(xs, oracle.QSpec(8, 0, 0, seed, 3))[0]
+        assert np.array_equal(c.cpu().numpy(), ref)
