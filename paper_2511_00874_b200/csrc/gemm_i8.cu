@@ -40,7 +40,7 @@ struct SharedTail {                                    // after the stage ring
     volatile uint32_t abort_flag;
     uint32_t last_flag[2];
     uint32_t epi_abort;
-    float s_col[2][BN];
+    alignas(16) float s_col[2][BN];   // read as float4
 };
 constexpr size_t GEMM_SMEM = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + sizeof(SharedTail);
 
