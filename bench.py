@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the SR-quantized linear layer (forward + both backward products) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one batch: qlinear_fwd, qlinear_bwd_input and
+qlinear_bwd_weight (five absmax reductions and quantizations, three int8 tensor-core products
+with dequantizing epilogues) on a 4096 x 4096 linear layer with 65536 tokens, fp32 inputs,
+8-bit per-tensor stochastic rounding.  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "sr_quantized_linear_fwd_bwd_tops"
+UNIT = "TOPS"
+WORKLOAD = "linear 4096->4096, tokens 65536, fp32 inputs, 8-bit per-tensor SR on A, W, dY (fwd + bwd)"
+T_FULL, N_FULL, K_FULL = 65536, 4096, 4096
+
+# DRAM bytes (read + write) of one gemm_i8_kernel launch of this workload, from the ncu capture
+# summarised in profiles/; None until a capture has been taken.
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def layer_ops(T, N, K):
+    return 6.0 * T * N * K      # three products, 2 T N K integer operations each
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_burst": float(d["bf16_tflops"]),
+                "bf16_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); pw.append(float(f[3]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        # samples under load: the upper half by power draw
+        order = sorted(range(len(sm)), key=lambda i: pw[i])
+        loaded = [sm[i] for i in order[len(order) // 2:]]
+        return {"sm_mhz": statistics.median(loaded), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(pw)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle timing (reported baseline and the --impl reference arm)
+# ---------------------------------------------------------------------------------------------
+def oracle_layer_seconds(T, N, K, seed=0):
+    """Seconds the oracle takes for fwd + bwd_input + bwd_weight of a T-token slice."""
+    import torch
+    import oracle
+    from paper_2511_00874_b200 import synth
+    A, W, dY = synth.layer_inputs(T, N, K, seed, torch.float32, "cpu", std_dy=1e-3)
+    A, W, dY = A.numpy(), W.numpy(), dY.numpy()
+    q = [oracle.QSpec(8, oracle.PER_TENSOR, oracle.SR, seed, i) for i in range(5)]
+    t0 = time.perf_counter()
+    oracle.qlinear_fwd(A, W, q[0], q[1])
+    oracle.qlinear_bwd_input(dY, W, q[4], q[3])
+    oracle.qlinear_bwd_weight(dY, A, q[4], q[2])
+    return time.perf_counter() - t0
+
+
+def pick_oracle_sample(target_s):
+    """Token count of the slice the oracle can do in about target_s seconds on this host."""
+    probe_T = 32
+    t = oracle_layer_seconds(probe_T, N_FULL, K_FULL)
+    Ts = probe_T
+    while Ts * 2 <= T_FULL and t * (Ts * 2 / probe_T) <= target_s:
+        Ts *= 2
+    return Ts
+
+
+def cpu_baseline(target_s=15.0):
+    import oracle
+    Ts = pick_oracle_sample(target_s)
+    sec = oracle_layer_seconds(Ts, N_FULL, K_FULL)
+    return {"value": layer_ops(Ts, N_FULL, K_FULL) / sec / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds": sec,
+            "sample": f"same layer (4096->4096, fp32, 8-bit per-tensor SR), first {Ts} of 65536 tokens, "
+                      f"fwd + bwd_input + bwd_weight, ops counted as 6*T*N*K"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    Ts = pick_oracle_sample(per_step)
+    for _ in range(args.warmup):
+        oracle_layer_seconds(Ts, N_FULL, K_FULL)
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        oracle_layer_seconds(Ts, N_FULL, K_FULL, seed=s)
+    sec = (time.perf_counter() - t0) / max(1, args.steps)
+    val = layer_ops(Ts, N_FULL, K_FULL) / sec / 1e12
+    sample = (f"CPU oracle on {oracle.num_threads()} host threads; each step = fwd + bwd of the first {Ts} of "
+              f"65536 tokens of the same layer (input generation included)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample_tokens": Ts},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2511_00874_b200 as srq
+    from paper_2511_00874_b200 import binding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    binding.lib()                      # fails loudly if libsrq.so is missing
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    T, N, K = T_FULL, N_FULL, K_FULL
+    peaks = load_peaks()
+
+    # each rank holds its own token shard (weak scaling); W is replicated
+    A = synth.normal((T, K), 1.0, 1000 + 3 * rank, torch.float32, dev)
+    dY = synth.normal((T, N), 1e-3, 1001 + 3 * rank, torch.float32, dev)
+    W = synth.normal((N, K), 0.02, 7, torch.float32, dev)
+    Y = torch.empty((T, N), device=dev)
+    dA = torch.empty((T, K), device=dev)
+    dW = torch.empty((N, K), device=dev)
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K), dev)
+
+    def specs(step):
+        off_a, off_y = rank * T * K, rank * T * N       # thresholds follow the global flat index
+        return (srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 0, off_a), srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 1),
+                srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 2, off_a), srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 3),
+                srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 4, off_y))
+
+    def step(i, a=A, w=W, dy=dY):
+        qa_f, qw_f, qa_b, qw_b, qdy = specs(i)
+        srq.qlinear_fwd(a, w, qa_f, qw_f, Y, None, ws)
+        srq.qlinear_bwd_input(dy, w, qdy, qw_b, dA, None, ws)
+        srq.qlinear_bwd_weight(dy, a, qdy, qa_b, dW, None, ws)
+        if world > 1:
+            dist.all_reduce(dW)        # the batch average of the weight gradient spans all shards
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    st = srq.srq_poll_status(ws)
+    if st != 0:
+        raise SystemExit("device status after warm-up: " + srq.status_string(st))
+
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    l0 = srq.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    e1.record()
+    barrier()
+    launches = srq.launch_count() - l0
+    ms = e0.elapsed_time(e1) / args.steps
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = t.item()
+    clocks = sampler.stop() if rank == 0 else None
+    st = srq.srq_poll_status(ws)
+    if st != 0:
+        raise SystemExit("device status after the timed region: " + srq.status_string(st))
+    value = world * layer_ops(T, N, K) / (ms * 1e-3) / 1e12
+
+    result = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+              "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+              "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+              "config": {"workload": WORKLOAD, "tokens_per_gpu": T, "l2": "inputs (1 GiB each) are larger than L2",
+                         "multi_gpu": "token shards, one NCCL all-reduce of dW per step" if world > 1 else "single GPU"},
+              "gpu_launches": int(launches)}
+
+    # ---- end to end through the public API with host buffers (every rank, max over ranks)
+    hA, hW, hdY = (t.cpu().pin_memory() for t in (A, W, dY))
+    hY, hdA, hdW = (torch.empty_like(t, device="cpu").pin_memory() for t in (Y, dA, dW))
+    e_steps = max(1, min(3, args.steps))
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e_steps):
+        a_ = hA.to(dev, non_blocking=True)
+        w_ = hW.to(dev, non_blocking=True)
+        y_ = hdY.to(dev, non_blocking=True)
+        step(1000 + i, a_, w_, y_)
+        hY.copy_(Y, non_blocking=True)
+        hdA.copy_(dA, non_blocking=True)
+        hdW.copy_(dW, non_blocking=True)
+        torch.cuda.synchronize()
+    e_sec = (time.perf_counter() - t0) / e_steps
+    if world > 1:
+        t = torch.tensor([e_sec], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e_sec = t.item()
+    h2d = sum(t.numel() * 4 for t in (hA, hW, hdY))
+    d2h = sum(t.numel() * 4 for t in (hY, hdA, hdW))
+    result["e2e"] = {"value": world * layer_ops(T, N, K) / e_sec / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                     "d2h_bytes_per_step": d2h, "steps": e_steps, "ms_per_step": e_sec * 1e3,
+                     "note": "per rank: pinned host A, W, dY copied in and Y, dA, dW copied out every step"}
+    del hA, hW, hdY, hY, hdA, hdW
+
+    if rank == 0:
+        # ---- per-kernel timing of the dominant kernel: the three products of one step, on the codes
+        # the quantizer wrote, each launch bracketed by CUDA events on the launching stream
+        one = torch.ones(1, device=dev)
+
+        def codes(x, rows, cols, q, rm, tr):
+            crm = torch.empty((rows, cols), dtype=torch.int8, device=dev) if rm else None
+            ctr = torch.empty((cols, rows), dtype=torch.int8, device=dev) if tr else None
+            s1, s2 = torch.empty(1, device=dev), torch.empty(1, device=dev)
+            srq.sr_quantize(x, q, crm, s1 if rm else None, ctr, s2 if tr else None)
+            return crm, ctr
+
+        qs = specs(0)
+        cA, cAt = codes(A, T, K, qs[0], True, True)
+        cW, cWt = codes(W, N, K, qs[1], True, True)
+        cdY, cdYt = codes(dY, T, N, qs[4], True, True)
+        gemms = [(cA, cW, Y), (cdY, cWt, dA), (cdYt, cAt, dW)]
+        gws = srq.new_workspace(max(srq.srq_gemm_workspace_bytes(o.shape[0], o.shape[1]) for _, _, o in gemms), dev)
+        for a_, b_, o_ in gemms:
+            srq.srq_gemm_i8(a_, b_, one, one, o_, None, gws)
+        torch.cuda.synchronize()
+        reps = max(3, args.steps)
+        evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in gemms]
+               for _ in range(reps)]
+        for r in range(reps):
+            for j, (a_, b_, o_) in enumerate(gemms):
+                evs[r][j][0].record()
+                srq.srq_gemm_i8(a_, b_, one, one, o_, None, gws)
+                evs[r][j][1].record()
+        torch.cuda.synchronize()
+        gemm_ms = [statistics.mean(evs[r][j][0].elapsed_time(evs[r][j][1]) for r in range(reps)) for j in range(3)]
+        launch_ms = statistics.mean(gemm_ms)
+        ops_per_launch = 2.0 * T * N * K
+        achieved = ops_per_launch / (launch_ms * 1e-3) / 1e12
+        peak = 2.0 * peaks["bf16_sustained"]        # int8 : bf16 dense nominal ratio is 2
+        result["roofline"] = {
+            "bound": "tensor", "kernel": "gemm_i8_kernel", "achieved": achieved, "peak": peak, "unit": "TOPS",
+            "frac": achieved / peak, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
+            "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS TFLOP/s (int8:bf16 nominal ratio 2)",
+            "frac_of_burst": achieved / (2.0 * peaks["bf16_burst"]), "frac_of_nominal_4500": achieved / 4500.0,
+            "ms_per_launch": {"fwd": gemm_ms[0], "bwd_input": gemm_ms[1], "bwd_weight": gemm_ms[2]},
+            "ops_per_launch": ops_per_launch}
+        del cA, cAt, cW, cWt, cdY, cdYt
+
+        # ---- the quantizer alone on the largest tensor of the sweep: 2^28 fp32 elements
+        n_q = 1 << 28
+        xq = synth.with_outliers((n_q // 4096, 4096), 11, torch.float32, dev)
+        cq = torch.empty((n_q // 4096, 4096), dtype=torch.int8, device=dev)
+        sq = torch.empty(1, device=dev)
+        qws = srq.new_workspace(srq.srq_quantize_workspace_bytes(n_q // 4096, 4096), dev)
+        for i in range(3):
+            srq.sr_quantize(xq, srq.QSpec(8, 0, 0, i, 9), cq, sq, ws=qws)
+        torch.cuda.synchronize()
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        q0.record()
+        for i in range(10):
+            srq.sr_quantize(xq, srq.QSpec(8, 0, 0, i, 9), cq, sq, ws=qws)
+        q1.record()
+        torch.cuda.synchronize()
+        q_ms = q0.elapsed_time(q1) / 10
+        q_bytes = n_q * (4 + 4 + 1)       # absmax read + quantize read + one code layout written
+        result["quantizer"] = {"bound": "hbm", "achieved": q_bytes / (q_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                               "unit": "GB/s", "frac": q_bytes / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                               "ms": q_ms, "workload": "sr_quantize 2^28 fp32, per-tensor 8-bit SR, row-major codes "
+                                                       "(absmax pass + quantize pass, 9 bytes per element)"}
+        del xq, cq
+
+        result["clocks"] = clocks
+        if world == 1:
+            result["cpu_baseline"] = cpu_baseline()
+        print(json.dumps(result))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -78,59 +78,63 @@ constexpr int AMAX_THREADS = 256;
 constexpr int AMAX_TILE_C = 512;   // 32 lanes x 4 groups x 4 elements
 constexpr int AMAX_TILE_R = 64;    // 8 warps x 8 rows
 
-// what each layout needs: nothing, one word for the whole tensor, or one word per row (rm) / column (tr)
-enum : int { AMAX_NONE = 0, AMAX_TENSOR = 1, AMAX_GROUPS = 2 };
-
-template <typename T>
+// ROWS: one word per row wanted; COLS: one word per column wanted; neither: one word for the tensor.
+// Two rows (eight 16-byte loads per thread) are in flight at a time.
+template <typename T, bool ROWS, bool COLS>
 __global__ void __launch_bounds__(AMAX_THREADS)
 amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok,
-            uint32_t* __restrict__ amax_rm, int rm_mode, uint32_t* __restrict__ amax_tr, int tr_mode) {
-    __shared__ uint32_t col_max[AMAX_TILE_C];
+            uint32_t* __restrict__ amax_rm, uint32_t* __restrict__ amax_tr) {
+    __shared__ uint32_t col_max[COLS ? AMAX_TILE_C : 1];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t n_tc = (cols + AMAX_TILE_C - 1) / AMAX_TILE_C;
     const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * AMAX_TILE_C;
     const int64_t r0 = ((int64_t)blockIdx.x / n_tc) * AMAX_TILE_R;
-    const bool want_cols = (tr_mode == AMAX_GROUPS);
-    const bool want_rows = (rm_mode == AMAX_GROUPS);
-    if (want_cols) {
+    if constexpr (COLS) {
         for (int i = threadIdx.x; i < AMAX_TILE_C; i += AMAX_THREADS) col_max[i] = 0u;
         __syncthreads();
     }
-    uint32_t cm[16];
+    uint32_t cm[COLS ? 16 : 1];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) cm[i] = 0u;
+    for (int i = 0; i < (COLS ? 16 : 1); ++i) cm[i] = 0u;
     uint32_t all = 0u;
-    for (int rr = 0; rr < AMAX_TILE_R / 8; ++rr) {
-        const int64_t r = r0 + warp + 8 * rr;
-        if (r >= rows) break;
-        const T* row = x + r * ld;
-        uint32_t rmax = 0u;
+#pragma unroll 1
+    for (int rr = 0; rr < AMAX_TILE_R / 8; rr += 2) {
+        float v[2][4][4];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const int64_t c = c0 + (int64_t)(g * 32 + lane) * 4;
-            if (c < cols) {
-                float v[4];
-                load4(row, c, cols, vec_ok, v);
+        for (int h = 0; h < 2; ++h) {
+            const int64_t r = r0 + warp + 8 * (rr + h);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    uint32_t b = abs_bits(v[e]);
-                    rmax = max(rmax, b);
-                    cm[g * 4 + e] = max(cm[g * 4 + e], b);
-                }
+            for (int g = 0; g < 4; ++g) {
+                const int64_t c = c0 + (int64_t)(g * 32 + lane) * 4;
+                if (r < rows && c < cols) load4(x + r * ld, c, cols, vec_ok, v[h][g]);
+                else { v[h][g][0] = v[h][g][1] = v[h][g][2] = v[h][g][3] = 0.0f; }
             }
         }
-        if (want_rows) {
-            rmax = __reduce_max_sync(0xFFFFFFFFu, rmax);
-            if (lane == 0 && rmax) atomicMax(&amax_rm[r], rmax);
-        } else {
-            all = max(all, rmax);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int64_t r = r0 + warp + 8 * (rr + h);
+            uint32_t rmax = 0u;
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t b = abs_bits(v[h][g][e]);
+                    rmax = max(rmax, b);
+                    if constexpr (COLS) cm[g * 4 + e] = max(cm[g * 4 + e], b);
+                }
+            if constexpr (ROWS) {
+                rmax = __reduce_max_sync(0xFFFFFFFFu, rmax);
+                if (lane == 0 && rmax && r < rows) atomicMax(&amax_rm[r], rmax);
+            } else {
+                all = max(all, rmax);
+            }
         }
     }
-    if (rm_mode == AMAX_TENSOR) {
+    if constexpr (!ROWS && !COLS) {
         all = __reduce_max_sync(0xFFFFFFFFu, all);
         if (lane == 0 && all) atomicMax(&amax_rm[0], all);
     }
-    if (want_cols) {
+    if constexpr (COLS) {
 #pragma unroll
         for (int g = 0; g < 4; ++g)
 #pragma unroll
@@ -142,6 +146,16 @@ amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, boo
             if (c < cols && col_max[i]) atomicMax(&amax_tr[c], col_max[i]);
         }
     }
+}
+
+template <typename T>
+static void launch_amax(const void* x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok, uint32_t* amax_rm, bool want_rows,
+                        uint32_t* amax_tr, bool want_cols, unsigned grid, cudaStream_t st) {
+    const T* p = (const T*)x;
+    if (want_rows && want_cols) amax_kernel<T, true, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
+    else if (want_rows) amax_kernel<T, true, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
+    else if (want_cols) amax_kernel<T, false, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
+    else amax_kernel<T, false, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -177,24 +191,25 @@ __global__ void scales_kernel(const uint32_t* amax_rm, int64_t n_rm, float* inv_
 }
 
 // ------------------------------------------------------------------------------------------
-// Philox4x32-10 (Salmon et al., SC'11): ten rounds, two 32x32->64 multiplies per round
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds, two 32x32->64 multiplies per round.
+// The ten round keys (key + r * Weyl constants) are the same for every thread; the host
+// computes them once and passes them in the kernel parameters.
 // ------------------------------------------------------------------------------------------
-struct Philox {
-    uint32_t k0[10], k1[10];   // round keys: key + r * Weyl constants (same for every thread)
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+    uint32_t tid0, tid1;     // counter words 2 and 3 (tensor_id)
 };
 
-__device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              uint32_t key0, uint32_t key1, uint32_t out[4]) {
+__device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, const PhiloxKeys& K, uint32_t out[4]) {
+    uint32_t c2 = K.tid0, c3 = K.tid1;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        const uint32_t k0 = key0 + (uint32_t)r * 0x9E3779B9u;
-        const uint32_t k1 = key1 + (uint32_t)r * 0xBB67AE85u;
-        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-        c0 = hi1 ^ c1 ^ k0;
-        c1 = lo1;
-        c2 = hi0 ^ c3 ^ k1;
-        c3 = lo0;
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;    // one wide multiply: hi and lo
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
+        c3 = (uint32_t)p0;
     }
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
@@ -203,18 +218,19 @@ __device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, uint32_t
 // quantizer
 // ------------------------------------------------------------------------------------------
 // Def. 1 for one element; returns the code as a small integer held in a float.
-__device__ __forceinline__ float quantize_elem(float x, float inv, float qmax, bool sr, uint32_t word) {
+template <bool SRM>
+__device__ __forceinline__ float quantize_elem(float x, float inv, float qmax, uint32_t word) {
     const float t = __fmul_rn(x, inv);
     const float f = floorf(t);
     const float p = __fsub_rn(t, f);
     bool up;
-    if (sr) {
+    if constexpr (SRM) {
         // eps < p  <=>  u24 < p * 2^24 ; both sides exact in binary32
         up = __uint2float_rn(word >> 8) < __fmul_rn(p, 16777216.0f);
     } else {
         up = p >= 0.5f;
     }
-    float q = up ? __fadd_rn(f, 1.0f) : f;
+    const float q = up ? __fadd_rn(f, 1.0f) : f;
     return fminf(fmaxf(q, -qmax), qmax);
 }
 
@@ -225,13 +241,28 @@ __device__ __forceinline__ uint32_t pack4(uint32_t b0, uint32_t b1, uint32_t b2,
     return __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
 }
 
+template <bool SRM>
+__device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3, float qmax,
+                                              const uint32_t rnd[4]) {
+    return pack4(code_bits(quantize_elem<SRM>(v[0], i0, qmax, rnd[0])), code_bits(quantize_elem<SRM>(v[1], i1, qmax, rnd[1])),
+                 code_bits(quantize_elem<SRM>(v[2], i2, qmax, rnd[2])), code_bits(quantize_elem<SRM>(v[3], i3, qmax, rnd[3])));
+}
+
+// 4x4 byte transpose: w[i] holds columns c..c+3 of row i -> o[e] holds rows 0..3 of column c+e
+__device__ __forceinline__ void transpose4x4(const uint32_t w[4], uint32_t o[4]) {
+    const uint32_t lo01 = __byte_perm(w[0], w[1], 0x5140), hi01 = __byte_perm(w[0], w[1], 0x7362);
+    const uint32_t lo23 = __byte_perm(w[2], w[3], 0x5140), hi23 = __byte_perm(w[2], w[3], 0x7362);
+    o[0] = __byte_perm(lo01, lo23, 0x5410); o[1] = __byte_perm(lo01, lo23, 0x7632);
+    o[2] = __byte_perm(hi01, hi23, 0x5410); o[3] = __byte_perm(hi01, hi23, 0x7632);
+}
+
 constexpr int Q_THREADS = 256;
 constexpr int Q_TILE = 128;          // 128 x 128 elements per CTA
 
 struct QuantParams {
     int64_t rows, cols, ld;
     uint64_t index_offset;
-    uint32_t key0, key1, tid0, tid1;
+    PhiloxKeys keys;
     float qmax;
     int sr;                       // 1 = SR, 0 = RTN
     int per_row;                  // step size per row of each layout
@@ -243,7 +274,129 @@ struct QuantParams {
     int vec_rm, vec_tr;           // 4-byte code stores allowed
 };
 
-template <typename T, bool ALIGNED>
+// Row-wise read of the transposed tile and its stores: one warp per tile column, lane = row quad.
+__device__ __forceinline__ void store_transposed_tile(const uint32_t* tileT, const QuantParams& P, int64_t r0, int64_t c0,
+                                                      int warp, int lane) {
+    const int64_t r = r0 + lane * 4;
+#pragma unroll 4
+    for (int col = warp; col < Q_TILE; col += 8) {
+        const int64_t cc = c0 + col;
+        if (cc >= P.cols || r >= P.rows) continue;
+        const uint32_t w = tileT[col * 32 + (lane ^ ((col >> 2) & 31))];
+        int8_t* dst = P.codes_tr + cc * P.ld_tr + r;
+        if (P.vec_tr && r + 4 <= P.rows) {
+            *reinterpret_cast<uint32_t*>(dst) = w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (r + e < P.rows) dst[e] = (int8_t)((w >> (8 * e)) & 0xFF);
+        }
+    }
+}
+
+// Raw 4-element group as loaded, and its widening to binary32.
+template <typename T> struct Raw4;
+template <> struct Raw4<float> { using type = float4; };
+template <> struct Raw4<__nv_bfloat16> { using type = uint2; };
+
+__device__ __forceinline__ void widen(const float4& q, float v[4]) { v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w; }
+__device__ __forceinline__ void widen(const uint2& q, float v[4]) {
+    v[0] = __uint_as_float(q.x << 16); v[1] = __uint_as_float(q.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(q.y << 16); v[3] = __uint_as_float(q.y & 0xFFFF0000u);
+}
+
+// Fast path: extents, pitches and index offset are multiples of 4, pointers are aligned, so every
+// 4-element group is one vector load, one Philox block and one 4-byte store.  LAYOUT bit 0 = row-major
+// codes wanted, bit 1 = transposed codes wanted.  The loads of the next row quad are issued before the
+// current one is processed, which keeps two quads of loads in flight per thread.
+template <typename T, bool SRM, int LAYOUT, bool PER_ROW>
+__global__ void __launch_bounds__(Q_THREADS)
+quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P) {
+    using Raw = typename Raw4<T>::type;
+    constexpr bool WANT_RM = (LAYOUT & 1) != 0, WANT_TR = (LAYOUT & 2) != 0;
+    constexpr bool TWO_STEPS = WANT_TR && PER_ROW;     // transposed layout has its own step sizes
+    __shared__ uint32_t tileT[WANT_TR ? Q_TILE * (Q_TILE / 4) : 1];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t n_tc = (P.cols + Q_TILE - 1) / Q_TILE;
+    const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * Q_TILE;
+    const int64_t r0 = ((int64_t)blockIdx.x / n_tc) * Q_TILE;
+    const int64_t c = c0 + lane * 4;
+    const bool col_ok = c < P.cols;                     // cols % 4 == 0: a group is all in or all out
+    const float qmax = P.qmax;
+
+    float ic[4] = {0.f, 0.f, 0.f, 0.f};
+    if constexpr (TWO_STEPS) {
+        if (col_ok) { const float4 t = *reinterpret_cast<const float4*>(P.inv_tr + c); ic[0] = t.x; ic[1] = t.y; ic[2] = t.z; ic[3] = t.w; }
+    }
+    const float inv_tensor = PER_ROW ? 0.0f : P.inv_rm[0];
+
+    const T* xp = x + (r0 + warp * 4) * P.ld + c;       // first row of this thread's first quad
+    const int64_t quad_stride = 32 * P.ld;              // 8 warps x 4 rows between successive quads
+    // Philox block index of (row, c): (index_offset + row * cols + c) / 4, advanced by cols / 4 per row
+    uint64_t j = (P.index_offset + (uint64_t)(r0 + warp * 4) * (uint64_t)P.cols + (uint64_t)c) >> 2;
+    const uint64_t j_row = (uint64_t)P.cols >> 2, j_quad = 32 * j_row;
+
+    Raw cur[4], nxt[4];
+    float inv_cur[4], inv_nxt[4];
+    auto load_quad = [&](int it, Raw raw[4], float inv_r[4]) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t r = r0 + (warp + 8 * it) * 4 + i;
+            if (col_ok && r < P.rows) {
+                raw[i] = __ldcs(reinterpret_cast<const Raw*>(xp + (int64_t)it * quad_stride + i * P.ld));
+                if constexpr (PER_ROW && WANT_RM) inv_r[i] = P.inv_rm[r];
+            } else {
+                raw[i] = Raw{};
+                if constexpr (PER_ROW && WANT_RM) inv_r[i] = 0.0f;
+            }
+        }
+    };
+    load_quad(0, cur, inv_cur);
+
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        if (it + 1 < 4) load_quad(it + 1, nxt, inv_nxt);
+        const int rq = warp + 8 * it;
+        uint32_t wr[4], wt[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float v[4];
+            widen(cur[i], v);
+            uint32_t rnd[4] = {0u, 0u, 0u, 0u};
+            if constexpr (SRM) {
+                const uint64_t jj = j + (uint64_t)i * j_row;
+                philox_rounds((uint32_t)jj, (uint32_t)(jj >> 32), P.keys, rnd);
+            }
+            if constexpr (WANT_RM || !TWO_STEPS) {
+                const float ir = (PER_ROW && WANT_RM) ? inv_cur[i] : inv_tensor;
+                wr[i] = quantize4<SRM>(v, ir, ir, ir, ir, qmax, rnd);
+            }
+            if constexpr (TWO_STEPS) wt[i] = quantize4<SRM>(v, ic[0], ic[1], ic[2], ic[3], qmax, rnd);
+            else wt[i] = wr[i];
+            if constexpr (WANT_RM) {
+                const int64_t r = r0 + rq * 4 + i;
+                if (col_ok && r < P.rows) *reinterpret_cast<uint32_t*>(P.codes_rm + r * P.ld_rm + c) = wr[i];
+            }
+        }
+        if constexpr (WANT_TR) {
+            uint32_t o[4];
+            transpose4x4(wt, o);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) tileT[(lane * 4 + e) * 32 + (rq ^ lane)] = o[e];
+        }
+        j += j_quad;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { cur[i] = nxt[i]; inv_cur[i] = inv_nxt[i]; }
+    }
+    if constexpr (WANT_TR) {
+        __syncthreads();
+        store_transposed_tile(tileT, P, r0, c0, warp, lane);
+    }
+}
+
+// General path: any extent, pitch, alignment and index offset; one Philox block per element
+// when the groups of four do not line up with the flat index.  Same results as the fast path.
+template <typename T>
 __global__ void __launch_bounds__(Q_THREADS)
 quantize_kernel(const T* __restrict__ x, const QuantParams P) {
     // transposed tile: column c of the tile holds 128 row codes = 32 words; the word index is
@@ -280,35 +433,24 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
                 uint32_t rnd[4] = {0u, 0u, 0u, 0u};
                 if (sr) {
                     const uint64_t i0 = P.index_offset + (uint64_t)r * (uint64_t)P.cols + (uint64_t)c;
-                    if constexpr (ALIGNED) {
-                        const uint64_t j = i0 >> 2;
-                        philox_rounds((uint32_t)j, (uint32_t)(j >> 32), P.tid0, P.tid1, P.key0, P.key1, rnd);
-                    } else {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const uint64_t ie = i0 + e, j = ie >> 2;
-                            uint32_t o[4];
-                            philox_rounds((uint32_t)j, (uint32_t)(j >> 32), P.tid0, P.tid1, P.key0, P.key1, o);
-                            const uint32_t s = (uint32_t)ie & 3u;
-                            rnd[e] = s == 0 ? o[0] : s == 1 ? o[1] : s == 2 ? o[2] : o[3];
-                        }
+                    for (int e = 0; e < 4; ++e) {
+                        const uint64_t ie = i0 + e, jb = ie >> 2;
+                        uint32_t o[4];
+                        philox_rounds((uint32_t)jb, (uint32_t)(jb >> 32), P.keys, o);
+                        const uint32_t s = (uint32_t)ie & 3u;
+                        rnd[e] = s == 0 ? o[0] : s == 1 ? o[1] : s == 2 ? o[2] : o[3];
                     }
                 }
                 const float inv_r = P.per_row ? P.inv_rm[want_rm ? r : 0] : inv_tensor;
-                if (want_rm || !two_steps) {
-                    uint32_t b[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) b[e] = code_bits(quantize_elem(v[e], inv_r, P.qmax, sr, rnd[e]));
-                    wr[i] = pack4(b[0], b[1], b[2], b[3]);
-                }
-                if (two_steps) {
-                    uint32_t b[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) b[e] = code_bits(quantize_elem(v[e], inv_c[e], P.qmax, sr, rnd[e]));
-                    wt[i] = pack4(b[0], b[1], b[2], b[3]);
-                } else {
+                if (want_rm || !two_steps)
+                    wr[i] = sr ? quantize4<true>(v, inv_r, inv_r, inv_r, inv_r, P.qmax, rnd)
+                               : quantize4<false>(v, inv_r, inv_r, inv_r, inv_r, P.qmax, rnd);
+                if (two_steps)
+                    wt[i] = sr ? quantize4<true>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], P.qmax, rnd)
+                               : quantize4<false>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], P.qmax, rnd);
+                else
                     wt[i] = wr[i];
-                }
                 if (want_rm) {
                     int8_t* dst = P.codes_rm + r * P.ld_rm + c;
                     if (P.vec_rm && c + 4 <= P.cols) {
@@ -322,39 +464,42 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
             }
         }
         if (want_tr) {
-            // 4x4 byte transpose: wt[i] holds columns c..c+3 of row i -> o[e] holds rows 0..3 of column c+e
-            const uint32_t lo01 = __byte_perm(wt[0], wt[1], 0x5140), hi01 = __byte_perm(wt[0], wt[1], 0x7362);
-            const uint32_t lo23 = __byte_perm(wt[2], wt[3], 0x5140), hi23 = __byte_perm(wt[2], wt[3], 0x7362);
             uint32_t o[4];
-            o[0] = __byte_perm(lo01, lo23, 0x5410); o[1] = __byte_perm(lo01, lo23, 0x7632);
-            o[2] = __byte_perm(hi01, hi23, 0x5410); o[3] = __byte_perm(hi01, hi23, 0x7632);
+            transpose4x4(wt, o);
 #pragma unroll
             for (int e = 0; e < 4; ++e) tileT[(lane * 4 + e) * 32 + (rq ^ lane)] = o[e];
         }
     }
     if (!want_tr) return;
     __syncthreads();
-    // row-wise read of the transposed tile: one warp per tile column, lane = row quad
-    const int64_t r = r0 + lane * 4;
-#pragma unroll 4
-    for (int col = warp; col < Q_TILE; col += 8) {
-        const int64_t cc = c0 + col;
-        if (cc >= P.cols || r >= P.rows) continue;
-        const uint32_t w = tileT[col * 32 + (lane ^ ((col >> 2) & 31))];
-        int8_t* dst = P.codes_tr + cc * P.ld_tr + r;
-        if (P.vec_tr && r + 4 <= P.rows) {
-            *reinterpret_cast<uint32_t*>(dst) = w;
-        } else {
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (r + e < P.rows) dst[e] = (int8_t)((w >> (8 * e)) & 0xFF);
-        }
-    }
+    store_transposed_tile(tileT, P, r0, c0, warp, lane);
 }
 
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
+template <typename T, bool SRM, int LAYOUT>
+static void launch_fast_pr(bool per_row, const void* x, const QuantParams& P, unsigned grid, cudaStream_t st) {
+    if (per_row) quantize_fast_kernel<T, SRM, LAYOUT, true><<<grid, Q_THREADS, 0, st>>>((const T*)x, P);
+    else quantize_fast_kernel<T, SRM, LAYOUT, false><<<grid, Q_THREADS, 0, st>>>((const T*)x, P);
+}
+template <typename T, bool SRM>
+static void launch_fast_layout(int layout, bool per_row, const void* x, const QuantParams& P, unsigned grid, cudaStream_t st) {
+    if (layout == 1) launch_fast_pr<T, SRM, 1>(per_row, x, P, grid, st);
+    else if (layout == 2) launch_fast_pr<T, SRM, 2>(per_row, x, P, grid, st);
+    else launch_fast_pr<T, SRM, 3>(per_row, x, P, grid, st);
+}
+static void launch_fast(srq_dtype_t dt, bool sr, int layout, bool per_row, const void* x, const QuantParams& P, unsigned grid,
+                        cudaStream_t st) {
+    if (dt == SRQ_F32) {
+        if (sr) launch_fast_layout<float, true>(layout, per_row, x, P, grid, st);
+        else launch_fast_layout<float, false>(layout, per_row, x, P, grid, st);
+    } else {
+        if (sr) launch_fast_layout<__nv_bfloat16, true>(layout, per_row, x, P, grid, st);
+        else launch_fast_layout<__nv_bfloat16, false>(layout, per_row, x, P, grid, st);
+    }
+}
+
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream) {
     const bool want_rm = a.codes_rm != nullptr, want_tr = a.codes_tr != nullptr;
     const bool per_row = a.q.scale == SRQ_PER_ROW;
@@ -377,14 +522,9 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     const bool vec_in = ((uintptr_t)a.x % (4 * esize) == 0) && (a.ld % 4 == 0);
     {
         const unsigned grid = (unsigned)(((cols + AMAX_TILE_C - 1) / AMAX_TILE_C) * ((rows + AMAX_TILE_R - 1) / AMAX_TILE_R));
-        const int rm_mode = per_row ? (want_rm ? AMAX_GROUPS : AMAX_NONE) : AMAX_TENSOR;
-        const int tr_mode = per_row ? (want_tr ? AMAX_GROUPS : AMAX_NONE) : AMAX_NONE;
-        if (a.dt == SRQ_F32)
-            amax_kernel<float><<<grid, AMAX_THREADS, 0, stream>>>((const float*)a.x, rows, cols, a.ld, vec_in,
-                                                                 amax_rm, rm_mode, amax_tr, tr_mode);
-        else
-            amax_kernel<__nv_bfloat16><<<grid, AMAX_THREADS, 0, stream>>>((const __nv_bfloat16*)a.x, rows, cols, a.ld,
-                                                                         vec_in, amax_rm, rm_mode, amax_tr, tr_mode);
+        const bool want_rows = per_row && want_rm, want_cols = per_row && want_tr;
+        if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, vec_in, amax_rm, want_rows, amax_tr, want_cols, grid, stream);
+        else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, vec_in, amax_rm, want_rows, amax_tr, want_cols, grid, stream);
         ++g_launches;
     }
     {
@@ -402,8 +542,11 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         QuantParams P;
         P.rows = rows; P.cols = cols; P.ld = a.ld;
         P.index_offset = a.q.index_offset;
-        P.key0 = (uint32_t)a.q.seed; P.key1 = (uint32_t)(a.q.seed >> 32);
-        P.tid0 = (uint32_t)a.q.tensor_id; P.tid1 = (uint32_t)(a.q.tensor_id >> 32);
+        for (int r = 0; r < 10; ++r) {
+            P.keys.k0[r] = (uint32_t)a.q.seed + (uint32_t)r * 0x9E3779B9u;
+            P.keys.k1[r] = (uint32_t)(a.q.seed >> 32) + (uint32_t)r * 0xBB67AE85u;
+        }
+        P.keys.tid0 = (uint32_t)a.q.tensor_id; P.keys.tid1 = (uint32_t)(a.q.tensor_id >> 32);
         P.qmax = qmax;
         P.sr = a.q.round == SRQ_SR;
         P.per_row = per_row;
@@ -413,15 +556,12 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         P.vec_in = vec_in;
         P.vec_rm = want_rm && ((uintptr_t)a.codes_rm % 4 == 0) && (a.ld_rm % 4 == 0);
         P.vec_tr = want_tr && ((uintptr_t)a.codes_tr % 4 == 0) && (a.ld_tr % 4 == 0);
-        const bool aligned = (cols % 4 == 0) && (a.q.index_offset % 4 == 0);
+        const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && (!want_rm || P.vec_rm) &&
+                          (!want_tr || (P.vec_tr && rows % 4 == 0));
         const unsigned grid = (unsigned)(((cols + Q_TILE - 1) / Q_TILE) * ((rows + Q_TILE - 1) / Q_TILE));
-        if (a.dt == SRQ_F32) {
-            if (aligned) quantize_kernel<float, true><<<grid, Q_THREADS, 0, stream>>>((const float*)a.x, P);
-            else quantize_kernel<float, false><<<grid, Q_THREADS, 0, stream>>>((const float*)a.x, P);
-        } else {
-            if (aligned) quantize_kernel<__nv_bfloat16, true><<<grid, Q_THREADS, 0, stream>>>((const __nv_bfloat16*)a.x, P);
-            else quantize_kernel<__nv_bfloat16, false><<<grid, Q_THREADS, 0, stream>>>((const __nv_bfloat16*)a.x, P);
-        }
+        if (fast) launch_fast(a.dt, P.sr != 0, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);
+        else if (a.dt == SRQ_F32) quantize_kernel<float><<<grid, Q_THREADS, 0, stream>>>((const float*)a.x, P);
+        else quantize_kernel<__nv_bfloat16><<<grid, Q_THREADS, 0, stream>>>((const __nv_bfloat16*)a.x, P);
         ++g_launches;
     }
     return cudaGetLastError();
