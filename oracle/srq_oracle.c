@@ -118,13 +118,18 @@ void orc_scale_from_absmax(float m, int bits, float *delta, float *inv)
 /* Def. 1-3: one element                                                    */
 /* ---------------------------------------------------------------------- */
 /*
- * Code q such that Q_D(x, eps) = q * D, with x/D evaluated as x * inv:
- *   t = x * inv;  f = floor(t);  p = t - f   (the fractional part)
+ * Code q such that Q_D(x, eps) = q * D, with x/D evaluated as t = x * inv
+ * (one binary32 multiply).  With f = floor(t) and the fractional part
+ * p = t - f:
  *   SR : round up  iff  eps < p   (strict, so grid-exact x never moves;
  *        Def. 1 rounds down when p < eps, up otherwise; with eps on a
  *        2^-24 lattice the strict form keeps P(up) within 2^-24 of p)
  *   RTN: round up  iff  p >= 1/2  (Def. 1 with eps = 1/2; a tie goes up,
  *        i.e. toward +infinity, Def. 2)
+ * Def. 1 states these comparisons on real numbers, so they are evaluated
+ * without rounding p: multiplied through by 2^24, eps < t - f becomes
+ * u24 + f 2^24 < t 2^24, and every term of that is exact in binary64
+ * (t has 24 significant bits, f is an integer of magnitude <= 2^8).
  *   q = f + up, clamped to [-qmax, qmax] (the rounded product t can exceed
  *   qmax by one ulp at the extreme element).
  */
@@ -132,15 +137,13 @@ int orc_quantize_scalar(float x, float inv, int bits, int round_mode, uint32_t u
 {
     int qmax = orc_qmax(bits);
     float t = x * inv;
-    float f = floorf(t);
-    float p = t - f;
+    double td = (double)t;
+    double f = floor(td);
     int up;
-    if (round_mode == ORC_SR) {
-        float eps = (float)u24 * 0x1p-24f; /* exact: 24-bit integer times a power of two */
-        up = (eps < p);
-    } else {
-        up = (p >= 0.5f);
-    }
+    if (round_mode == ORC_SR)
+        up = ((double)u24 + f * 0x1p24) < td * 0x1p24;
+    else
+        up = (f * 0x1p24 + 0x1p23) <= td * 0x1p24;
     int q = (int)f + up;
     if (q > qmax) q = qmax;
     if (q < -qmax) q = -qmax;

@@ -61,28 +61,34 @@ def scale_ref(m, bits):
 
 
 def quantize_scalar_ref(x, inv, bits, sr, u24=0):
-    """Def. 1 for one element; the threshold comparison is done in exact rationals."""
-    t = np.float32(np.float32(x) * np.float32(inv))
-    f = np.floor(t)
-    p = np.float32(t - f)
+    """Def. 1 for one element: t in binary32, everything after it in exact rationals."""
+    t = Fraction(float(np.float32(np.float32(x) * np.float32(inv))))
+    f = t.numerator // t.denominator
+    p = t - f
     if sr:
-        up = Fraction(int(u24), 2 ** 24) < Fraction(float(p))
+        up = Fraction(int(u24), 2 ** 24) < p
     else:
-        up = Fraction(float(p)) >= Fraction(1, 2)
+        up = p >= Fraction(1, 2)
     q = int(f) + int(up)
     return max(-qmax_of(bits), min(qmax_of(bits), q))
 
 
 def quantize_matrix_ref(x, inv, bits, sr, u24):
-    """Vectorised Def. 1 with a broadcastable inv; same binary32 steps."""
+    """Def. 1 over a matrix with a broadcastable inv: t in binary32, the threshold comparison in
+    exact rationals (slow; for the small matrices of the tests)."""
     x = np.asarray(x, dtype=np.float32)
     t = (x * np.asarray(inv, dtype=np.float32)).astype(np.float32)
-    f = np.floor(t)
-    p = (t - f).astype(np.float32)
-    if sr:
-        # p * 2^24 is exact in float64; compare as integers-or-fractions
-        up = u24.astype(np.float64) < p.astype(np.float64) * 2.0 ** 24
-    else:
-        up = p >= np.float32(0.5)
-    q = f.astype(np.int64) + up.astype(np.int64)
-    return np.clip(q, -qmax_of(bits), qmax_of(bits)).astype(np.int8)
+    out = np.empty(t.shape, dtype=np.int64)
+    flat_t = t.ravel()
+    flat_u = None if u24 is None else np.asarray(u24).ravel()
+    o = out.ravel()
+    for i in range(flat_t.size):
+        T = Fraction(float(flat_t[i])) * 2 ** 24            # exact
+        f = T.numerator // (T.denominator * 2 ** 24)          # floor(t)
+        P = T - f * 2 ** 24                                    # p * 2^24, exact
+        if sr:
+            up = int(flat_u[i]) < P
+        else:
+            up = P >= 2 ** 23
+        o[i] = f + int(up)
+    return np.clip(out, -qmax_of(bits), qmax_of(bits)).astype(np.int8)

@@ -89,7 +89,10 @@ def test_worked_example_sum_of_ten_0p7():
 
 # ---------------------------------------------------------------- Def. 3: SR
 @pytest.mark.parametrize("t", [0.0, 2.0 ** -24, 0.3, 0.5, 0.7, 1 - 2.0 ** -24, 5.25, -0.3, -7.75,
-                               -100.5, 126.999])
+                               -100.5, 126.999,
+                               # fractional parts that binary32 cannot hold (t - floor(t) would round)
+                               -2.0 ** -30, -10066331 * 2.0 ** -25, -8388609 * 2.0 ** -25 , 2.0 ** -40,
+                               -1e-30, 1e-40, -1e-40])
 def test_sr_probability_of_rounding_up_is_the_fraction_exactly(t):
     t32 = np.float32(t)
     f = math.floor(Fraction(float(t32)))
