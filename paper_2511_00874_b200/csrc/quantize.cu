@@ -5,15 +5,17 @@
 //                    binary32 bit pattern (non-negative floats order like unsigned integers,
 //                    so atomicMax on the bits is exact and order independent)
 //   scales_kernel    D = m / qmax and 1/D = qmax / m per group (one IEEE division each)
-//   quantize_kernel  second read of x; t = x * (1/D), f = floor(t), p = t - f;
-//                    SR: up iff u24 * 2^-24 < p with u24 from Philox4x32-10 keyed by
-//                    (seed, tensor_id, flat index); RTN: up iff p >= 1/2; code = clamp(f + up).
+//   quantize_kernel  second read of x; t = x * (1/D) (one binary32 multiply), then Def. 1 on
+//                    real numbers: SR rounds up iff u24 * 2^-24 < frac(t) with u24 from
+//                    Philox4x32-10 keyed by (seed, tensor_id, flat index); RTN rounds up iff
+//                    frac(t) >= 1/2; code = clamp(floor(t) + up).  The comparison is evaluated
+//                    exactly, in fixed point with 24 fractional bits (see quantize_elem).
 //                    Writes the row-major code layout directly and the transposed layout
 //                    through a swizzled shared-memory tile, so that both are stored with
 //                    full 128-byte lines.
 //
-// Arithmetic that decides a code uses explicit round-to-nearest intrinsics so that the
-// compiler cannot contract x * inv - f into a fused multiply-add.
+// The two multiplies that produce the fixed-point quotient use explicit round-to-nearest
+// intrinsics so that the compiler cannot merge them.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -217,35 +219,38 @@ __device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, const Ph
 // ------------------------------------------------------------------------------------------
 // quantizer
 // ------------------------------------------------------------------------------------------
-// Def. 1 for one element; returns the code as a small integer held in a float.
+// Def. 1 for one element; returns the code as a two's complement integer.
+// The comparison frac(t) > eps of Def. 1 is taken on real numbers, with no rounding of the
+// fractional part, in fixed point with 24 fractional bits.  Let S = t * 2^24 (exact: a power-of
+// -two scaling of the binary32 product t = x * (1/D)), u = u24 the 24-bit threshold.
+//   SR : for an integer L, L < S  <=>  L < ceil(S); with C = ceil(S) = f' 2^24 + low,
+//        0 <= low < 2^24, the code is f' + (u < low) = (C + (2^24 - 1 - u)) >> 24.
+//        (When S is not an integer and C is a multiple of 2^24, f' is floor(t) + 1 and
+//        low = 0: the code is f' either way, as Def. 1 gives with frac(t) > 1 - 2^-24 > eps.)
+//   RTN: frac(t) >= 1/2  <=>  floor(S) - floor(t) 2^24 >= 2^23, so the code is
+//        (floor(S) + 2^23) >> 24.
+// Clamping C to +-qmax 2^24 first clamps the code to +-qmax and keeps the sum inside int32.
 template <bool SRM>
-__device__ __forceinline__ float quantize_elem(float x, float inv, float qmax, uint32_t word) {
-    const float t = __fmul_rn(x, inv);
-    const float f = floorf(t);
-    const float p = __fsub_rn(t, f);
-    bool up;
+__device__ __forceinline__ int quantize_elem(float x, float inv, int lim, uint32_t word) {
+    const float s = __fmul_rn(__fmul_rn(x, inv), 16777216.0f);
     if constexpr (SRM) {
-        // eps < p  <=>  u24 < p * 2^24 ; both sides exact in binary32
-        up = __uint2float_rn(word >> 8) < __fmul_rn(p, 16777216.0f);
+        const int c = min(max(__float2int_ru(s), -lim), lim);
+        return (c + (int)(0x00FFFFFFu - (word >> 8))) >> 24;
     } else {
-        up = p >= 0.5f;
+        const int c = min(max(__float2int_rd(s), -lim), lim);
+        return (c + 0x00800000) >> 24;
     }
-    const float q = up ? __fadd_rn(f, 1.0f) : f;
-    return fminf(fmaxf(q, -qmax), qmax);
 }
 
-// Low byte of the two's complement integer held exactly in q (|q| <= 127).
-__device__ __forceinline__ uint32_t code_bits(float q) { return __float_as_uint(__fadd_rn(q, 12582912.0f)); }
-
-__device__ __forceinline__ uint32_t pack4(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3) {
-    return __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
+__device__ __forceinline__ uint32_t pack4(int b0, int b1, int b2, int b3) {
+    return __byte_perm(__byte_perm((uint32_t)b0, (uint32_t)b1, 0x0040), __byte_perm((uint32_t)b2, (uint32_t)b3, 0x0040), 0x5410);
 }
 
 template <bool SRM>
-__device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3, float qmax,
+__device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3, int lim,
                                               const uint32_t rnd[4]) {
-    return pack4(code_bits(quantize_elem<SRM>(v[0], i0, qmax, rnd[0])), code_bits(quantize_elem<SRM>(v[1], i1, qmax, rnd[1])),
-                 code_bits(quantize_elem<SRM>(v[2], i2, qmax, rnd[2])), code_bits(quantize_elem<SRM>(v[3], i3, qmax, rnd[3])));
+    return pack4(quantize_elem<SRM>(v[0], i0, lim, rnd[0]), quantize_elem<SRM>(v[1], i1, lim, rnd[1]),
+                 quantize_elem<SRM>(v[2], i2, lim, rnd[2]), quantize_elem<SRM>(v[3], i3, lim, rnd[3]));
 }
 
 // 4x4 byte transpose: w[i] holds columns c..c+3 of row i -> o[e] holds rows 0..3 of column c+e
@@ -263,7 +268,7 @@ struct QuantParams {
     int64_t rows, cols, ld;
     uint64_t index_offset;
     PhiloxKeys keys;
-    float qmax;
+    int lim;                      // qmax * 2^24: clamp of the fixed-point quotient
     int sr;                       // 1 = SR, 0 = RTN
     int per_row;                  // step size per row of each layout
     int8_t* codes_rm; int64_t ld_rm;
@@ -322,7 +327,7 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
     const int64_t r0 = ((int64_t)blockIdx.x / n_tc) * Q_TILE;
     const int64_t c = c0 + lane * 4;
     const bool col_ok = c < P.cols;                     // cols % 4 == 0: a group is all in or all out
-    const float qmax = P.qmax;
+    const int lim = P.lim;
 
     float ic[4] = {0.f, 0.f, 0.f, 0.f};
     if constexpr (TWO_STEPS) {
@@ -369,9 +374,9 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
             }
             if constexpr (WANT_RM || !TWO_STEPS) {
                 const float ir = (PER_ROW && WANT_RM) ? inv_cur[i] : inv_tensor;
-                wr[i] = quantize4<SRM>(v, ir, ir, ir, ir, qmax, rnd);
+                wr[i] = quantize4<SRM>(v, ir, ir, ir, ir, lim, rnd);
             }
-            if constexpr (TWO_STEPS) wt[i] = quantize4<SRM>(v, ic[0], ic[1], ic[2], ic[3], qmax, rnd);
+            if constexpr (TWO_STEPS) wt[i] = quantize4<SRM>(v, ic[0], ic[1], ic[2], ic[3], lim, rnd);
             else wt[i] = wr[i];
             if constexpr (WANT_RM) {
                 const int64_t r = r0 + rq * 4 + i;
@@ -444,11 +449,11 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
                 }
                 const float inv_r = P.per_row ? P.inv_rm[want_rm ? r : 0] : inv_tensor;
                 if (want_rm || !two_steps)
-                    wr[i] = sr ? quantize4<true>(v, inv_r, inv_r, inv_r, inv_r, P.qmax, rnd)
-                               : quantize4<false>(v, inv_r, inv_r, inv_r, inv_r, P.qmax, rnd);
+                    wr[i] = sr ? quantize4<true>(v, inv_r, inv_r, inv_r, inv_r, P.lim, rnd)
+                               : quantize4<false>(v, inv_r, inv_r, inv_r, inv_r, P.lim, rnd);
                 if (two_steps)
-                    wt[i] = sr ? quantize4<true>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], P.qmax, rnd)
-                               : quantize4<false>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], P.qmax, rnd);
+                    wt[i] = sr ? quantize4<true>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], P.lim, rnd)
+                               : quantize4<false>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], P.lim, rnd);
                 else
                     wt[i] = wr[i];
                 if (want_rm) {
@@ -547,7 +552,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
             P.keys.k1[r] = (uint32_t)(a.q.seed >> 32) + (uint32_t)r * 0xBB67AE85u;
         }
         P.keys.tid0 = (uint32_t)a.q.tensor_id; P.keys.tid1 = (uint32_t)(a.q.tensor_id >> 32);
-        P.qmax = qmax;
+        P.lim = ((1 << (a.q.bits - 1)) - 1) << 24;
         P.sr = a.q.round == SRQ_SR;
         P.per_row = per_row;
         P.codes_rm = a.codes_rm; P.ld_rm = a.ld_rm;
