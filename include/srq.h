@@ -120,6 +120,32 @@ srq_status_t sr_quantize(const void *x, srq_dtype_t dt, int64_t rows, int64_t co
                          void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * sr_quantize for callers that cannot allocate device memory.  (The paper has no counterpart
+ * of this entry point; it exists for deployment reasons only.)  Same operation, arguments and
+ * results as sr_quantize, but without a workspace: the scratch words come from a 1 MiB array
+ * built into the library, which every device that loads the library holds until the process
+ * exits.  Meant for code that runs where cudaMalloc is unavailable or unwelcome: inside a
+ * framework whose memory pool is already fully assigned, in a plug-in that is handed only its
+ * input and output tensors, or in a latency-critical loop that must not hit the allocator's
+ * implicit synchronisation.  The call itself allocates nothing, on the host or the device.
+ *   - Limit: 256 + 2 * (pad64(rows) + pad64(cols)) * 4 bytes must fit in 1 MiB, pad64 rounding
+ *     up to a multiple of 64 (about rows + cols <= 131000); larger inputs return
+ *     SRQ_ERR_WORKSPACE and enqueue nothing.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - device_status: optional caller-owned device word (4-byte aligned) that is cleared and
+ *     then receives SRQ_ERR_NONFINITE if an input group is not finite; pass NULL to ignore.
+ *   - All calls on a device share the array, and it keeps the previous call's contents; each
+ *     call clears what it needs.  Calls whose kernels may overlap on the same device (streams
+ *     with no ordering between them) race with each other: order them, or use sr_quantize.
+ */
+srq_status_t sr_quantize_static(const void *x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+                                const srq_qspec_t *q,
+                                int8_t *codes_rm, int64_t ld_rm, float *scale_rm,
+                                int8_t *codes_tr, int64_t ld_tr, float *scale_tr,
+                                uint32_t *device_status, void *cuda_stream);
+
+/*
  * The product of two quantized matrices (mixed-precision matmul subsection): int8 codes
  * a[M, Kc] (pitch lda) and b[N, Kc] (pitch ldb), both with the contracted axis contiguous,
  * multiplied on the tensor cores with exact int32 accumulation, then

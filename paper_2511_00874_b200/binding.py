@@ -25,7 +25,7 @@ PER_TENSOR, PER_ROW = 0, 1
 SR, RTN = 0, 1
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
-           "sr_quantize", "srq_gemm_i8", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight",
+           "sr_quantize", "sr_quantize_static", "srq_gemm_i8", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight",
            "srq_poll_status", "srq_status_string", "srq_launch_count"]
 
 
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
     L.srq_workspace_bytes.restype = sz
     L.sr_quantize.argtypes = [vp, ctypes.c_int, i64, i64, i64, qp, vp, i64, vp, vp, i64, vp, vp, sz, vp]
     L.sr_quantize.restype = ctypes.c_int
+    L.sr_quantize_static.argtypes = [vp, ctypes.c_int, i64, i64, i64, qp, vp, i64, vp, vp, i64, vp, vp, vp]
+    L.sr_quantize_static.restype = ctypes.c_int
     L.srq_gemm_i8.argtypes = [vp, i64, vp, i64, i64, i64, i64, vp, i32, vp, i32, vp, i64, vp, vp, sz, vp]
     L.srq_gemm_i8.restype = ctypes.c_int
     for name in ("qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight"):
@@ -167,6 +169,25 @@ def sr_quantize(x: torch.Tensor, q: QSpec, codes_rm: Optional[torch.Tensor] = No
                            _ptr(codes_tr), codes_tr.stride(0) if codes_tr is not None else 0,
                            _ptr(scale_tr), ws.data_ptr(), ws.numel(), _stream())
     _check(st, "sr_quantize")
+
+
+def sr_quantize_static(x: torch.Tensor, q: QSpec, codes_rm: Optional[torch.Tensor] = None,
+                       scale_rm: Optional[torch.Tensor] = None, codes_tr: Optional[torch.Tensor] = None,
+                       scale_tr: Optional[torch.Tensor] = None,
+                       device_status: Optional[torch.Tensor] = None) -> None:
+    """sr_quantize without a workspace, for callers that must not allocate device memory: the
+    scratch is the library's built-in 1 MiB array (shared by all calls on the device, so calls
+    that may overlap must be ordered).  ``device_status`` is an optional int32 CUDA tensor of
+    one element that receives the device-side status."""
+    _dev2d(x, "x")
+    rows, cols = x.shape
+    cq = q.c()
+    st = lib().sr_quantize_static(x.data_ptr(), _dtype_of(x), rows, cols, x.stride(0), ctypes.byref(cq),
+                                  _ptr(codes_rm), codes_rm.stride(0) if codes_rm is not None else 0,
+                                  _ptr(scale_rm),
+                                  _ptr(codes_tr), codes_tr.stride(0) if codes_tr is not None else 0,
+                                  _ptr(scale_tr), _ptr(device_status), _stream())
+    _check(st, "sr_quantize_static")
 
 
 def srq_gemm_i8(a: torch.Tensor, b: torch.Tensor, s_row: torch.Tensor, s_col: torch.Tensor,

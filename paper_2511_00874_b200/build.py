@@ -11,7 +11,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB = os.path.join(_PKG, "libsrq.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm_i8.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm_i8.cu", "noalloc.cu"]
 
 
 def _nvcc() -> str:
