@@ -33,8 +33,9 @@
  *
  * Step size.  The paper leaves the precision level D of Def. 1 free.  Here
  * D_g = absmax_g / qmax with qmax = 2^(bits-1) - 1 and codes in
- * [-qmax, qmax]; x / D is evaluated as x * (qmax / absmax_g), one binary32
- * multiply.  The group g is the whole tensor (SRQ_PER_TENSOR) or one row of
+ * [-qmax, qmax]; x / D is evaluated as x * inv_g, one binary32 multiply,
+ * with inv_g = qmax / absmax_g rounded toward zero, so that the quotient of
+ * every element of the group stays within [-qmax, qmax] as in Def. 1.  The group g is the whole tensor (SRQ_PER_TENSOR) or one row of
  * the code layout being written (SRQ_PER_ROW), i.e. one index of the
  * dimension that is NOT contracted in the product that consumes the codes.
  *

@@ -99,17 +99,28 @@ uint32_t orc_threshold_u24(uint64_t seed, uint64_t tensor_id, uint64_t i)
 static int orc_qmax(int bits) { return (1 << (bits - 1)) - 1; }
 
 /*
- * D = m / qmax and the reciprocal 1/D actually multiplied in, inv = qmax / m,
- * both one binary32 division.  m = 0 is Def. 1's D = 0 case (Q_0 is the
- * identity, and the group is all zeros, so codes 0 with scale 0 reproduce
- * it).  A group whose absmax is so small that qmax / m overflows binary32
- * (m below about 4e-37) is treated the same way.
+ * D = m / qmax (one binary32 division, round to nearest) and the reciprocal
+ * actually multiplied in, inv = qmax / m ROUNDED TOWARD ZERO: the largest
+ * binary32 number not above qmax / m.  Def. 1 has no saturation: with
+ * D = m / qmax every |x / D| of the group is at most qmax.  Rounding the
+ * reciprocal toward zero keeps that property for the computed quotient
+ * (|x| <= m gives |x * inv| <= m * inv <= qmax in real numbers, and rounding
+ * the product to binary32 cannot pass the representable number qmax), so no
+ * code ever leaves [-qmax, qmax].  A reciprocal rounded to nearest would let
+ * the extreme element overshoot qmax by an ulp and force a clamp that the
+ * definition does not have.
+ * m = 0 is Def. 1's D = 0 case (Q_0 is the identity, and the group is all
+ * zeros, so codes 0 with scale 0 reproduce it).  A group whose absmax is so
+ * small that qmax / m overflows binary32 (m below about 4e-37) is treated
+ * the same way.
  */
 void orc_scale_from_absmax(float m, int bits, float *delta, float *inv)
 {
     float qmax = (float)orc_qmax(bits);
     float r = (m == 0.0f) ? 0.0f : qmax / m;
     if (isinf(r) || r != r) r = 0.0f;
+    /* the product of two binary32 numbers is exact in binary64 */
+    if (r != 0.0f && (double)r * (double)m > (double)qmax) r = nextafterf(r, 0.0f);
     *inv = r;
     *delta = (r == 0.0f) ? 0.0f : m / qmax;
 }
@@ -130,8 +141,9 @@ void orc_scale_from_absmax(float m, int bits, float *delta, float *inv)
  * without rounding p: multiplied through by 2^24, eps < t - f becomes
  * u24 + f 2^24 < t 2^24, and every term of that is exact in binary64
  * (t has 24 significant bits, f is an integer of magnitude <= 2^8).
- *   q = f + up, clamped to [-qmax, qmax] (the rounded product t can exceed
- *   qmax by one ulp at the extreme element).
+ *   q = f + up.  With inv from orc_scale_from_absmax and |x| <= absmax the
+ *   result is always inside [-qmax, qmax]; the clamp below only matters for
+ *   callers that pass some other inv.
  */
 int orc_quantize_scalar(float x, float inv, int bits, int round_mode, uint32_t u24)
 {

@@ -4,7 +4,8 @@
 //   amax_kernel      one read of x; max |x| per tensor, per row and/or per column, kept as the
 //                    binary32 bit pattern (non-negative floats order like unsigned integers,
 //                    so atomicMax on the bits is exact and order independent)
-//   scales_kernel    D = m / qmax and 1/D = qmax / m per group (one IEEE division each)
+//   scales_kernel    D = m / qmax (round to nearest) and 1/D = qmax / m rounded toward zero, so
+//                    that no quotient x * (1/D) of the group exceeds qmax and no clamp is needed
 //   quantize_kernel  second read of x; t = x * (1/D) (one binary32 multiply), then Def. 1 on
 //                    real numbers: SR rounds up iff u24 * 2^-24 < frac(t) with u24 from
 //                    Philox4x32-10 keyed by (seed, tensor_id, flat index); RTN rounds up iff
@@ -167,8 +168,10 @@ __device__ __forceinline__ void scale_from_bits(uint32_t bits, float qmax, float
                                                 uint32_t* status) {
     if (bits >= 0x7F800000u) record_status(status, SRQ_ERR_NONFINITE);
     const float m = __uint_as_float(bits);
-    float r = (m == 0.0f) ? 0.0f : __fdiv_rn(qmax, m);
-    if (!(fabsf(r) <= 3.402823466e38f)) r = 0.0f;   // overflowed reciprocal: treat the group as zero
+    // toward zero, so that |x * r| <= qmax for the whole group; a reciprocal that overflows when
+    // rounded to nearest marks a group too small to scale, which is treated as all zeros
+    float r = 0.0f;
+    if (m != 0.0f && fabsf(__fdiv_rn(qmax, m)) <= 3.402823466e38f) r = __fdiv_rz(qmax, m);
     *inv = r;
     *delta = (r == 0.0f) ? 0.0f : __fdiv_rn(m, qmax);
 }
@@ -219,7 +222,7 @@ __device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, const Ph
 // ------------------------------------------------------------------------------------------
 // quantizer
 // ------------------------------------------------------------------------------------------
-// Def. 1 for one element; returns the code as a two's complement integer.
+// Def. 1 for one element.
 // The comparison frac(t) > eps of Def. 1 is taken on real numbers, with no rounding of the
 // fractional part, in fixed point with 24 fractional bits.  Let S = t * 2^24 (exact: a power-of
 // -two scaling of the binary32 product t = x * (1/D)), u = u24 the 24-bit threshold.
@@ -229,28 +232,32 @@ __device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, const Ph
 //        low = 0: the code is f' either way, as Def. 1 gives with frac(t) > 1 - 2^-24 > eps.)
 //   RTN: frac(t) >= 1/2  <=>  floor(S) - floor(t) 2^24 >= 2^23, so the code is
 //        (floor(S) + 2^23) >> 24.
-// Clamping C to +-qmax 2^24 first clamps the code to +-qmax and keeps the sum inside int32.
+// |t| <= qmax for every element of a group (the reciprocal step is rounded toward zero), so
+// |C| <= qmax 2^24, the sum stays inside int32 and the code inside [-qmax, qmax] without a clamp.
+// quantize_sum returns the 32-bit sum whose top byte is the code (two's complement); pack4 takes
+// the top bytes, so the final shift costs nothing.
 template <bool SRM>
-__device__ __forceinline__ int quantize_elem(float x, float inv, int lim, uint32_t word) {
+__device__ __forceinline__ uint32_t quantize_sum(float x, float inv, uint32_t word) {
     const float s = __fmul_rn(__fmul_rn(x, inv), 16777216.0f);
     if constexpr (SRM) {
-        const int c = min(max(__float2int_ru(s), -lim), lim);
-        return (c + (int)(0x00FFFFFFu - (word >> 8))) >> 24;
+        const int c = __float2int_ru(s);
+        uint32_t sum;   // (~word >> 8) + c = (2^24 - 1 - u24) + c in one multiply-add (high half)
+        asm("mad.hi.u32 %0, %1, 16777216, %2;" : "=r"(sum) : "r"(~word), "r"((uint32_t)c));
+        return sum;
     } else {
-        const int c = min(max(__float2int_rd(s), -lim), lim);
-        return (c + 0x00800000) >> 24;
+        return (uint32_t)__float2int_rd(s) + 0x00800000u;
     }
 }
 
-__device__ __forceinline__ uint32_t pack4(int b0, int b1, int b2, int b3) {
-    return __byte_perm(__byte_perm((uint32_t)b0, (uint32_t)b1, 0x0040), __byte_perm((uint32_t)b2, (uint32_t)b3, 0x0040), 0x5410);
+__device__ __forceinline__ uint32_t pack4(uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3) {
+    return __byte_perm(__byte_perm(s0, s1, 0x0073), __byte_perm(s2, s3, 0x0073), 0x5410);
 }
 
 template <bool SRM>
-__device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3, int lim,
+__device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3,
                                               const uint32_t rnd[4]) {
-    return pack4(quantize_elem<SRM>(v[0], i0, lim, rnd[0]), quantize_elem<SRM>(v[1], i1, lim, rnd[1]),
-                 quantize_elem<SRM>(v[2], i2, lim, rnd[2]), quantize_elem<SRM>(v[3], i3, lim, rnd[3]));
+    return pack4(quantize_sum<SRM>(v[0], i0, rnd[0]), quantize_sum<SRM>(v[1], i1, rnd[1]),
+                 quantize_sum<SRM>(v[2], i2, rnd[2]), quantize_sum<SRM>(v[3], i3, rnd[3]));
 }
 
 // 4x4 byte transpose: w[i] holds columns c..c+3 of row i -> o[e] holds rows 0..3 of column c+e
@@ -268,7 +275,6 @@ struct QuantParams {
     int64_t rows, cols, ld;
     uint64_t index_offset;
     PhiloxKeys keys;
-    int lim;                      // qmax * 2^24: clamp of the fixed-point quotient
     int sr;                       // 1 = SR, 0 = RTN
     int per_row;                  // step size per row of each layout
     int8_t* codes_rm; int64_t ld_rm;
@@ -314,20 +320,17 @@ __device__ __forceinline__ void widen(const uint2& q, float v[4]) {
 // 4-element group is one vector load, one Philox block and one 4-byte store.  LAYOUT bit 0 = row-major
 // codes wanted, bit 1 = transposed codes wanted.  The loads of the next row quad are issued before the
 // current one is processed, which keeps two quads of loads in flight per thread.
-template <typename T, bool SRM, int LAYOUT, bool PER_ROW>
-__global__ void __launch_bounds__(Q_THREADS)
-quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P) {
+// FULL: the 128 x 128 tile lies inside the matrix and its Philox block indices do not carry into the
+// upper counter word, so rows need no bounds checks and the counter is one 32-bit multiply-add.
+template <typename T, bool SRM, int LAYOUT, bool PER_ROW, bool FULL>
+__device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const QuantParams& P, uint32_t* tileT,
+                                              int64_t r0, int64_t c0) {
     using Raw = typename Raw4<T>::type;
     constexpr bool WANT_RM = (LAYOUT & 1) != 0, WANT_TR = (LAYOUT & 2) != 0;
     constexpr bool TWO_STEPS = WANT_TR && PER_ROW;     // transposed layout has its own step sizes
-    __shared__ uint32_t tileT[WANT_TR ? Q_TILE * (Q_TILE / 4) : 1];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t n_tc = (P.cols + Q_TILE - 1) / Q_TILE;
-    const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * Q_TILE;
-    const int64_t r0 = ((int64_t)blockIdx.x / n_tc) * Q_TILE;
     const int64_t c = c0 + lane * 4;
-    const bool col_ok = c < P.cols;                     // cols % 4 == 0: a group is all in or all out
-    const int lim = P.lim;
+    const bool col_ok = FULL || c < P.cols;             // cols % 4 == 0: a group is all in or all out
 
     float ic[4] = {0.f, 0.f, 0.f, 0.f};
     if constexpr (TWO_STEPS) {
@@ -335,21 +338,25 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
     }
     const float inv_tensor = PER_ROW ? 0.0f : P.inv_rm[0];
 
-    const T* xp = x + (r0 + warp * 4) * P.ld + c;       // first row of this thread's first quad
-    const int64_t quad_stride = 32 * P.ld;              // 8 warps x 4 rows between successive quads
-    // Philox block index of (row, c): (index_offset + row * cols + c) / 4, advanced by cols / 4 per row
-    uint64_t j = (P.index_offset + (uint64_t)(r0 + warp * 4) * (uint64_t)P.cols + (uint64_t)c) >> 2;
-    const uint64_t j_row = (uint64_t)P.cols >> 2, j_quad = 32 * j_row;
+    // element (tr, lane * 4) of the tile, tr = (warp + 8 * it) * 4 + i: 32-bit offsets from the tile corner
+    const T* xt = x + r0 * P.ld + c;
+    const uint32_t ld = (uint32_t)P.ld;
+    int8_t* out_rm = WANT_RM ? P.codes_rm + r0 * P.ld_rm + c : nullptr;
+    const uint32_t ld_rm = (uint32_t)P.ld_rm;
+    // Philox block index of (row, c): (index_offset + row * cols + c) / 4 = jb + tr * j_row
+    const uint64_t jb = (P.index_offset + (uint64_t)r0 * (uint64_t)P.cols + (uint64_t)c) >> 2;
+    const uint32_t j_row = (uint32_t)((uint64_t)P.cols >> 2);
+    const uint32_t jb_lo = (uint32_t)jb, jb_hi = (uint32_t)(jb >> 32);
 
     Raw cur[4], nxt[4];
     float inv_cur[4], inv_nxt[4];
     auto load_quad = [&](int it, Raw raw[4], float inv_r[4]) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const int64_t r = r0 + (warp + 8 * it) * 4 + i;
-            if (col_ok && r < P.rows) {
-                raw[i] = __ldcs(reinterpret_cast<const Raw*>(xp + (int64_t)it * quad_stride + i * P.ld));
-                if constexpr (PER_ROW && WANT_RM) inv_r[i] = P.inv_rm[r];
+            const uint32_t tr = (uint32_t)(warp + 8 * it) * 4 + i;
+            if (FULL || (col_ok && r0 + tr < P.rows)) {
+                raw[i] = __ldcs(reinterpret_cast<const Raw*>(xt + tr * ld));
+                if constexpr (PER_ROW && WANT_RM) inv_r[i] = P.inv_rm[r0 + tr];
             } else {
                 raw[i] = Raw{};
                 if constexpr (PER_ROW && WANT_RM) inv_r[i] = 0.0f;
@@ -365,22 +372,26 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
         uint32_t wr[4], wt[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
+            const uint32_t tr = (uint32_t)rq * 4 + i;
             float v[4];
             widen(cur[i], v);
             uint32_t rnd[4] = {0u, 0u, 0u, 0u};
             if constexpr (SRM) {
-                const uint64_t jj = j + (uint64_t)i * j_row;
-                philox_rounds((uint32_t)jj, (uint32_t)(jj >> 32), P.keys, rnd);
+                if constexpr (FULL) {
+                    philox_rounds(jb_lo + tr * j_row, jb_hi, P.keys, rnd);
+                } else {
+                    const uint64_t jj = jb + (uint64_t)tr * j_row;
+                    philox_rounds((uint32_t)jj, (uint32_t)(jj >> 32), P.keys, rnd);
+                }
             }
             if constexpr (WANT_RM || !TWO_STEPS) {
                 const float ir = (PER_ROW && WANT_RM) ? inv_cur[i] : inv_tensor;
-                wr[i] = quantize4<SRM>(v, ir, ir, ir, ir, lim, rnd);
+                wr[i] = quantize4<SRM>(v, ir, ir, ir, ir, rnd);
             }
-            if constexpr (TWO_STEPS) wt[i] = quantize4<SRM>(v, ic[0], ic[1], ic[2], ic[3], lim, rnd);
+            if constexpr (TWO_STEPS) wt[i] = quantize4<SRM>(v, ic[0], ic[1], ic[2], ic[3], rnd);
             else wt[i] = wr[i];
             if constexpr (WANT_RM) {
-                const int64_t r = r0 + rq * 4 + i;
-                if (col_ok && r < P.rows) *reinterpret_cast<uint32_t*>(P.codes_rm + r * P.ld_rm + c) = wr[i];
+                if (FULL || (col_ok && r0 + tr < P.rows)) *reinterpret_cast<uint32_t*>(out_rm + tr * ld_rm) = wr[i];
             }
         }
         if constexpr (WANT_TR) {
@@ -389,7 +400,6 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
 #pragma unroll
             for (int e = 0; e < 4; ++e) tileT[(lane * 4 + e) * 32 + (rq ^ lane)] = o[e];
         }
-        j += j_quad;
 #pragma unroll
         for (int i = 0; i < 4; ++i) { cur[i] = nxt[i]; inv_cur[i] = inv_nxt[i]; }
     }
@@ -397,6 +407,21 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
         __syncthreads();
         store_transposed_tile(tileT, P, r0, c0, warp, lane);
     }
+}
+
+template <typename T, bool SRM, int LAYOUT, bool PER_ROW>
+__global__ void __launch_bounds__(Q_THREADS)
+quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P) {
+    __shared__ uint32_t tileT[(LAYOUT & 2) ? Q_TILE * (Q_TILE / 4) : 1];
+    const int64_t n_tc = (P.cols + Q_TILE - 1) / Q_TILE;
+    const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * Q_TILE;
+    const int64_t r0 = ((int64_t)blockIdx.x / n_tc) * Q_TILE;
+    // last Philox block index of the tile, relative to its first: no carry if it fits in the low word
+    const uint64_t j_first = (P.index_offset + (uint64_t)r0 * (uint64_t)P.cols + (uint64_t)c0) >> 2;
+    const uint64_t j_span = (uint64_t)(Q_TILE - 1) * ((uint64_t)P.cols >> 2) + (Q_TILE / 4 - 1);
+    const bool full = r0 + Q_TILE <= P.rows && c0 + Q_TILE <= P.cols && (j_first & 0xFFFFFFFFull) + j_span <= 0xFFFFFFFFull;
+    if (full) quantize_tile<T, SRM, LAYOUT, PER_ROW, true>(x, P, tileT, r0, c0);
+    else quantize_tile<T, SRM, LAYOUT, PER_ROW, false>(x, P, tileT, r0, c0);
 }
 
 // General path: any extent, pitch, alignment and index offset; one Philox block per element
@@ -449,11 +474,11 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
                 }
                 const float inv_r = P.per_row ? P.inv_rm[want_rm ? r : 0] : inv_tensor;
                 if (want_rm || !two_steps)
-                    wr[i] = sr ? quantize4<true>(v, inv_r, inv_r, inv_r, inv_r, P.lim, rnd)
-                               : quantize4<false>(v, inv_r, inv_r, inv_r, inv_r, P.lim, rnd);
+                    wr[i] = sr ? quantize4<true>(v, inv_r, inv_r, inv_r, inv_r, rnd)
+                               : quantize4<false>(v, inv_r, inv_r, inv_r, inv_r, rnd);
                 if (two_steps)
-                    wt[i] = sr ? quantize4<true>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], P.lim, rnd)
-                               : quantize4<false>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], P.lim, rnd);
+                    wt[i] = sr ? quantize4<true>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], rnd)
+                               : quantize4<false>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], rnd);
                 else
                     wt[i] = wr[i];
                 if (want_rm) {
@@ -552,7 +577,6 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
             P.keys.k1[r] = (uint32_t)(a.q.seed >> 32) + (uint32_t)r * 0xBB67AE85u;
         }
         P.keys.tid0 = (uint32_t)a.q.tensor_id; P.keys.tid1 = (uint32_t)(a.q.tensor_id >> 32);
-        P.lim = ((1 << (a.q.bits - 1)) - 1) << 24;
         P.sr = a.q.round == SRQ_SR;
         P.per_row = per_row;
         P.codes_rm = a.codes_rm; P.ld_rm = a.ld_rm;
@@ -561,7 +585,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         P.vec_in = vec_in;
         P.vec_rm = want_rm && ((uintptr_t)a.codes_rm % 4 == 0) && (a.ld_rm % 4 == 0);
         P.vec_tr = want_tr && ((uintptr_t)a.codes_tr % 4 == 0) && (a.ld_tr % 4 == 0);
-        const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && (!want_rm || P.vec_rm) &&
+        const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) &&
                           (!want_tr || (P.vec_tr && rows % 4 == 0));
         const unsigned grid = (unsigned)(((cols + Q_TILE - 1) / Q_TILE) * ((rows + Q_TILE - 1) / Q_TILE));
         if (fast) launch_fast(a.dt, P.sr != 0, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);

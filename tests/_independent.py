@@ -48,7 +48,8 @@ def qmax_of(bits):
 
 
 def scale_ref(m, bits):
-    """(Delta, 1/Delta) by the absmax rule, one binary32 division each."""
+    """(Delta, 1/Delta) by the absmax rule: Delta one binary32 division rounded to nearest, the
+    reciprocal the largest binary32 number not above qmax / m (found with exact rationals)."""
     m = np.float32(m)
     q = np.float32(qmax_of(bits))
     if m == 0:
@@ -57,6 +58,11 @@ def scale_ref(m, bits):
         inv = q / m
     if not np.isfinite(inv):
         return np.float32(0), np.float32(0)
+    exact = Fraction(int(q)) / Fraction(float(m))
+    while Fraction(float(inv)) > exact:
+        inv = np.nextafter(inv, np.float32(0))
+    while Fraction(float(np.nextafter(inv, np.float32(np.inf)))) <= exact:
+        inv = np.nextafter(inv, np.float32(np.inf))
     return np.float32(m / q), np.float32(inv)
 
 

@@ -230,10 +230,17 @@ def test_absmax_matches_numpy_and_handles_pitch():
 
 
 def test_scale_rule_and_zero_group():
+    from fractions import Fraction
+    rng = np.random.default_rng(9)
     for bits in (8, 6, 4, 3, 2):
         q = qmax_of(bits)
-        d, inv = oracle.scale_from_absmax(3.0, bits)
-        assert d == np.float32(3.0) / np.float32(q) and inv == np.float32(q) / np.float32(3.0)
+        for m in [3.0, 1.0, 127.0] + list(rng.uniform(1e-3, 50, 300).astype(np.float32)):
+            d, inv = oracle.scale_from_absmax(float(m), bits)
+            assert d == np.float32(m) / np.float32(q)
+            # inv is the largest binary32 number <= qmax / m (round toward zero)
+            exact = Fraction(q) / Fraction(float(np.float32(m)))
+            assert Fraction(float(inv)) <= exact < Fraction(float(np.nextafter(inv, np.float32(np.inf))))
+            assert (d, inv) == scale_ref(m, bits)
     # Delta = 0: Q_0 is the identity (note in Def. 1); only an all-zero group reaches it
     d, inv = oracle.scale_from_absmax(0.0, 8)
     assert d == 0 and inv == 0
@@ -249,21 +256,24 @@ def test_scale_rule_and_zero_group():
     assert s[0] == 0 and not c[0].any() and c[1, 1] == -127
 
 
-def test_extreme_element_is_clamped_to_qmax():
-    # for some absmax values fl(m * fl(qmax/m)) exceeds qmax by an ulp; the code must stay qmax
+def test_quotient_of_the_extreme_element_never_passes_qmax():
+    # Def. 1 has no saturation: |x / D| <= qmax for the whole group.  With the reciprocal rounded
+    # toward zero the binary32 quotient of the absmax element itself stays <= qmax, so every code
+    # is inside [-qmax, qmax] before any clamp; the extreme element lands on qmax or qmax - 1.
     rng = np.random.default_rng(10)
     ms = rng.uniform(0.1, 10, 2000).astype(np.float32)
-    seen_excess = False
-    for m in ms:
-        d, inv = oracle.scale_from_absmax(float(m), 8)
-        excess = bool(np.float32(m) * inv > 127)
-        seen_excess |= excess
-        for u in (0, 1, 2 ** 23, 2 ** 24 - 1):
-            hi = oracle.quantize_scalar(float(m), float(inv), 8, SR, u)
-            lo = oracle.quantize_scalar(-float(m), float(inv), 8, SR, u)
-            assert -127 <= lo <= -126 and 126 <= hi <= 127
-            if excess:
-                assert hi == 127 and lo == -127
-        assert oracle.quantize_scalar(float(m), float(inv), 8, RTN) == 127
-        assert oracle.quantize_scalar(-float(m), float(inv), 8, RTN) == -127
-    assert seen_excess
+    below = False
+    for bits in (8, 4):
+        q = qmax_of(bits)
+        for m in ms:
+            d, inv = oracle.scale_from_absmax(float(m), bits)
+            t = np.float32(m) * inv
+            assert t <= q
+            below |= bool(t < q)
+            for u in (0, 1, 2 ** 23, 2 ** 24 - 1):
+                hi = oracle.quantize_scalar(float(m), float(inv), bits, SR, u)
+                lo = oracle.quantize_scalar(-float(m), float(inv), bits, SR, u)
+                assert -q <= lo <= -q + 1 and q - 1 <= hi <= q
+            assert oracle.quantize_scalar(float(m), float(inv), bits, RTN) == q
+            assert oracle.quantize_scalar(-float(m), float(inv), bits, RTN) == -q
+    assert below
