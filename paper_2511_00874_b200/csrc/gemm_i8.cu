@@ -5,12 +5,20 @@
 //   acc[i,j] = sum_k a[i,k] * b[j,k]          int8 x int8 -> int32, exact
 //   out[i,j] = float(acc[i,j]) * (s_row[i] * s_col[j])
 //
-// One persistent CTA per SM, 6 warps:
-//   warp 0      TMA producer: 128 x 128-byte tiles of a and 256 x 128-byte tiles of b into a
-//               4-stage shared-memory ring (128-byte swizzle), signalled through mbarriers
-//   warp 1      allocates TMEM and issues tcgen05.mma.kind::i8 (M128 x N256 x K32) from one
-//               thread; accumulators live in TMEM, two buffers of 256 columns, so the tensor
-//               pipe starts the next tile while the previous one is being drained
+// Persistent kernel, one CTA per SM, 6 warps.  Two forms of the same code (template CTAS):
+//   CTAS = 2  two CTAs on neighbouring SMs (a cluster) share one 256 x 256 output tile: each stages
+//             its own 128 rows of a and 128 of the 256 rows of b, and the leader CTA issues
+//             tcgen05.mma.cta_group::2 (M256 x N256 x K32), which reads both CTAs' shared memory
+//             and writes 128 accumulator rows into each CTA's TMEM.  Per SM this halves the b
+//             traffic and the shared-memory reads per MMA; used whenever M > 128.
+//   CTAS = 1  one CTA per 128 x 256 tile with tcgen05.mma.cta_group::1 (M128 x N256 x K32).
+// Roles:
+//   warp 0      TMA producer: 128-byte-swizzled tiles of a and b into a shared-memory ring
+//               (6 stages of 32 KB, or 4 of 48 KB), signalled through mbarriers; with CTAS = 2
+//               both CTAs' loads complete on the leader's barrier (no multicast is used)
+//   warp 1      allocates TMEM; in the leader one thread issues the MMAs; accumulators live in
+//               TMEM, two buffers of 256 columns, so the tensor pipe starts the next tile while
+//               the previous one is being drained
 //   warps 2-5   epilogue: tcgen05.ld the accumulator (one TMEM lane quarter per warp), convert,
 //               scale and store; or, for a split contraction, add the exact int32 partial
 //               sums into a workspace, the CTA that finishes a tile last doing the scaling
@@ -25,15 +33,22 @@
 
 namespace srq {
 
-constexpr int BM = 128, BN = 256, BK = 128;          // tile extents; BK in bytes = int8 elements
-constexpr int STAGES = 4;
+constexpr int BM = 128, BN = 256, BK = 128;          // per-CTA rows, tile columns, k-block (bytes = int8 elements)
 constexpr int UMMA_K = 32;                             // bytes of K per tcgen05.mma.kind::i8
-constexpr int A_STAGE_BYTES = BM * BK, B_STAGE_BYTES = BN * BK;
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int A_STAGE_BYTES = BM * BK;
 constexpr int TMEM_COLS = 512;                         // two accumulator buffers of BN columns
 constexpr int GEMM_THREADS = 192;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;      // 2 s
 
+template <int CTAS>
+struct Cfg {
+    static constexpr int B_ROWS = BN / CTAS;                         // rows of b staged by each CTA
+    static constexpr int B_STAGE_BYTES = B_ROWS * BK;
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    static constexpr int STAGES = CTAS == 1 ? 4 : 6;
+};
+
+template <int STAGES>
 struct SharedTail {                                    // after the stage ring
     uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain;
     uint32_t tmem_base;
@@ -42,7 +57,10 @@ struct SharedTail {                                    // after the stage ring
     uint32_t epi_abort;
     alignas(16) float s_col[2][BN];   // read as float4
 };
-constexpr size_t GEMM_SMEM = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + sizeof(SharedTail);
+template <int CTAS>
+constexpr size_t gemm_smem() {
+    return 1024 /*alignment slack*/ + (size_t)Cfg<CTAS>::STAGES * Cfg<CTAS>::STAGE_BYTES + sizeof(SharedTail<Cfg<CTAS>::STAGES>);
+}
 
 // ------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -85,33 +103,92 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int32_t x, int32_t y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+// Cluster helpers (CTAS = 2): rank of this CTA in its pair, the pair-wide barrier, and the address
+// of a shared-memory object of the pair's CTA `rank` in the shared::cluster window.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+// Tile load into this CTA's shared memory.  CTAS = 2: the completion bytes are counted on the
+// barrier at `bar_addr`, which may belong to the other CTA of the pair (no multicast).
+template <int CTAS>
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar_addr) {
+    if constexpr (CTAS == 1) {
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+            ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_addr) : "memory");
+    } else {
+        asm volatile(
+            "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+            ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_addr) : "memory");
+    }
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// One warp per CTA; with CTAS = 2 the same warp of both CTAs of the pair, same shared-memory offset.
+template <int CTAS>
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (CTAS == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
 }
+template <int CTAS>
 __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+    if constexpr (CTAS == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem], int8 operands, int32 accumulators, issued by one thread.
+// D[tmem] (+)= A[smem] * B[smem], int8 operands, int32 accumulators, issued by one thread (of the
+// leader CTA when CTAS = 2; the descriptors then address the same offsets in both CTAs).
+template <int CTAS>
 __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    if constexpr (CTAS == 1) {
+        asm volatile(
+            "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    } else {
+        asm volatile(
+            "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    }
 }
 // The mbarrier gets one arrival once every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+// CTAS = 2, both = true: the barrier at the same offset in both CTAs of the pair gets it.
+template <int CTAS>
+__device__ __forceinline__ void umma_commit(uint64_t* bar, bool both) {
+    if constexpr (CTAS == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    } else {
+        if (both) {
+            const uint16_t mask = 3;
+            asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                         ::"r"(smem_u32(bar)), "h"(mask) : "memory");
+        } else {
+            asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+        }
+    }
 }
 
 // 32 lanes x 32 consecutive 32-bit columns: thread t of the warp receives lane (base + t).
@@ -153,42 +230,52 @@ struct GemmParams {
     int64_t M, N;
     int32_t num_kb;            // 128-byte blocks along the contraction
     int32_t splits;            // parts the contraction is cut into (1 = none)
-    int32_t tiles_m, tiles_n;
+    int32_t tiles_m, tiles_n;  // tiles of (128 * CTAS) x 256
     const float* s_row; int32_t row_stride;
     const float* s_col; int32_t col_stride;
     float* out; int64_t ldo;
     int32_t* acc_out;          // optional raw sums [M, N]
     int32_t* part;             // split contraction: zeroed int32 [M, N]
-    uint32_t* tickets;         // split contraction: zeroed, one per output tile
+    uint32_t* tickets;         // split contraction: zeroed, one per 128-row half of an output tile
     uint32_t* status;
     int32_t vec_out;           // 16-byte stores to out allowed
 };
 
-__device__ __forceinline__ void give_up(SharedTail* T, uint32_t* status) {
+template <int STAGES>
+__device__ __forceinline__ void give_up(SharedTail<STAGES>* T, uint32_t* status) {
     T->abort_flag = 1u;
     record_status(status, SRQ_ERR_TIMEOUT);
 }
 
+template <int CTAS>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams P) {
+    using C = Cfg<CTAS>;
+    constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES;
+    using Tail = SharedTail<STAGES>;
     extern __shared__ uint8_t smem_raw[];
+    // the dynamic window starts at the same offset in every CTA, so the aligned layouts coincide
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    SharedTail* T = (SharedTail*)(smem + (size_t)STAGES * STAGE_BYTES);
+    Tail* T = (Tail*)(smem + (size_t)STAGES * STAGE_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = CTAS == 1 ? 0u : cluster_ctarank();   // position in the CTA pair
+    const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&T->full[s], 1); mbar_init(&T->empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&T->tmem_full[b], 1); mbar_init(&T->tmem_empty[b], 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&T->tmem_full[b], 1); mbar_init(&T->tmem_empty[b], 4 * CTAS); }
         mbar_init(&T->drain, 1);
         T->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(&T->tmem_base, TMEM_COLS);
+    __syncwarp();
+    if (warp == 1) tmem_alloc<CTAS>(&T->tmem_base, TMEM_COLS);
     tc_fence_before();
-    __syncthreads();
+    if constexpr (CTAS == 1) __syncthreads(); else cluster_sync();   // the peer's barriers exist from here on
     tc_fence_after();
     const uint32_t tmem_base = T->tmem_base;
 
+    const int64_t groups = gridDim.x / CTAS, group = blockIdx.x / CTAS;   // a group = the CTAs of one tile
     const int64_t units = (int64_t)P.tiles_m * P.tiles_n * P.splits;
     const int32_t kb_per_split = (P.num_kb + P.splits - 1) / P.splits;
 
@@ -199,38 +286,47 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t u = blockIdx.x; u < units && ok; u += gridDim.x) {
+            for (int64_t u = group; u < units && ok; u += groups) {
                 const int32_t split = (int32_t)(u % P.splits);
                 const int64_t tile = u / P.splits;
                 const int32_t tn = (int32_t)(tile % P.tiles_n), tm = (int32_t)(tile / P.tiles_n);
                 const int32_t kb0 = split * kb_per_split;
                 const int32_t kb1 = min(kb0 + kb_per_split, P.num_kb);
+                const int32_t row_a = (tm * CTAS + (int32_t)rank) * BM;
+                const int32_t row_b = tn * BN + (int32_t)rank * C::B_ROWS;
                 for (int32_t kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!mbar_wait(&T->empty[s], ph ^ 1u, &T->abort_flag)) { give_up(T, P.status); ok = false; break; }
-                    mbar_expect_tx(&T->full[s], STAGE_BYTES);
+                    // the bytes of every CTA of the group are counted on the leader's barrier
+                    if (leader) mbar_expect_tx(&T->full[s], STAGE_BYTES * CTAS);
+                    const uint32_t bar = CTAS == 1 ? smem_u32(&T->full[s]) : map_to_cta(smem_u32(&T->full[s]), 0);
                     uint8_t* sa = smem + (size_t)s * STAGE_BYTES;
-                    tma_load_2d(sa, &map_a, kb * BK, tm * BM, &T->full[s]);
-                    tma_load_2d(sa + A_STAGE_BYTES, &map_b, kb * BK, tn * BN, &T->full[s]);
+                    tma_load_2d<CTAS>(sa, &map_a, kb * BK, row_a, bar);
+                    tma_load_2d<CTAS>(sa + A_STAGE_BYTES, &map_b, kb * BK, row_b, bar);
                 }
             }
             if (!ok) {
                 // loads already issued must land before the CTA may leave
-                const uint32_t back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
-                for (uint32_t j = 1; j <= back; ++j) {
-                    const uint32_t jt = it - j;
-                    const uint64_t t0 = global_ns();
-                    while (!mbar_try_wait(&T->full[jt % STAGES], (jt / STAGES) & 1u) && global_ns() - t0 < WAIT_LIMIT_NS) {}
+                if (leader) {
+                    const uint32_t back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+                    for (uint32_t j = 1; j <= back; ++j) {
+                        const uint32_t jt = it - j;
+                        const uint64_t t0 = global_ns();
+                        while (!mbar_try_wait(&T->full[jt % STAGES], (jt / STAGES) & 1u) && global_ns() - t0 < WAIT_LIMIT_NS) {}
+                    }
+                } else {
+                    const uint64_t t0 = global_ns();          // their barrier is not ours to wait on: give them time
+                    while (global_ns() - t0 < 1000000ull) {}
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_i8(BM, BN);
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
+            const uint32_t idesc = make_idesc_i8(BM * CTAS, BN);
             uint32_t it = 0, lt = 0;
             bool ok = true;
-            for (int64_t u = blockIdx.x; u < units && ok; u += gridDim.x, ++lt) {
+            for (int64_t u = group; u < units && ok; u += groups, ++lt) {
                 const int32_t split = (int32_t)(u % P.splits);
                 const int32_t kb0 = split * kb_per_split;
                 const int32_t kb1 = min(kb0 + kb_per_split, P.num_kb);
@@ -247,15 +343,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         // advancing K inside the swizzle atom = advancing the start address
-                        umma_i8(d_tmem, da + (uint64_t)((k * UMMA_K) >> 4), db + (uint64_t)((k * UMMA_K) >> 4), idesc,
-                                (kb > kb0 || k > 0) ? 1u : 0u);
+                        umma_i8<CTAS>(d_tmem, da + (uint64_t)((k * UMMA_K) >> 4), db + (uint64_t)((k * UMMA_K) >> 4), idesc,
+                                      (kb > kb0 || k > 0) ? 1u : 0u);
                     }
-                    umma_commit(&T->empty[s]);       // stage reusable once these MMAs have read it
+                    umma_commit<CTAS>(&T->empty[s], true);       // stage reusable (in every CTA) once these MMAs have read it
                 }
-                if (ok) umma_commit(&T->tmem_full[buf]);   // accumulator complete
+                if (ok) umma_commit<CTAS>(&T->tmem_full[buf], true);   // accumulator complete
             }
             if (!ok) {
-                umma_commit(&T->drain);
+                umma_commit<CTAS>(&T->drain, false);
                 const uint64_t t0 = global_ns();
                 while (!mbar_try_wait(&T->drain, 0u) && global_ns() - t0 < WAIT_LIMIT_NS) {}
             }
@@ -264,13 +360,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;                    // TMEM lanes this warp may read
         const int etid = threadIdx.x - 64;               // 0..127 within the epilogue group
+        // the MMA issuer's barriers (in the leader CTA)
+        const uint32_t empty_bar0 = CTAS == 1 ? smem_u32(&T->tmem_empty[0]) : map_to_cta(smem_u32(&T->tmem_empty[0]), 0);
+        const uint32_t empty_bar1 = CTAS == 1 ? smem_u32(&T->tmem_empty[1]) : map_to_cta(smem_u32(&T->tmem_empty[1]), 0);
         uint32_t lt = 0;
         bool ok = true;
-        for (int64_t u = blockIdx.x; u < units && ok; u += gridDim.x, ++lt) {
+        for (int64_t u = group; u < units && ok; u += groups, ++lt) {
             const int64_t tile = u / P.splits;
             const int32_t tn = (int32_t)(tile % P.tiles_n), tm = (int32_t)(tile / P.tiles_n);
             const uint32_t buf = lt & 1u, use = lt >> 1;
-            const int64_t row = (int64_t)tm * BM + quarter * 32 + lane;
+            const int64_t row0 = ((int64_t)tm * CTAS + rank) * BM;      // first row of this CTA's half
+            const int64_t row = row0 + quarter * 32 + lane;
             const int64_t col_base = (int64_t)tn * BN;
             // stage this tile's column step sizes (other buffer may still be read by slower warps)
             for (int i = etid; i < BN; i += 128) {
@@ -322,7 +422,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&T->tmem_empty[buf]);
+                if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             } else {
                 // exact partial sums: integer adds commute, so any arrival order gives the same total
 #pragma unroll 1
@@ -340,20 +440,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&T->tmem_empty[buf]);
+                if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (etid == 0) {
-                    const uint32_t t = atomicAdd(&P.tickets[tile], 1u);
+                    const uint32_t t = atomicAdd(&P.tickets[tile * CTAS + rank], 1u);
                     T->last_flag[buf] = (t == (uint32_t)P.splits - 1u) ? 1u : 0u;
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (T->last_flag[buf]) {
                     __threadfence();
-                    // the last contributor scales the finished tile: warp w takes rows w, w+4, ...
+                    // the last contributor scales the finished half tile: warp w takes rows w, w+4, ...
                     const int ew = warp - 2;
                     for (int r = ew; r < BM; r += 4) {
-                        const int64_t grow = (int64_t)tm * BM + r;
+                        const int64_t grow = row0 + r;
                         if (grow >= P.M) break;
                         const float srr = P.s_row[grow * P.row_stride];
                         for (int cidx = lane; cidx < BN; cidx += 32) {
@@ -370,12 +470,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     }
 
+    // nobody leaves while the other CTA of the pair may still address this one's barriers, shared
+    // memory or TMEM
+    __syncwarp();
     tc_fence_before();
-    __syncthreads();
+    if constexpr (CTAS == 1) __syncthreads(); else cluster_sync();
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        tmem_dealloc<CTAS>(tmem_base, TMEM_COLS);
     }
 }
 
@@ -411,21 +514,43 @@ static bool encode_operand(CUtensorMap* map, const int8_t* base, int64_t rows, i
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 1;
+// Per device: SM count, the number of CTA pairs that can be resident at once, and the one-time
+// opt-in to the large dynamic shared-memory carve-out.
+struct DeviceInfo { bool ready = false; int sms = 1; int pairs = 0; };
+
+static bool device_info(DeviceInfo** out) {
+    static DeviceInfo info[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    DeviceInfo& d = info[dev];
+    if (!d.ready) {
+        if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || d.sms <= 0) return false;
+        if (cudaFuncSetAttribute(gemm_i8_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<1>()) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_i8_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<2>()) != cudaSuccess) return false;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(d.sms / 2 * 2)); cfg.blockDim = dim3(GEMM_THREADS); cfg.dynamicSmemBytes = gemm_smem<2>();
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+        cfg.attrs = &at; cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<2>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+        d.pairs = n < d.sms / 2 ? n : d.sms / 2;
+        d.ready = true;
     }
-    return n;
+    *out = &d;
+    return true;
 }
 
-static int choose_splits(int64_t tiles, int32_t num_kb) {
-    const int sms = sm_count();
-    if (tiles * 2 > sms || num_kb < 16) return 1;          // enough tiles to fill the machine
-    int s = (int)(sms / tiles);
+// Parts the contraction is cut into when there are too few tiles to fill the machine (`groups`
+// tiles run at a time).
+static int choose_splits(int64_t tiles, int32_t num_kb, int groups) {
+    if (num_kb < 16) return 1;
+    int s = 1;
+    if (tiles * 2 <= groups) {
+        s = (int)(groups / tiles);
+    }
     const int max_by_k = num_kb / 8;                        // keep at least 8 k-blocks per part
     if (s > max_by_k) s = max_by_k;
     if (s < 1) s = 1;
@@ -433,39 +558,47 @@ static int choose_splits(int64_t tiles, int32_t num_kb) {
     return (num_kb + per - 1) / per;
 }
 
+// Upper bound of what launch_gemm_i8 may use: int32 partial sums plus tickets, for outputs small
+// enough to be split.
 size_t gemm_splitk_bytes(int64_t M, int64_t N) {
-    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-    if (tiles * 2 > 160) return 0;   // never split (bound is generous with respect to the SM count)
+    const int64_t tiles = 2 * ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);      // 128-row halves of whole pairs
+    if (tiles > 16 * 160) return 0;   // never split (bound is generous with respect to the SM count)
     return align_up((size_t)M * N * 4) + align_up((size_t)tiles * 4);
+}
+
+template <int CTAS>
+static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& P,
+                                 cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(groups * CTAS); cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = gemm_smem<CTAS>(); cfg.stream = stream;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = CTAS; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+    cfg.attrs = &at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_i8_kernel<CTAS>, map_a, map_b, P);
 }
 
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream) {
     if (g.M == 0 || g.N == 0) return SRQ_OK;
-    {   // opt in to the large dynamic shared-memory carve-out once per device
-        static bool done[64] = {};
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return SRQ_ERR_CUDA;
-        if (dev < 0 || dev >= 64 || !done[dev]) {
-            if (cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM) != cudaSuccess)
-                return SRQ_ERR_CUDA;
-            if (dev >= 0 && dev < 64) done[dev] = true;
-        }
-    }
+    DeviceInfo* dev = nullptr;
+    if (!device_info(&dev)) return SRQ_ERR_CUDA;
+    const int ctas = (g.M > BM && dev->pairs > 0) ? 2 : 1;
+    const int groups_max = ctas == 2 ? dev->pairs : dev->sms;
 
     CUtensorMap map_a, map_b;
     if (!encode_operand(&map_a, g.a, g.M, g.Kc, g.lda, BM)) return SRQ_ERR_CUDA;
-    if (!encode_operand(&map_b, g.b, g.N, g.Kc, g.ldb, BN)) return SRQ_ERR_CUDA;
+    if (!encode_operand(&map_b, g.b, g.N, g.Kc, g.ldb, BN / ctas)) return SRQ_ERR_CUDA;
 
     GemmParams P;
     P.M = g.M; P.N = g.N;
     P.num_kb = (int32_t)((g.Kc + BK - 1) / BK);
-    P.tiles_m = (int32_t)((g.M + BM - 1) / BM);
+    P.tiles_m = (int32_t)((g.M + BM * ctas - 1) / (BM * ctas));
     P.tiles_n = (int32_t)((g.N + BN - 1) / BN);
     const int64_t tiles = (int64_t)P.tiles_m * P.tiles_n;
-    P.splits = choose_splits(tiles, P.num_kb);
+    P.splits = choose_splits(tiles, P.num_kb, groups_max);
     P.part = nullptr; P.tickets = nullptr;
     if (P.splits > 1) {
-        const size_t part_bytes = align_up((size_t)g.M * g.N * 4), ticket_bytes = align_up((size_t)tiles * 4);
+        const size_t part_bytes = align_up((size_t)g.M * g.N * 4), ticket_bytes = align_up((size_t)tiles * ctas * 4);
         if (g.splitk_ws == nullptr || g.splitk_ws_bytes < part_bytes + ticket_bytes) {
             P.splits = 1;   // no room: run unsplit (same result)
         } else {
@@ -481,10 +614,11 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.vec_out = ((uintptr_t)g.out % 16 == 0) && (g.ldo % 4 == 0);
 
     const int64_t units = tiles * P.splits;
-    const unsigned grid = (unsigned)(units < sm_count() ? units : sm_count());
-    gemm_i8_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(map_a, map_b, P);
+    const unsigned groups = (unsigned)(units < groups_max ? units : groups_max);
+    const cudaError_t e = ctas == 2 ? launch_kernel<2>(groups, map_a, map_b, P, stream)
+                                    : launch_kernel<1>(groups, map_a, map_b, P, stream);
     ++g_launches;
-    return cudaGetLastError() == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+    return e == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
 }
 
 }  // namespace srq
