@@ -3,9 +3,9 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-One step = one pass of the whole hot path over one batch: qlinear_fwd, qlinear_bwd_input and
-qlinear_bwd_weight (five absmax reductions and quantizations, three int8 tensor-core products
-with dequantizing epilogues) on a 4096 x 4096 linear layer with 65536 tokens, fp32 inputs,
+One step = one pass of the whole hot path over one batch: qlinear_fwd (Alg. 1) and qlinear_bwd
+(Alg. 2: both backward products) - five absmax reductions and quantizations, three int8
+tensor-core products with dequantizing epilogues - on a 4096 x 4096 linear layer with 65536 tokens, fp32 inputs,
 8-bit per-tensor stochastic rounding.  Prints one JSON line.
 """
 from __future__ import annotations
@@ -200,8 +200,7 @@ def run_ours(args):
     def step(i, a=A, w=W, dy=dY):
         qa_f, qw_f, qa_b, qw_b, qdy = specs(i)
         srq.qlinear_fwd(a, w, qa_f, qw_f, Y, None, ws)
-        srq.qlinear_bwd_input(dy, w, qdy, qw_b, dA, None, ws)
-        srq.qlinear_bwd_weight(dy, a, qdy, qa_b, dW, None, ws)
+        srq.qlinear_bwd(dy, a, w, qdy, qa_b, qw_b, dA, dW, None, None, ws)      # Alg. 2: both backward products
         if world > 1:
             dist.all_reduce(dW)        # the batch average of the weight gradient spans all shards
 

@@ -98,7 +98,7 @@ typedef struct {
 /* Bytes of workspace sr_quantize needs for a [rows, cols] input. */
 size_t srq_quantize_workspace_bytes(int64_t rows, int64_t cols);
 
-/* Bytes of workspace srq_gemm_i8 needs for an [M, N] output (split accumulators). */
+/* Bytes of workspace srq_gemm_i8 needs for an [M, N] output (partial sums of a split contraction). */
 size_t srq_gemm_workspace_bytes(int64_t M, int64_t N);
 
 /* Bytes of workspace that suffices for any one of the qlinear_* calls on a layer with
@@ -188,6 +188,19 @@ srq_status_t qlinear_bwd_weight(const void *dY, const void *A, srq_dtype_t dt,
                                 const srq_qspec_t *qdY, const srq_qspec_t *qA,
                                 float *dW, const srq_debug_out_t *dbg,
                                 void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Alg. 2 as a whole: dA[T,K] = Q(dY) Q(W) and dW[N,K] = Q(dY)^T Q(A) in one call.  Alg. 2
+ * quantizes dY once and uses it in both products; here dY is read once and its codes are written
+ * in both layouts ([T,N] for dA, [N,T] for dW) by the same pass, which saves one absmax and one
+ * quantization pass over dY compared with qlinear_bwd_input followed by qlinear_bwd_weight.  The
+ * results are bit for bit those of the two separate calls with the same quantization points.
+ * dbg_input / dbg_weight receive the operands and sums of the dA and dW products. */
+srq_status_t qlinear_bwd(const void *dY, const void *A, const void *W, srq_dtype_t dt,
+                         int64_t T, int64_t N, int64_t K,
+                         const srq_qspec_t *qdY, const srq_qspec_t *qA, const srq_qspec_t *qW,
+                         float *dA, float *dW,
+                         const srq_debug_out_t *dbg_input, const srq_debug_out_t *dbg_weight,
+                         void *ws, size_t ws_bytes, void *cuda_stream);
 
 /* Waits for the stream, then returns the device status word of the workspace: SRQ_OK, or the
  * first device-side condition recorded by the calls that used this workspace since its header

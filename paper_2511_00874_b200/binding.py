@@ -25,7 +25,7 @@ PER_TENSOR, PER_ROW = 0, 1
 SR, RTN = 0, 1
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
-           "sr_quantize", "sr_quantize_static", "srq_gemm_i8", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight",
+           "sr_quantize", "sr_quantize_static", "srq_gemm_i8", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
            "srq_poll_status", "srq_status_string", "srq_launch_count"]
 
 
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         f = getattr(L, name)
         f.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, qp, qp, vp, dp, vp, sz, vp]
         f.restype = ctypes.c_int
+    L.qlinear_bwd.argtypes = [vp, vp, vp, ctypes.c_int, i64, i64, i64, qp, qp, qp, vp, vp, dp, dp, vp, sz, vp]
+    L.qlinear_bwd.restype = ctypes.c_int
     L.srq_poll_status.argtypes = [vp, vp]
     L.srq_poll_status.restype = ctypes.c_int
     L.srq_status_string.argtypes = [ctypes.c_int]
@@ -270,6 +272,37 @@ def qlinear_bwd_weight(dY: torch.Tensor, A: torch.Tensor, qdY: QSpec, qA: QSpec,
     if T != T2 or tuple(dW.shape) != (N, K):
         raise ValueError("qlinear_bwd_weight: shapes must be dY[T,N], A[T,K], dW[N,K]")
     _layer("qlinear_bwd_weight", dY, A, T, N, K, qdY, qA, dW, dbg, ws)
+
+
+def qlinear_bwd(dY: torch.Tensor, A: torch.Tensor, W: torch.Tensor, qdY: QSpec, qA: QSpec, qW: QSpec,
+                dA: torch.Tensor, dW: torch.Tensor, dbg_input: Optional[DebugOut] = None,
+                dbg_weight: Optional[DebugOut] = None, ws: Optional[torch.Tensor] = None) -> None:
+    """Alg. 2 in one call: dA[T,K] = Q(dY) Q(W), dW[N,K] = Q(dY)^T Q(A); dY is read once."""
+    T, N = dY.shape
+    T2, K = A.shape
+    N2, K2 = W.shape
+    if T != T2 or N != N2 or K != K2 or tuple(dA.shape) != (T, K) or tuple(dW.shape) != (N, K):
+        raise ValueError("qlinear_bwd: shapes must be dY[T,N], A[T,K], W[N,K], dA[T,K], dW[N,K]")
+    for t, n in ((dY, "dY"), (A, "A"), (W, "W")):
+        _dev2d(t, n)
+        if not t.is_contiguous():
+            raise ValueError(f"{n} must be contiguous")
+    if not (_dtype_of(dY) == _dtype_of(A) == _dtype_of(W)):
+        raise TypeError("all operands must have the same dtype")
+    for t in (dA, dW):
+        if t.dtype != torch.float32 or not t.is_contiguous():
+            raise TypeError("outputs must be contiguous float32 tensors")
+    if ws is None:
+        ws = new_workspace(srq_workspace_bytes(T, N, K), dY.device)
+    c0, c1, c2 = qdY.c(), qA.c(), qW.c()
+    d0 = dbg_input.c() if dbg_input is not None else None
+    d1 = dbg_weight.c() if dbg_weight is not None else None
+    st = lib().qlinear_bwd(dY.data_ptr(), A.data_ptr(), W.data_ptr(), _dtype_of(dY), T, N, K,
+                           ctypes.byref(c0), ctypes.byref(c1), ctypes.byref(c2), dA.data_ptr(), dW.data_ptr(),
+                           ctypes.byref(d0) if d0 is not None else None,
+                           ctypes.byref(d1) if d1 is not None else None,
+                           ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "qlinear_bwd")
 
 
 def srq_poll_status(ws: torch.Tensor) -> int:

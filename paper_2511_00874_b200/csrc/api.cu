@@ -115,6 +115,114 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
     return SRQ_OK;
 }
 
+// Alg. 2 as one call: dY is read once and written in both code layouts, then both products run.
+struct BwdPlan {
+    size_t off_scratch[3], off_scale[4], off_codes[4], off_split[2], total;
+    int64_t pitch_n, pitch_t;
+};
+
+BwdPlan plan_bwd(int64_t T, int64_t N, int64_t K) {
+    BwdPlan p;
+    size_t o = sizeof(WsHeader);
+    const int64_t src[3][2] = {{T, N}, {N, K}, {T, K}};                 // dY, W, A
+    for (int i = 0; i < 3; ++i) { p.off_scratch[i] = o; o += quant_scratch_bytes(src[i][0], src[i][1]); }
+    const int64_t nscale[4] = {T, N, K, K};                             // dY [T,N], dY^T [N,T], W^T [K,N], A^T [K,T]
+    for (int i = 0; i < 4; ++i) { p.off_scale[i] = o; o += f32_block(nscale[i]); }
+    p.pitch_n = pitch16(N); p.pitch_t = pitch16(T);
+    const int64_t rows[4] = {T, N, K, K};
+    const int64_t pitch[4] = {p.pitch_n, p.pitch_t, p.pitch_n, p.pitch_t};
+    for (int i = 0; i < 4; ++i) { p.off_codes[i] = o; o += align_up((size_t)rows[i] * pitch[i]); }
+    p.off_split[0] = o; o += gemm_splitk_bytes(T, K);
+    p.off_split[1] = o; o += gemm_splitk_bytes(N, K);
+    p.total = o;
+    return p;
+}
+
+srq_status_t copy_debug(const srq_debug_out_t* dbg, const int8_t* ca, const float* sa, int64_t rows_a, bool per_row_a,
+                        const int8_t* cb, const float* sb, int64_t rows_b, bool per_row_b, int64_t Kc, int64_t pitch,
+                        cudaStream_t st) {
+    if (!dbg) return SRQ_OK;
+    if (dbg->codes_a && cudaMemcpy2DAsync(dbg->codes_a, (size_t)Kc, ca, (size_t)pitch, (size_t)Kc, (size_t)rows_a, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    if (dbg->codes_b && cudaMemcpy2DAsync(dbg->codes_b, (size_t)Kc, cb, (size_t)pitch, (size_t)Kc, (size_t)rows_b, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    if (dbg->scale_a && cudaMemcpyAsync(dbg->scale_a, sa, (per_row_a ? (size_t)rows_a : 1) * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    if (dbg->scale_b && cudaMemcpyAsync(dbg->scale_b, sb, (per_row_b ? (size_t)rows_b : 1) * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    return SRQ_OK;
+}
+
+srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
+                     const srq_qspec_t* qdY, const srq_qspec_t* qA, const srq_qspec_t* qW, float* dA, float* dW,
+                     const srq_debug_out_t* dbg_in, const srq_debug_out_t* dbg_w, void* ws, size_t ws_bytes, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!dY || !A || !W || !dA || !dW || !ws) return SRQ_ERR_INVALID_ARG;
+    if (dt != SRQ_F32 && dt != SRQ_BF16) return SRQ_ERR_INVALID_ARG;
+    if (T < 0 || N < 0 || K < 0) return SRQ_ERR_INVALID_ARG;
+    srq_status_t s;
+    if ((s = check_qspec(qdY)) != SRQ_OK) return s;
+    if ((s = check_qspec(qA)) != SRQ_OK) return s;
+    if ((s = check_qspec(qW)) != SRQ_OK) return s;
+    if (!aligned_to(dY, 16) || !aligned_to(A, 16) || !aligned_to(W, 16) || !aligned_to(dA, 16) || !aligned_to(dW, 16) || !aligned_to(ws, 256))
+        return SRQ_ERR_INVALID_ARG;
+    if ((double)N * qmax_of(qdY->bits) * qmax_of(qW->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
+    if ((double)T * qmax_of(qdY->bits) * qmax_of(qA->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
+    const BwdPlan p = plan_bwd(T, N, K);
+    if (ws_bytes < p.total) return SRQ_ERR_WORKSPACE;
+
+    char* base = (char*)ws;
+    uint32_t* status = &((WsHeader*)ws)->status;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    float* sc[4]; int8_t* cd[4];
+    for (int i = 0; i < 4; ++i) { sc[i] = (float*)(base + p.off_scale[i]); cd[i] = (int8_t*)(base + p.off_codes[i]); }
+
+    if (T > 0 && N > 0) {      // dY -> [T,N] codes for dA and [N,T] codes for dW, one read of dY
+        QuantArgs q; q.x = dY; q.dt = dt; q.rows = T; q.cols = N; q.ld = N; q.q = *qdY;
+        q.codes_rm = cd[0]; q.ld_rm = p.pitch_n; q.scale_rm = sc[0];
+        q.codes_tr = cd[1]; q.ld_tr = p.pitch_t; q.scale_tr = sc[1];
+        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[0], T, N), status, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    }
+    if (N > 0 && K > 0) {      // W -> [K,N]
+        QuantArgs q; q.x = W; q.dt = dt; q.rows = N; q.cols = K; q.ld = K; q.q = *qW;
+        q.codes_rm = nullptr; q.ld_rm = 0; q.scale_rm = nullptr;
+        q.codes_tr = cd[2]; q.ld_tr = p.pitch_n; q.scale_tr = sc[2];
+        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[1], N, K), status, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    }
+    if (T > 0 && K > 0) {      // A -> [K,T]
+        QuantArgs q; q.x = A; q.dt = dt; q.rows = T; q.cols = K; q.ld = K; q.q = *qA;
+        q.codes_rm = nullptr; q.ld_rm = 0; q.scale_rm = nullptr;
+        q.codes_tr = cd[3]; q.ld_tr = p.pitch_t; q.scale_tr = sc[3];
+        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[2], T, K), status, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    }
+
+    // dA[T,K] = Q(dY)[T,N] . Q(W)^T[K,N]
+    if (T > 0 && K > 0) {
+        if (N == 0) {
+            if (cudaMemset2DAsync(dA, (size_t)K * 4, 0, (size_t)K * 4, (size_t)T, st) != cudaSuccess) return SRQ_ERR_CUDA;
+        } else {
+            GemmArgs g;
+            g.a = cd[0]; g.lda = p.pitch_n; g.b = cd[2]; g.ldb = p.pitch_n; g.M = T; g.N = K; g.Kc = N;
+            g.s_row = sc[0]; g.row_stride = qdY->scale == SRQ_PER_ROW; g.s_col = sc[2]; g.col_stride = qW->scale == SRQ_PER_ROW;
+            g.out = dA; g.ldo = K; g.acc_out = dbg_in ? dbg_in->acc : nullptr;
+            g.splitk_ws = base + p.off_split[0]; g.splitk_ws_bytes = p.off_split[1] - p.off_split[0];
+            if ((s = launch_gemm_i8(g, status, st)) != SRQ_OK) return s;
+            if ((s = copy_debug(dbg_in, cd[0], sc[0], T, g.row_stride, cd[2], sc[2], K, g.col_stride, N, p.pitch_n, st)) != SRQ_OK) return s;
+        }
+    }
+    // dW[N,K] = Q(dY)^T[N,T] . Q(A)^T[K,T]
+    if (N > 0 && K > 0) {
+        if (T == 0) {
+            if (cudaMemset2DAsync(dW, (size_t)K * 4, 0, (size_t)K * 4, (size_t)N, st) != cudaSuccess) return SRQ_ERR_CUDA;
+        } else {
+            GemmArgs g;
+            g.a = cd[1]; g.lda = p.pitch_t; g.b = cd[3]; g.ldb = p.pitch_t; g.M = N; g.N = K; g.Kc = T;
+            g.s_row = sc[1]; g.row_stride = qdY->scale == SRQ_PER_ROW; g.s_col = sc[3]; g.col_stride = qA->scale == SRQ_PER_ROW;
+            g.out = dW; g.ldo = K; g.acc_out = dbg_w ? dbg_w->acc : nullptr;
+            g.splitk_ws = base + p.off_split[1]; g.splitk_ws_bytes = p.total - p.off_split[1];
+            if ((s = launch_gemm_i8(g, status, st)) != SRQ_OK) return s;
+            if ((s = copy_debug(dbg_w, cd[1], sc[1], N, g.row_stride, cd[3], sc[3], K, g.col_stride, T, p.pitch_t, st)) != SRQ_OK) return s;
+        }
+    }
+    return SRQ_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -139,6 +247,8 @@ size_t srq_workspace_bytes(int64_t T, int64_t N, int64_t K) {
     const size_t m1 = plan_layer(iy, iw).total, m2 = plan_layer(wy, wa).total;
     if (m1 > m) m = m1;
     if (m2 > m) m = m2;
+    const size_t m3 = plan_bwd(T, N, K).total;
+    if (m3 > m) m = m3;
     return m;
 }
 
@@ -206,6 +316,13 @@ srq_status_t qlinear_bwd_weight(const void* dY, const void* A, srq_dtype_t dt, i
                                 void* ws, size_t ws_bytes, void* cuda_stream) {
     const Operand a{dY, T, N, true, qdY}, b{A, T, K, true, qA};
     return run_layer(a, b, dt, dW, dbg, ws, ws_bytes, cuda_stream);
+}
+
+srq_status_t qlinear_bwd(const void* dY, const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
+                         const srq_qspec_t* qdY, const srq_qspec_t* qA, const srq_qspec_t* qW, float* dA, float* dW,
+                         const srq_debug_out_t* dbg_input, const srq_debug_out_t* dbg_weight,
+                         void* ws, size_t ws_bytes, void* cuda_stream) {
+    return run_bwd(dY, A, W, dt, T, N, K, qdY, qA, qW, dA, dW, dbg_input, dbg_weight, ws, ws_bytes, cuda_stream);
 }
 
 srq_status_t srq_poll_status(void* ws, void* cuda_stream) {

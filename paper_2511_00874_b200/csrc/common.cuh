@@ -59,7 +59,7 @@ struct GemmArgs {
     int64_t M, N, Kc;
     const float* s_row; int32_t row_stride; const float* s_col; int32_t col_stride;
     float* out; int64_t ldo; int32_t* acc_out;
-    void* splitk_ws; size_t splitk_ws_bytes;   // int32 [M,N] partial sums + tile tickets
+    void* splitk_ws; size_t splitk_ws_bytes;   // int32 [M,N] partial sums
 };
 size_t gemm_splitk_bytes(int64_t M, int64_t N);
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream);

@@ -20,8 +20,9 @@
 //               TMEM, two buffers of 256 columns, so the tensor pipe starts the next tile while
 //               the previous one is being drained
 //   warps 2-5   epilogue: tcgen05.ld the accumulator (one TMEM lane quarter per warp), convert,
-//               scale and store; or, for a split contraction, add the exact int32 partial
-//               sums into a workspace, the CTA that finishes a tile last doing the scaling
+//               scale and store (through shared memory and TMA block stores); or, for a split
+//               contraction, add the exact int32 partial sums into a zeroed workspace (TMA block
+//               reductions), which dequant_kernel scales afterwards
 // Ragged edges rely on TMA zero fill for loads and on bounds checks for stores.
 // Every wait is bounded by a wall-clock limit; on expiry the CTA records SRQ_ERR_TIMEOUT,
 // stops issuing work, waits (bounded) for what it has in flight, frees its TMEM and returns.
@@ -53,13 +54,14 @@ struct SharedTail {                                    // after the stage ring
     uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain;
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
-    uint32_t last_flag[2];
     uint32_t epi_abort;
     alignas(16) float s_col[2][BN];   // read as float4
 };
+constexpr int OUT_STAGE_BYTES = 32 * 32 * 4;           // one 32 x 32 block of 32-bit results per epilogue warp
 template <int CTAS>
 constexpr size_t gemm_smem() {
-    return 1024 /*alignment slack*/ + (size_t)Cfg<CTAS>::STAGES * Cfg<CTAS>::STAGE_BYTES + sizeof(SharedTail<Cfg<CTAS>::STAGES>);
+    return 1024 /*alignment slack*/ + (size_t)Cfg<CTAS>::STAGES * Cfg<CTAS>::STAGE_BYTES + 4 * OUT_STAGE_BYTES +
+           sizeof(SharedTail<Cfg<CTAS>::STAGES>);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -136,6 +138,32 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
             "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
             ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_addr) : "memory");
     }
+}
+
+// Block of results from shared memory to global memory; elements outside the tensor are clipped.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src_smem, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src_smem), "r"(x), "r"(y) : "memory");
+}
+// Same, added into global memory (32-bit integer adds performed by the memory system).
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src_smem, int32_t x, int32_t y) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src_smem), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }   // source reusable
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }         // writes performed
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Thread `lane` holds 32 consecutive 32-bit results of row `lane` of a 32 x 32 block: writes them as a
+// dense block with 128-byte rows in the 128-byte swizzle the tensor maps of the outputs use (16-byte
+// chunk index xor row mod 8), which also spreads each 16-byte store of a warp over all banks.
+__device__ __forceinline__ void stage_block(uint32_t stage, int lane, const uint32_t w[32]) {
+    const uint32_t row = stage + (uint32_t)lane * 128u;
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (uint32_t)((q ^ (lane & 7)) << 4)),
+                     "r"(w[4 * q]), "r"(w[4 * q + 1]), "r"(w[4 * q + 2]), "r"(w[4 * q + 3]) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -236,9 +264,10 @@ struct GemmParams {
     float* out; int64_t ldo;
     int32_t* acc_out;          // optional raw sums [M, N]
     int32_t* part;             // split contraction: zeroed int32 [M, N]
-    uint32_t* tickets;         // split contraction: zeroed, one per 128-row half of an output tile
     uint32_t* status;
     int32_t vec_out;           // 16-byte stores to out allowed
+    int32_t tma_out;           // out is written with TMA stores (map_out valid, no acc_out)
+    int32_t tma_part;          // partial sums are added with TMA reductions (map_part valid)
 };
 
 template <int STAGES>
@@ -249,14 +278,16 @@ __device__ __forceinline__ void give_up(SharedTail<STAGES>* T, uint32_t* status)
 
 template <int CTAS>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams P) {
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_part, const GemmParams P) {
     using C = Cfg<CTAS>;
     constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES;
     using Tail = SharedTail<STAGES>;
     extern __shared__ uint8_t smem_raw[];
     // the dynamic window starts at the same offset in every CTA, so the aligned layouts coincide
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    Tail* T = (Tail*)(smem + (size_t)STAGES * STAGE_BYTES);
+    uint8_t* out_stage = smem + (size_t)STAGES * STAGE_BYTES;          // 1024-byte aligned, 4 KB per epilogue warp
+    Tail* T = (Tail*)(out_stage + 4 * OUT_STAGE_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = CTAS == 1 ? 0u : cluster_ctarank();   // position in the CTA pair
     const bool leader = rank == 0;
@@ -386,7 +417,36 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (T->epi_abort) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
-            if (P.splits == 1) {
+            const uint32_t stage = smem_u32(out_stage + (warp - 2) * OUT_STAGE_BYTES);
+            const int32_t wrow = (int32_t)(row0 + quarter * 32);           // first row of this warp's blocks
+            if (P.splits == 1 && P.tma_out) {
+                // registers -> swizzled shared-memory block -> one TMA store per 32 x 32 block
+#pragma unroll 1
+                for (int j = 0; j < BN / 32; ++j) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + j * 32, v);
+                    tmem_ld_wait();
+                    const float* sc = &T->s_col[buf][j * 32];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 c4 = *reinterpret_cast<const float4*>(sc + 4 * q);
+                        v[4 * q + 0] = __float_as_uint(__fmul_rn(__int2float_rn((int)v[4 * q + 0]), __fmul_rn(sr, c4.x)));
+                        v[4 * q + 1] = __float_as_uint(__fmul_rn(__int2float_rn((int)v[4 * q + 1]), __fmul_rn(sr, c4.y)));
+                        v[4 * q + 2] = __float_as_uint(__fmul_rn(__int2float_rn((int)v[4 * q + 2]), __fmul_rn(sr, c4.z)));
+                        v[4 * q + 3] = __float_as_uint(__fmul_rn(__int2float_rn((int)v[4 * q + 3]), __fmul_rn(sr, c4.w)));
+                    }
+                    if (lane == 0) bulk_wait_read();          // the previous block has left the staging buffer
+                    __syncwarp();
+                    stage_block(stage, lane, v);
+                    fence_async_smem();
+                    __syncwarp();
+                    const int32_t col0 = (int32_t)col_base + j * 32;
+                    if (lane == 0 && wrow < P.M && col0 < P.N) { tma_store_2d(&map_out, stage, col0, wrow); bulk_commit(); }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
+            } else if (P.splits == 1) {
 #pragma unroll 1
                 for (int j = 0; j < BN / 32; ++j) {
                     uint32_t v[32];
@@ -431,7 +491,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
                     const int64_t col0 = col_base + j * 32;
-                    if (row < P.M && col0 < P.N) {
+                    if (P.tma_part) {
+                        if (lane == 0) bulk_wait_read();
+                        __syncwarp();
+                        stage_block(stage, lane, v);
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0 && wrow < P.M && col0 < P.N) { tma_reduce_add_2d(&map_part, stage, (int32_t)col0, wrow); bulk_commit(); }
+                    } else if (row < P.M && col0 < P.N) {
                         int32_t* pd = P.part + row * P.N + col0;
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
@@ -441,35 +508,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
-                __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (etid == 0) {
-                    const uint32_t t = atomicAdd(&P.tickets[tile * CTAS + rank], 1u);
-                    T->last_flag[buf] = (t == (uint32_t)P.splits - 1u) ? 1u : 0u;
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (T->last_flag[buf]) {
-                    __threadfence();
-                    // the last contributor scales the finished half tile: warp w takes rows w, w+4, ...
-                    const int ew = warp - 2;
-                    for (int r = ew; r < BM; r += 4) {
-                        const int64_t grow = row0 + r;
-                        if (grow >= P.M) break;
-                        const float srr = P.s_row[grow * P.row_stride];
-                        for (int cidx = lane; cidx < BN; cidx += 32) {
-                            const int64_t gcol = col_base + cidx;
-                            if (gcol < P.N) {
-                                const int32_t a = __ldcg(P.part + grow * P.N + gcol);
-                                P.out[grow * P.ldo + gcol] = __fmul_rn(__int2float_rn(a), __fmul_rn(srr, T->s_col[buf][cidx]));
-                                if (P.acc_out) P.acc_out[grow * P.N + gcol] = a;
-                            }
-                        }
-                    }
-                }
             }
         }
     }
 
+    if (warp >= 2 && lane == 0) bulk_wait_all();      // stores still reading the staging buffers
     // nobody leaves while the other CTA of the pair may still address this one's barriers, shared
     // memory or TMEM
     __syncwarp();
@@ -479,6 +522,34 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         __syncwarp();
         tc_fence_after();
         tmem_dealloc<CTAS>(tmem_base, TMEM_COLS);
+    }
+}
+
+// Second step of a split contraction: out = float(sum) * (s_row * s_col) over the finished sums.
+__global__ void __launch_bounds__(256)
+dequant_kernel(const int32_t* __restrict__ part, int64_t M, int64_t N, const float* __restrict__ s_row, int32_t row_stride,
+               const float* __restrict__ s_col, int32_t col_stride, float* __restrict__ out, int64_t ldo,
+               int32_t* __restrict__ acc_out, int vec) {
+    const int64_t nq = (N + 3) / 4;                      // groups of four columns per row
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < M * nq; g += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = g / nq, c = (g % nq) * 4;
+        const float sr = s_row[r * row_stride];
+        if (vec) {
+            const int4 a = __ldcg(reinterpret_cast<const int4*>(part + r * N + c));
+            float4 o;
+            o.x = __fmul_rn(__int2float_rn(a.x), __fmul_rn(sr, s_col[(c + 0) * col_stride]));
+            o.y = __fmul_rn(__int2float_rn(a.y), __fmul_rn(sr, s_col[(c + 1) * col_stride]));
+            o.z = __fmul_rn(__int2float_rn(a.z), __fmul_rn(sr, s_col[(c + 2) * col_stride]));
+            o.w = __fmul_rn(__int2float_rn(a.w), __fmul_rn(sr, s_col[(c + 3) * col_stride]));
+            *reinterpret_cast<float4*>(out + r * ldo + c) = o;
+            if (acc_out) *reinterpret_cast<int4*>(acc_out + r * N + c) = a;
+        } else {
+            for (int e = 0; e < 4 && c + e < N; ++e) {
+                const int32_t a = __ldcg(part + r * N + c + e);
+                out[r * ldo + c + e] = __fmul_rn(__int2float_rn(a), __fmul_rn(sr, s_col[(c + e) * col_stride]));
+                if (acc_out) acc_out[r * N + c + e] = a;
+            }
+        }
     }
 }
 
@@ -512,6 +583,18 @@ static bool encode_operand(CUtensorMap* map, const int8_t* base, int64_t rows, i
     cuuint32_t estr[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// [rows, cols] matrix of 32-bit elements with row pitch ld elements, boxes of 32 x 32, 128-byte swizzle.
+static bool encode_output(CUtensorMap* map, void* base, CUtensorMapDataType dt, int64_t rows, int64_t cols, int64_t ld) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Per device: SM count, the number of CTA pairs that can be resident at once, and the one-time
@@ -558,24 +641,23 @@ static int choose_splits(int64_t tiles, int32_t num_kb, int groups) {
     return (num_kb + per - 1) / per;
 }
 
-// Upper bound of what launch_gemm_i8 may use: int32 partial sums plus tickets, for outputs small
-// enough to be split.
+// What launch_gemm_i8 may use: an int32 matrix of partial sums, for outputs small enough to be split.
 size_t gemm_splitk_bytes(int64_t M, int64_t N) {
-    const int64_t tiles = 2 * ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);      // 128-row halves of whole pairs
-    if (tiles > 16 * 160) return 0;   // never split (bound is generous with respect to the SM count)
-    return align_up((size_t)M * N * 4) + align_up((size_t)tiles * 4);
+    const int64_t tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
+    if (tiles > 8 * 160) return 0;   // never split (bound is generous with respect to the SM count)
+    return align_up((size_t)M * N * 4);
 }
 
 template <int CTAS>
-static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& P,
-                                 cudaStream_t stream) {
+static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out,
+                                 const CUtensorMap& map_part, const GemmParams& P, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(groups * CTAS); cfg.blockDim = dim3(GEMM_THREADS);
     cfg.dynamicSmemBytes = gemm_smem<CTAS>(); cfg.stream = stream;
     cudaLaunchAttribute at;
     at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = CTAS; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
     cfg.attrs = &at; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_i8_kernel<CTAS>, map_a, map_b, P);
+    return cudaLaunchKernelEx(&cfg, gemm_i8_kernel<CTAS>, map_a, map_b, map_out, map_part, P);
 }
 
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream) {
@@ -596,15 +678,14 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.tiles_n = (int32_t)((g.N + BN - 1) / BN);
     const int64_t tiles = (int64_t)P.tiles_m * P.tiles_n;
     P.splits = choose_splits(tiles, P.num_kb, groups_max);
-    P.part = nullptr; P.tickets = nullptr;
+    P.part = nullptr;
     if (P.splits > 1) {
-        const size_t part_bytes = align_up((size_t)g.M * g.N * 4), ticket_bytes = align_up((size_t)tiles * ctas * 4);
-        if (g.splitk_ws == nullptr || g.splitk_ws_bytes < part_bytes + ticket_bytes) {
+        const size_t part_bytes = align_up((size_t)g.M * g.N * 4);
+        if (g.splitk_ws == nullptr || g.splitk_ws_bytes < part_bytes) {
             P.splits = 1;   // no room: run unsplit (same result)
         } else {
             P.part = (int32_t*)g.splitk_ws;
-            P.tickets = (uint32_t*)((char*)g.splitk_ws + part_bytes);
-            if (cudaMemsetAsync(g.splitk_ws, 0, part_bytes + ticket_bytes, stream) != cudaSuccess) return SRQ_ERR_CUDA;
+            if (cudaMemsetAsync(g.splitk_ws, 0, part_bytes, stream) != cudaSuccess) return SRQ_ERR_CUDA;
         }
     }
     P.s_row = g.s_row; P.row_stride = g.row_stride;
@@ -613,12 +694,30 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.status = status;
     P.vec_out = ((uintptr_t)g.out % 16 == 0) && (g.ldo % 4 == 0);
 
+    // results leave through TMA stores when the output (and the partial sums) meet the 16-byte rules
+    CUtensorMap map_out = map_a, map_part = map_a;       // placeholders when unused
+    P.tma_out = P.vec_out && !g.acc_out && g.M < (1ll << 31) && g.N < (1ll << 31) &&
+                encode_output(&map_out, g.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.M, g.N, g.ldo);
+    P.tma_part = P.splits > 1 && g.N % 4 == 0 && g.M < (1ll << 31) && g.N < (1ll << 31) &&
+                 encode_output(&map_part, P.part, CU_TENSOR_MAP_DATA_TYPE_INT32, g.M, g.N, g.N);
+
     const int64_t units = tiles * P.splits;
     const unsigned groups = (unsigned)(units < groups_max ? units : groups_max);
-    const cudaError_t e = ctas == 2 ? launch_kernel<2>(groups, map_a, map_b, P, stream)
-                                    : launch_kernel<1>(groups, map_a, map_b, P, stream);
+    const cudaError_t e = ctas == 2 ? launch_kernel<2>(groups, map_a, map_b, map_out, map_part, P, stream)
+                                    : launch_kernel<1>(groups, map_a, map_b, map_out, map_part, P, stream);
     ++g_launches;
-    return e == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+    if (e != cudaSuccess) return SRQ_ERR_CUDA;
+    if (P.splits > 1) {
+        const int vec = g.N % 4 == 0 && g.ldo % 4 == 0 && (uintptr_t)g.out % 16 == 0 && (!g.acc_out || (uintptr_t)g.acc_out % 16 == 0);
+        const int64_t work = g.M * ((g.N + 3) / 4);
+        const int64_t blocks = (work + 255) / 256;
+        const unsigned grid = (unsigned)(blocks < 8 * (int64_t)dev->sms ? blocks : 8 * (int64_t)dev->sms);
+        dequant_kernel<<<grid, 256, 0, stream>>>(P.part, g.M, g.N, g.s_row, g.row_stride, g.s_col, g.col_stride, g.out, g.ldo,
+                                                 g.acc_out, vec);
+        ++g_launches;
+        if (cudaGetLastError() != cudaSuccess) return SRQ_ERR_CUDA;
+    }
+    return SRQ_OK;
 }
 
 }  // namespace srq

@@ -43,6 +43,9 @@ def test_product_and_dequant_match_the_oracle(M, N, Kc, per_row):
     assert np.array_equal(acc, ref_acc)
     ref_out = oracle.dequant(ref_acc, s_row.cpu().numpy(), s_col.cpu().numpy())
     assert np.array_equal(out, ref_out)          # same two binary32 multiplies: 0 ulp
+    # without the raw sums the results leave through the block-store path: same values
+    out2, _ = _run(a, b, s_row, s_col, want_acc=False)
+    assert np.array_equal(out2, ref_out)
 
 
 def test_special_code_matrices():
@@ -73,6 +76,8 @@ def test_split_contraction_is_exact():
         ref_acc = oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy())
         assert np.array_equal(acc, ref_acc)
         assert np.array_equal(out, oracle.dequant(ref_acc, s_row.cpu().numpy(), s_col.cpu().numpy()))
+        out1, _ = _run(a, b, s_row, s_col, want_acc=False)     # split, partial sums added by block reductions
+        assert np.array_equal(out1, out)
         # and without the workspace (unsplit path) the result is the same
         out2 = torch.empty((M, N), device="cuda")
         ws = srq.new_workspace(256)
@@ -99,3 +104,24 @@ def test_many_tiles_per_cta_and_freivalds():
         l = rng.integers(-3, 4, (1, M))
         assert np.array_equal(l @ C64, (l @ A64) @ B64.T)
     assert np.array_equal(out, acc.astype(np.float32))
+    out2, _ = _run(a, b, one, one, want_acc=False)
+    assert np.array_equal(out2, out)
+
+
+@pytest.mark.parametrize("M,N,Kc,pad", [(300, 260, 256, 0), (257, 36, 130, 4), (4096, 96, 512, 0), (520, 1000, 384, 24), (130, 70, 64, 1)])
+def test_output_pitch_and_ragged_edges_on_the_block_store_path(M, N, Kc, pad):
+    """No raw sums requested: every result goes through shared memory and a clipped block store.
+    The output has a row pitch larger than N and guard values around it that must survive."""
+    a, b = _codes(M, Kc, 31), _codes(N, Kc, 32)
+    s_row = torch.rand(M, device="cuda") + 0.5
+    s_col = torch.rand(N, device="cuda") + 0.5
+    full = torch.full((M + 2, N + pad + 8), 7.5, device="cuda")
+    out = full[1:M + 1, 4:4 + N] if pad else full[1:M + 1, :N]
+    ws = srq.new_workspace(srq.srq_gemm_workspace_bytes(M, N))
+    srq.srq_gemm_i8(a, b, s_row, s_col, out, None, ws)
+    assert srq.srq_poll_status(ws) == 0
+    ref = oracle.dequant(oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy()), s_row.cpu().numpy(), s_col.cpu().numpy())
+    assert np.array_equal(out.cpu().numpy(), ref)
+    guard = full.clone()
+    guard[1:M + 1, (4 if pad else 0):(4 if pad else 0) + N] = 7.5
+    assert bool((guard == 7.5).all()), "a store went outside the output"

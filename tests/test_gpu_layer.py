@@ -53,6 +53,11 @@ def run_pass(name, X0, X1, T, N, K, q0, q1, ws=None, full=True):
         o = out.cpu().numpy()
         assert _ulp_diff(o, ref.out) <= 1, name + ": fp32 output beyond 1 ulp"
         assert np.array_equal(o, ref.out), name + ": fp32 output"
+        # the same call without the debug copies (the product then stores whole blocks): same output
+        out2 = torch.full(shapes[2], float("nan"), device=dev)
+        fn(X0, X1, q0, q1, out2, None, ws)
+        assert srq.srq_poll_status(ws) == 0
+        assert np.array_equal(out2.cpu().numpy(), ref.out), name + ": fp32 output without debug copies"
     return out, ref
 
 
@@ -117,6 +122,47 @@ def test_workspace_reuse_and_shared_quantized_weight():
     assert srq.srq_poll_status(ws) == 0
     assert torch.equal(cw.t(), cwt)
     all_passes(A, W, dY, q, ws)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("scale", [srq.PER_TENSOR, srq.PER_ROW])
+@pytest.mark.parametrize("shape", [(264, 392, 328), (37, 21, 50), (512, 256, 384)])
+def test_whole_backward_pass_in_one_call(dtype, scale, shape):
+    """qlinear_bwd (Alg. 2 as one call, dY read once) against the oracle's two backward products:
+    codes of all four operands, step sizes, int32 sums and outputs bit for bit."""
+    T, N, K = shape
+    A, W, dY = synth.layer_inputs(T, N, K, seed=5, dtype=dtype, device="cuda", std_dy=1e-3)
+    q = layer_specs(scale, srq.SR, seed=2, bits_fwd=8, bits_bwd=6)
+    dev = A.device
+    per_row = scale == srq.PER_ROW
+    n = lambda rows: rows if per_row else 1
+    dA = torch.full((T, K), float("nan"), device=dev)
+    dW = torch.full((N, K), float("nan"), device=dev)
+    di = srq.DebugOut(torch.empty((T, N), dtype=torch.int8, device=dev), torch.empty(n(T), device=dev),
+                      torch.empty((K, N), dtype=torch.int8, device=dev), torch.empty(n(K), device=dev),
+                      torch.empty((T, K), dtype=torch.int32, device=dev))
+    dw = srq.DebugOut(torch.empty((N, T), dtype=torch.int8, device=dev), torch.empty(n(N), device=dev),
+                      torch.empty((K, T), dtype=torch.int8, device=dev), torch.empty(n(K), device=dev),
+                      torch.empty((N, K), dtype=torch.int32, device=dev))
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K), dev)
+    srq.qlinear_bwd(dY, A, W, q["dy_bwd"], q["a_bwd"], q["w_bwd"], dA, dW, di, dw, ws)
+    assert srq.srq_poll_status(ws) == 0
+    oq = lambda s: oracle.QSpec(s.bits, s.scale, s.round, s.seed, s.tensor_id, s.index_offset)
+    f = lambda t: t.float().cpu().numpy()
+    ri = oracle.qlinear_bwd_input(f(dY), f(W), oq(q["dy_bwd"]), oq(q["w_bwd"]))
+    rw = oracle.qlinear_bwd_weight(f(dY), f(A), oq(q["dy_bwd"]), oq(q["a_bwd"]))
+    for name, dbg, out, ref in (("dA", di, dA, ri), ("dW", dw, dW, rw)):
+        assert np.array_equal(dbg.codes_a.cpu().numpy(), ref.codes_a), name + ": codes of first operand"
+        assert np.array_equal(dbg.codes_b.cpu().numpy(), ref.codes_b), name + ": codes of second operand"
+        assert np.array_equal(dbg.scale_a.cpu().numpy(), ref.scale_a), name + ": step sizes of first operand"
+        assert np.array_equal(dbg.scale_b.cpu().numpy(), ref.scale_b), name + ": step sizes of second operand"
+        assert np.array_equal(dbg.acc.cpu().numpy(), ref.acc), name + ": int32 sums"
+        assert np.array_equal(out.cpu().numpy(), ref.out), name + ": fp32 output"
+    # without debug copies (block-store epilogue), same outputs
+    dA2, dW2 = torch.empty_like(dA), torch.empty_like(dW)
+    srq.qlinear_bwd(dY, A, W, q["dy_bwd"], q["a_bwd"], q["w_bwd"], dA2, dW2, None, None, ws)
+    assert srq.srq_poll_status(ws) == 0
+    assert torch.equal(dA2, dA) and torch.equal(dW2, dW)
 
 
 def test_overflowing_contraction_is_refused():
