@@ -27,8 +27,8 @@ WORKLOAD = "linear 4096->4096, tokens 65536, fp32 inputs, 8-bit per-tensor SR on
 T_FULL, N_FULL, K_FULL = 65536, 4096, 4096
 
 # DRAM bytes (read + write) of one gemm_i8_kernel launch of this workload, from the ncu capture
-# summarised in profiles/; None until a capture has been taken.
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+# summarised in profiles/gemm_i8_kernel_M8192_N4096_K4096.md (its bench-size section).
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 1338378752   # forward-shaped launch, M=65536 N=4096 K=4096
 
 
 def layer_ops(T, N, K):
@@ -114,10 +114,13 @@ def oracle_layer_seconds(T, N, K, seed=0):
 
 def pick_oracle_sample(target_s):
     """Token count of the slice the oracle can do in about target_s seconds on this host."""
-    probe_T = 32
-    t = oracle_layer_seconds(probe_T, N_FULL, K_FULL)
-    Ts = probe_T
-    while Ts * 2 <= T_FULL and t * (Ts * 2 / probe_T) <= target_s:
+    # two probes separate the part that does not grow with the tokens (quantizing W) from the rest
+    t1 = oracle_layer_seconds(64, N_FULL, K_FULL)
+    t2 = oracle_layer_seconds(256, N_FULL, K_FULL)
+    per_token = max((t2 - t1) / 192.0, 1e-9)
+    fixed = max(t1 - 64 * per_token, 0.0)
+    Ts = 256
+    while Ts * 2 <= T_FULL and fixed + per_token * Ts * 2 <= target_s:
         Ts *= 2
     return Ts
 
@@ -197,12 +200,12 @@ def run_ours(args):
                 srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 2, off_a), srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 3),
                 srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 4, off_y))
 
-    def step(i, a=A, w=W, dy=dY):
+    def step(i, a=A, w=W, dy=dY, y=Y, da=dA, dw=dW):
         qa_f, qw_f, qa_b, qw_b, qdy = specs(i)
-        srq.qlinear_fwd(a, w, qa_f, qw_f, Y, None, ws)
-        srq.qlinear_bwd(dy, a, w, qdy, qa_b, qw_b, dA, dW, None, None, ws)      # Alg. 2: both backward products
+        srq.qlinear_fwd(a, w, qa_f, qw_f, y, None, ws)
+        srq.qlinear_bwd(dy, a, w, qdy, qa_b, qw_b, da, dw, None, None, ws)      # Alg. 2: both backward products
         if world > 1:
-            dist.all_reduce(dW)        # the batch average of the weight gradient spans all shards
+            dist.all_reduce(dw)        # the batch average of the weight gradient spans all shards
 
     def barrier():
         if world > 1:
@@ -247,21 +250,39 @@ def run_ours(args):
                          "multi_gpu": "token shards, one NCCL all-reduce of dW per step" if world > 1 else "single GPU"},
               "gpu_launches": int(launches)}
 
-    # ---- end to end through the public API with host buffers (every rank, max over ranks)
+    # ---- end to end through the public API with host buffers (every rank, max over ranks).
+    # Every step copies its inputs from pinned host memory and its results back; the copies of
+    # neighbouring steps overlap with the compute on two copy streams (two sets of device buffers).
     hA, hW, hdY = (t.cpu().pin_memory() for t in (A, W, dY))
     hY, hdA, hdW = (torch.empty_like(t, device="cpu").pin_memory() for t in (Y, dA, dW))
-    e_steps = max(1, min(3, args.steps))
+    e_steps = max(2, min(8, args.steps))
+    ins = [(A, W, dY), tuple(torch.empty_like(t) for t in (A, W, dY))]
+    outs = [(Y, dA, dW), tuple(torch.empty_like(t) for t in (Y, dA, dW))]
+    s_in, s_out, s_main = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+    ev_in = [torch.cuda.Event() for _ in range(e_steps)]
+    ev_comp = [torch.cuda.Event() for _ in range(e_steps)]
+    ev_out = [torch.cuda.Event() for _ in range(e_steps)]
     barrier()
     t0 = time.perf_counter()
     for i in range(e_steps):
-        a_ = hA.to(dev, non_blocking=True)
-        w_ = hW.to(dev, non_blocking=True)
-        y_ = hdY.to(dev, non_blocking=True)
-        step(1000 + i, a_, w_, y_)
-        hY.copy_(Y, non_blocking=True)
-        hdA.copy_(dA, non_blocking=True)
-        hdW.copy_(dW, non_blocking=True)
-        torch.cuda.synchronize()
+        b = i % 2
+        with torch.cuda.stream(s_in):
+            if i >= 2:
+                s_in.wait_event(ev_comp[i - 2])           # step i-2 no longer reads these inputs
+            for d, h in zip(ins[b], (hA, hW, hdY)):
+                d.copy_(h, non_blocking=True)
+            ev_in[i].record(s_in)
+        s_main.wait_event(ev_in[i])
+        if i >= 2:
+            s_main.wait_event(ev_out[i - 2])              # the results of step i-2 have left these outputs
+        step(1000 + i, *ins[b], *outs[b])
+        ev_comp[i].record(s_main)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_comp[i])
+            for h, d in zip((hY, hdA, hdW), outs[b]):
+                h.copy_(d, non_blocking=True)
+            ev_out[i].record(s_out)
+    torch.cuda.synchronize()
     e_sec = (time.perf_counter() - t0) / e_steps
     if world > 1:
         t = torch.tensor([e_sec], device=dev)
@@ -271,8 +292,9 @@ def run_ours(args):
     d2h = sum(t.numel() * 4 for t in (hY, hdA, hdW))
     result["e2e"] = {"value": world * layer_ops(T, N, K) / e_sec / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                      "d2h_bytes_per_step": d2h, "steps": e_steps, "ms_per_step": e_sec * 1e3,
-                     "note": "per rank: pinned host A, W, dY copied in and Y, dA, dW copied out every step"}
-    del hA, hW, hdY, hY, hdA, hdW
+                     "note": "per rank: pinned host A, W, dY copied in and Y, dA, dW copied out every step; "
+                             "copies of neighbouring steps overlap with compute (host link bound)"}
+    del hA, hW, hdY, hY, hdA, hdW, ins, outs
 
     if rank == 0:
         # ---- per-kernel timing of the dominant kernel: the three products of one step, on the codes
@@ -353,7 +375,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
