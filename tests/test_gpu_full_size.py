@@ -1,0 +1,108 @@
+"""Parity at the benchmark's full size and launch configuration.
+
+Linear layer 4096 -> 4096 with 65536 tokens, fp32 inputs, 8-bit per-tensor SR: the workload
+`bench.py` times, called the way it calls it (no debug copies, so the products run as CTA pairs
+and store their results as whole blocks).  The oracle cannot form 3 x 1.1e12 products in a test,
+so the comparison is:
+  - every int8 code and step size of all operands against the oracle's quantizer (bit for bit);
+  - sampled rows of Y, dA and dW against oracle products of the oracle's codes (bit for bit);
+  - the whole of every output against a second GPU path (the product on the same codes with raw
+    sums requested, which stores element-wise) and that path's int32 sums against exact
+    Freivalds products  acc r == qa (qb^T r)  evaluated in binary64, where they are exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2511_00874_b200 as srq
+from paper_2511_00874_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+T, N, K = 65536, 4096, 4096
+
+
+def _oq(q):
+    return oracle.QSpec(q.bits, q.scale, q.round, q.seed, q.tensor_id, q.index_offset)
+
+
+def _codes(x, q, rm, tr):
+    rows, cols = x.shape
+    crm = torch.empty((rows, cols), dtype=torch.int8, device="cuda") if rm else None
+    ctr = torch.empty((cols, rows), dtype=torch.int8, device="cuda") if tr else None
+    s1, s2 = torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
+    srq.sr_quantize(x, q, crm, s1 if rm else None, ctr, s2 if tr else None)
+    return crm, ctr, (s1 if rm else s2)
+
+
+def _freivalds(acc, qa, qb, rng):
+    """acc[M,N] == qa[M,Kc] qb[N,Kc]^T checked with random small-integer vectors, exactly."""
+    accd = acc.double()
+    for _ in range(2):
+        r = torch.from_numpy(rng.integers(-3, 4, (qb.shape[0], 1)).astype(np.float64)).cuda()
+        # chunked so that the binary64 copies of the code matrices stay small
+        right = torch.zeros((qb.shape[1], 1), dtype=torch.float64, device="cuda")
+        for j in range(0, qb.shape[0], 4096):
+            right += qb[j:j + 4096].double().t() @ r[j:j + 4096]
+        lhs = accd @ r
+        for i in range(0, qa.shape[0], 8192):
+            assert torch.equal(lhs[i:i + 8192], qa[i:i + 8192].double() @ right)
+
+
+def test_benchmark_layer_at_full_size():
+    A = synth.normal((T, K), 1.0, 1000, torch.float32, "cuda")
+    dY = synth.normal((T, N), 1e-3, 1001, torch.float32, "cuda")
+    W = synth.normal((N, K), 0.02, 7, torch.float32, "cuda")
+    q = {k: srq.QSpec(8, srq.PER_TENSOR, srq.SR, 3, i) for i, k in enumerate(["a_f", "w_f", "a_b", "w_b", "dy"])}
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
+    Y = torch.empty((T, N), device="cuda")
+    dA = torch.empty((T, K), device="cuda")
+    dW = torch.empty((N, K), device="cuda")
+    srq.qlinear_fwd(A, W, q["a_f"], q["w_f"], Y, None, ws)
+    srq.qlinear_bwd(dY, A, W, q["dy"], q["a_b"], q["w_b"], dA, dW, None, None, ws)
+    assert srq.srq_poll_status(ws) == 0
+
+    # ---- codes and step sizes of every operand, whole tensors, against the oracle
+    hA, hW, hdY = A.cpu().numpy(), W.cpu().numpy(), dY.cpu().numpy()
+    o_af = oracle.sr_quantize(hA, _oq(q["a_f"]), True, False)
+    o_wf = oracle.sr_quantize(hW, _oq(q["w_f"]), True, False)
+    o_dy = oracle.sr_quantize(hdY, _oq(q["dy"]), True, True)
+    o_wb = oracle.sr_quantize(hW, _oq(q["w_b"]), False, True)
+    o_ab = oracle.sr_quantize(hA, _oq(q["a_b"]), False, True)
+    g_af, _, s_af = _codes(A, q["a_f"], True, False)
+    g_wf, _, s_wf = _codes(W, q["w_f"], True, False)
+    g_dy, g_dyt, s_dy = _codes(dY, q["dy"], True, True)
+    _, g_wbt, s_wb = _codes(W, q["w_b"], False, True)
+    _, g_abt, s_ab = _codes(A, q["a_b"], False, True)
+    for name, g, o in (("A fwd", g_af, o_af[0]), ("W fwd", g_wf, o_wf[0]), ("dY", g_dy, o_dy[0]),
+                       ("dY^T", g_dyt, o_dy[2]), ("W^T bwd", g_wbt, o_wb[2]), ("A^T bwd", g_abt, o_ab[2])):
+        assert np.array_equal(g.cpu().numpy(), o), name + ": codes"
+    for name, g, o in (("A fwd", s_af, o_af[1]), ("W fwd", s_wf, o_wf[1]), ("dY", s_dy, o_dy[1]),
+                       ("W bwd", s_wb, o_wb[3]), ("A bwd", s_ab, o_ab[3])):
+        assert np.array_equal(g.cpu().numpy(), o), name + ": step size"
+
+    # ---- sampled rows of the three outputs against oracle products of the oracle's codes
+    rng = np.random.default_rng(0)
+    rows_t = np.sort(rng.choice(T, 48, replace=False))
+    rows_n = np.sort(rng.choice(N, 12, replace=False))
+    ref = oracle.dequant(oracle.gemm_i8_nt(o_af[0][rows_t], o_wf[0]), o_af[1], o_wf[1])
+    assert np.array_equal(Y[torch.from_numpy(rows_t).cuda()].cpu().numpy(), ref), "Y rows"
+    ref = oracle.dequant(oracle.gemm_i8_nt(o_dy[0][rows_t], o_wb[2]), o_dy[1], o_wb[3])
+    assert np.array_equal(dA[torch.from_numpy(rows_t).cuda()].cpu().numpy(), ref), "dA rows"
+    ref = oracle.dequant(oracle.gemm_i8_nt(o_dy[2][rows_n], o_ab[2]), o_dy[3], o_ab[3])
+    assert np.array_equal(dW[torch.from_numpy(rows_n).cuda()].cpu().numpy(), ref), "dW rows"
+    del hA, hW, hdY, o_af, o_wf, o_dy, o_wb, o_ab
+
+    # ---- whole outputs: the element-wise path on the same codes gives the same values, and its
+    # int32 sums pass exact Freivalds checks
+    gws = srq.new_workspace(srq.srq_gemm_workspace_bytes(N, K))
+    for name, qa, qb, sa, sb, out in (("Y", g_af, g_wf, s_af, s_wf, Y), ("dA", g_dy, g_wbt, s_dy, s_wb, dA),
+                                      ("dW", g_dyt, g_abt, s_dy, s_ab, dW)):
+        acc = torch.empty(out.shape, dtype=torch.int32, device="cuda")
+        out2 = torch.empty_like(out)
+        srq.srq_gemm_i8(qa, qb, sa, sb, out2, acc, gws)
+        assert srq.srq_poll_status(gws) == 0
+        assert torch.equal(out2, out), name + ": block-store path differs from the element-wise path"
+        _freivalds(acc, qa, qb, rng)
+        del acc, out2
