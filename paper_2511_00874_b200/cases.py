@@ -4,7 +4,12 @@
     python -m paper_2511_00874_b200.cases gemm --M 8192 --N 4096 --K 4096
     python -m paper_2511_00874_b200.cases layer --T 16384 --N 2304 --K 768
 
-Used for the per-configuration sweeps and as the small, self-ending command that profiler
+    python -m paper_2511_00874_b200.cases sweep --config 3
+
+`sweep` runs one of the synthetic workload families (2: quantizer sweep, 3: GPT-2-small shaped
+layers, 4: Llama-style 1.1B layers in bf16 with per-row scales, 5: batch size against precision
+on a 4096 x 4096 layer, with the error of the quantized weight gradient) and prints one JSON
+line per case.  The single-case commands are also the small, self-ending commands that profiler
 captures are taken on.  Timing is by CUDA events on the launching stream; between iterations a
 buffer larger than L2 is rewritten unless the case's own inputs exceed L2.
 """
@@ -78,24 +83,29 @@ def case_gemm(a):
             "out_GBps": 4.0 * a.M * a.N / med / 1e6}
 
 
+def _layer_fn(A, W, dY, q, Y, dA, dW, ws):
+    def fn():
+        B.qlinear_fwd(A, W, q["a_fwd"], q["w_fwd"], Y, None, ws)
+        B.qlinear_bwd(dY, A, W, q["dy"], q["a_bwd"], q["w_bwd"], dA, dW, None, None, ws)
+    return fn
+
+
+def _layer_specs(bits_fwd, bits_bwd, sc, rd, seed):
+    return {k: B.QSpec(b, sc, rd, seed, i) for i, (k, b) in enumerate(
+        [("a_fwd", bits_fwd), ("w_fwd", bits_fwd), ("a_bwd", bits_bwd), ("w_bwd", bits_bwd), ("dy", bits_bwd)])}
+
+
 def case_layer(a):
     dt = torch.float32 if a.dtype == "f32" else torch.bfloat16
     A, W, dY = synth.layer_inputs(a.T, a.N, a.K, a.seed, dt, "cuda", std_dy=1e-3)
     sc = B.PER_ROW if a.scale == "row" else B.PER_TENSOR
     rd = B.SR if a.round == "sr" else B.RTN
-    q = {k: B.QSpec(b, sc, rd, a.seed, i) for i, (k, b) in enumerate(
-        [("a_fwd", a.bits_fwd), ("w_fwd", a.bits_fwd), ("a_bwd", a.bits_bwd), ("w_bwd", a.bits_bwd),
-         ("dy", a.bits_bwd)])}
+    q = _layer_specs(a.bits_fwd, a.bits_bwd, sc, rd, a.seed)
     Y = torch.empty((a.T, a.N), device="cuda")
     dA = torch.empty((a.T, a.K), device="cuda")
     dW = torch.empty((a.N, a.K), device="cuda")
     ws = B.new_workspace(B.srq_workspace_bytes(a.T, a.N, a.K))
-
-    def fn():
-        B.qlinear_fwd(A, W, q["a_fwd"], q["w_fwd"], Y, None, ws)
-        B.qlinear_bwd_input(dY, W, q["dy"], q["w_bwd"], dA, None, ws)
-        B.qlinear_bwd_weight(dY, A, q["dy"], q["a_bwd"], dW, None, ws)
-
+    fn = _layer_fn(A, W, dY, q, Y, dA, dW, ws)
     small = (A.numel() + dY.numel()) * A.element_size() < 2 * L2_BYTES
     med, best = _time(fn, a.iters, a.warmup, flush=small)
     assert B.srq_poll_status(ws) == 0
@@ -105,10 +115,110 @@ def case_layer(a):
             "TOPS": ops / med / 1e9}
 
 
+# ---------------------------------------------------------------------------------------------
+# workload families
+# ---------------------------------------------------------------------------------------------
+def _ns(**kw):
+    return argparse.Namespace(**kw)
+
+
+def sweep_quantizer(a):
+    """Config 2: 2^20 .. 2^28 elements as [n / 4096, 4096], fp32 and bf16, bits 8 / 6 / 4, per tensor and
+    per row, SR and RTN, seeds 0-3 (median over the seeds)."""
+    for logn in (20, 22, 24, 26, 28):
+        rows = (1 << logn) // 4096
+        for dtype in ("f32", "bf16"):
+            for bits in (8, 6, 4):
+                for scale in ("tensor", "row"):
+                    for rnd in ("sr", "rtn"):
+                        ms, gb = [], []
+                        for seed in range(4):
+                            r = case_quantize(_ns(rows=rows, cols=4096, dtype=dtype, bits=bits, scale=scale, round=rnd,
+                                                  layouts="rm", seed=seed, iters=a.iters, warmup=a.warmup))
+                            ms.append(r["ms"]); gb.append(r["GBps"])
+                        yield {"config": 2, "elements": 1 << logn, "dtype": dtype, "bits": bits, "scale": scale,
+                               "round": rnd, "ms": statistics.median(ms), "GBps": statistics.median(gb)}
+
+
+def sweep_gpt2(a):
+    """Config 3: GPT-2-small shaped layers, fp32, 8-bit per-tensor SR on W, A and dY."""
+    for name, (K, N) in synth.GPT2_SMALL_LAYERS.items():
+        for batch in (1, 4, 16, 64):
+            r = case_layer(_ns(T=batch * 1024, N=N, K=K, dtype="f32", bits_fwd=8, bits_bwd=8, scale="tensor", round="sr",
+                               seed=0, iters=a.iters, warmup=a.warmup))
+            r.update({"config": 3, "layer": name})
+            yield r
+
+
+def sweep_llama(a):
+    """Config 4: Llama-style 1.1B layers, bf16 inputs, per-row scales, 8-bit forward, 4-bit SR backward."""
+    for name, (K, N) in synth.LLAMA_1B_LAYERS.items():
+        if name == "up":
+            continue                     # same shape as gate
+        for batch in (1, 8, 32):
+            r = case_layer(_ns(T=batch * 2048, N=N, K=K, dtype="bf16", bits_fwd=8, bits_bwd=4, scale="row", round="sr",
+                               seed=0, iters=a.iters, warmup=a.warmup))
+            r.update({"config": 4, "layer": name + ("/up" if name == "gate" else "")})
+            yield r
+
+
+def _rounding_variance(x, bits):
+    """Mean over the tensor of the variance SR adds to one element, D^2 p (1 - p) (per-tensor step)."""
+    m = x.abs().max()
+    qmax = float((1 << (bits - 1)) - 1)
+    d = m / qmax
+    t = x / d
+    p = t - torch.floor(t)
+    return float((d * d * (p * (1 - p)).mean()).item())
+
+
+def sweep_batch_precision(a):
+    """Config 5: 4096 x 4096 layer, tokens 512 .. 65536, bits 8 / 6 / 4 / 3, SR and RTN, 5 seeds.  Besides the
+    throughput, the mean squared error of the quantized dW / T against the unquantized dY^T A / T
+    (binary64), next to what the variance lemma (Lemma 3) predicts for SR:
+    (E[A^2] var_dY + E[dY^2] var_A + var_A var_dY) / T with var_X the mean rounding variance of X."""
+    N = K = 4096
+    for T in (512, 1024, 2048, 4096, 8192, 16384, 32768, 65536):
+        A, W, dY = synth.layer_inputs(T, N, K, 0, torch.float32, "cuda", std_dy=1e-3)
+        ref = torch.zeros((N, K), dtype=torch.float64, device="cuda")
+        for i in range(0, T, 8192):                        # binary64 in slices to bound memory
+            ref += dY[i:i + 8192].double().t() @ A[i:i + 8192].double()
+        ref /= T
+        Y = torch.empty((T, N), device="cuda")
+        dA = torch.empty((T, K), device="cuda")
+        dW = torch.empty((N, K), device="cuda")
+        ws = B.new_workspace(B.srq_workspace_bytes(T, N, K))
+        ea2, edy2 = float((A.double() ** 2).mean()), float((dY.double() ** 2).mean())
+        for bits in (8, 6, 4, 3):
+            va, vdy = _rounding_variance(A, bits), _rounding_variance(dY, bits)
+            predicted = (ea2 * vdy + edy2 * va + va * vdy) / T
+            for rnd in ("sr", "rtn"):
+                mses, times = [], []
+                for seed in range(5):
+                    q = _layer_specs(bits, bits, B.PER_TENSOR, B.SR if rnd == "sr" else B.RTN, seed)
+                    fn = _layer_fn(A, W, dY, q, Y, dA, dW, ws)
+                    med, _ = _time(fn, max(3, a.iters // 4), 2, flush=T < 8192)
+                    times.append(med)
+                    mses.append(float((((dW.double() / T) - ref) ** 2).mean()))
+                assert B.srq_poll_status(ws) == 0
+                ms = statistics.median(times)
+                yield {"config": 5, "T": T, "bits": bits, "round": rnd, "ms": ms, "TOPS": 6.0 * T * N * K / ms / 1e9,
+                       "dW_mse": statistics.mean(mses), "dW_mse_min": min(mses), "dW_mse_max": max(mses),
+                       "lemma3_sr_variance": predicted, "dW_ref_mean_square": float((ref ** 2).mean())}
+        del A, W, dY, Y, dA, dW, ws, ref
+
+
+def case_sweep(a):
+    gen = {2: sweep_quantizer, 3: sweep_gpt2, 4: sweep_llama, 5: sweep_batch_precision}[a.config](a)
+    for r in gen:
+        print(json.dumps(r), flush=True)
+    return None
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     sub = ap.add_subparsers(dest="op", required=True)
-    for name in ("quantize", "gemm", "layer"):
+    for name in ("quantize", "gemm", "layer", "sweep"):
         p = sub.add_parser(name)
         p.add_argument("--iters", type=int, default=20)
         p.add_argument("--warmup", type=int, default=3)
@@ -128,15 +238,18 @@ def main(argv=None):
             p.add_argument("--K", type=int, default=4096)
             p.add_argument("--bits-fwd", dest="bits_fwd", type=int, default=8)
             p.add_argument("--bits-bwd", dest="bits_bwd", type=int, default=8)
-        if name != "gemm":
+        if name == "sweep":
+            p.add_argument("--config", type=int, required=True, choices=[2, 3, 4, 5])
+        if name not in ("gemm", "sweep"):
             p.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
             p.add_argument("--scale", default="tensor", choices=["tensor", "row"])
             p.add_argument("--round", default="sr", choices=["sr", "rtn"])
     a = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("a CUDA device is required (there is no CPU fallback)")
-    res = {"quantize": case_quantize, "gemm": case_gemm, "layer": case_layer}[a.op](a)
-    print(json.dumps(res))
+    res = {"quantize": case_quantize, "gemm": case_gemm, "layer": case_layer, "sweep": case_sweep}[a.op](a)
+    if res is not None:
+        print(json.dumps(res))
 
 
 if __name__ == "__main__":
