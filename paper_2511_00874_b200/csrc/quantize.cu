@@ -78,53 +78,87 @@ __device__ __forceinline__ uint32_t abs_bits(float v) { return __float_as_uint(v
 // absmax
 // ------------------------------------------------------------------------------------------
 constexpr int AMAX_THREADS = 256;
-constexpr int AMAX_TILE_C = 512;   // 32 lanes x 4 groups x 4 elements
 constexpr int AMAX_TILE_R = 64;    // 8 warps x 8 rows
+constexpr int AMAX_GROUPS = 2;     // 16-byte groups per lane and row
+
+// Absolute-value bit patterns of the elements of one 16-byte group.
+__device__ __forceinline__ void abs_bits16(const uint4& q, uint32_t (&b)[4], float) {
+    b[0] = q.x & 0x7FFFFFFFu; b[1] = q.y & 0x7FFFFFFFu; b[2] = q.z & 0x7FFFFFFFu; b[3] = q.w & 0x7FFFFFFFu;
+}
+__device__ __forceinline__ void abs_bits16(const uint4& q, uint32_t (&b)[8], __nv_bfloat16) {
+    b[0] = (q.x << 16) & 0x7FFFFFFFu; b[1] = q.x & 0x7FFF0000u; b[2] = (q.y << 16) & 0x7FFFFFFFu; b[3] = q.y & 0x7FFF0000u;
+    b[4] = (q.z << 16) & 0x7FFFFFFFu; b[5] = q.z & 0x7FFF0000u; b[6] = (q.w << 16) & 0x7FFFFFFFu; b[7] = q.w & 0x7FFF0000u;
+}
+// Largest absolute-value bit pattern of the group (binary32 pattern in both cases).
+__device__ __forceinline__ uint32_t abs_max16(const uint4& q, float) {
+    return max(max(q.x & 0x7FFFFFFFu, q.y & 0x7FFFFFFFu), max(q.z & 0x7FFFFFFFu, q.w & 0x7FFFFFFFu));
+}
+__device__ __forceinline__ uint32_t abs_max16(const uint4& q, __nv_bfloat16) {
+    // two bfloat16 per word: packed 16-bit maxima, then the larger half widened
+    const uint32_t m = __vmaxu2(__vmaxu2(q.x & 0x7FFF7FFFu, q.y & 0x7FFF7FFFu), __vmaxu2(q.z & 0x7FFF7FFFu, q.w & 0x7FFF7FFFu));
+    return max(m << 16, m & 0xFFFF0000u);
+}
 
 // ROWS: one word per row wanted; COLS: one word per column wanted; neither: one word for the tensor.
-// Two rows (eight 16-byte loads per thread) are in flight at a time.
+// A CTA covers 64 rows x (32 lanes x 2 groups x 16 bytes); four rows (eight 16-byte loads per thread)
+// are in flight at a time.  vec_ok: base and pitch allow 16-byte loads.
 template <typename T, bool ROWS, bool COLS>
-__global__ void __launch_bounds__(AMAX_THREADS)
+__global__ void __launch_bounds__(AMAX_THREADS, COLS ? 3 : 4)
 amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok,
             uint32_t* __restrict__ amax_rm, uint32_t* __restrict__ amax_tr) {
-    __shared__ uint32_t col_max[COLS ? AMAX_TILE_C : 1];
+    constexpr int EPL = 16 / (int)sizeof(T);                   // elements per 16-byte group
+    constexpr int TILE_C = 32 * AMAX_GROUPS * EPL;
+    __shared__ uint32_t col_max[COLS ? TILE_C : 1];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t n_tc = (cols + AMAX_TILE_C - 1) / AMAX_TILE_C;
-    const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * AMAX_TILE_C;
+    const int64_t n_tc = (cols + TILE_C - 1) / TILE_C;
+    const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * TILE_C;
     const int64_t r0 = ((int64_t)blockIdx.x / n_tc) * AMAX_TILE_R;
     if constexpr (COLS) {
-        for (int i = threadIdx.x; i < AMAX_TILE_C; i += AMAX_THREADS) col_max[i] = 0u;
+        for (int i = threadIdx.x; i < TILE_C; i += AMAX_THREADS) col_max[i] = 0u;
         __syncthreads();
     }
-    uint32_t cm[COLS ? 16 : 1];
+    uint32_t cm[COLS ? AMAX_GROUPS * EPL : 1];
 #pragma unroll
-    for (int i = 0; i < (COLS ? 16 : 1); ++i) cm[i] = 0u;
+    for (int i = 0; i < (COLS ? AMAX_GROUPS * EPL : 1); ++i) cm[i] = 0u;
     uint32_t all = 0u;
 #pragma unroll 1
-    for (int rr = 0; rr < AMAX_TILE_R / 8; rr += 2) {
-        float v[2][4][4];
+    for (int rr = 0; rr < AMAX_TILE_R / 8; rr += 4) {
+        uint4 v[4][AMAX_GROUPS];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < 4; ++h) {
             const int64_t r = r0 + warp + 8 * (rr + h);
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                const int64_t c = c0 + (int64_t)(g * 32 + lane) * 4;
-                if (r < rows && c < cols) load4(x + r * ld, c, cols, vec_ok, v[h][g]);
-                else { v[h][g][0] = v[h][g][1] = v[h][g][2] = v[h][g][3] = 0.0f; }
+            for (int g = 0; g < AMAX_GROUPS; ++g) {
+                const int64_t c = c0 + (int64_t)(g * 32 + lane) * EPL;
+                v[h][g] = make_uint4(0u, 0u, 0u, 0u);
+                if (r < rows && c < cols) {
+                    const T* src = x + r * ld + c;
+                    if (vec_ok && c + EPL <= cols) {
+                        v[h][g] = __ldcs(reinterpret_cast<const uint4*>(src));
+                    } else {                                       // ragged or unaligned: element by element
+                        T tmp[EPL];
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) tmp[e] = (c + e < cols) ? src[e] : T(0.0f);
+                        memcpy(&v[h][g], tmp, 16);
+                    }
+                }
             }
         }
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < 4; ++h) {
             const int64_t r = r0 + warp + 8 * (rr + h);
             uint32_t rmax = 0u;
 #pragma unroll
-            for (int g = 0; g < 4; ++g)
+            for (int g = 0; g < AMAX_GROUPS; ++g) {
+                if constexpr (COLS) {
+                    uint32_t b[EPL];
+                    abs_bits16(v[h][g], b, T());
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const uint32_t b = abs_bits(v[h][g][e]);
-                    rmax = max(rmax, b);
-                    if constexpr (COLS) cm[g * 4 + e] = max(cm[g * 4 + e], b);
+                    for (int e = 0; e < EPL; ++e) { rmax = max(rmax, b[e]); cm[g * EPL + e] = max(cm[g * EPL + e], b[e]); }
+                } else {
+                    rmax = max(rmax, abs_max16(v[h][g], T()));
                 }
+            }
             if constexpr (ROWS) {
                 rmax = __reduce_max_sync(0xFFFFFFFFu, rmax);
                 if (lane == 0 && rmax && r < rows) atomicMax(&amax_rm[r], rmax);
@@ -134,17 +168,26 @@ amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, boo
         }
     }
     if constexpr (!ROWS && !COLS) {
+        // one word for the whole tensor: combine the CTA first, and only touch the word when this
+        // CTA can raise it (atomics on one address are serialised by the memory system)
+        __shared__ uint32_t warp_max[AMAX_THREADS / 32];
         all = __reduce_max_sync(0xFFFFFFFFu, all);
-        if (lane == 0 && all) atomicMax(&amax_rm[0], all);
+        if (lane == 0) warp_max[warp] = all;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int w = 1; w < AMAX_THREADS / 32; ++w) all = max(all, warp_max[w]);
+            if (all > __ldcg(&amax_rm[0])) atomicMax(&amax_rm[0], all);
+        }
     }
     if constexpr (COLS) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g)
+        for (int g = 0; g < AMAX_GROUPS; ++g)
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (cm[g * 4 + e]) atomicMax(&col_max[(g * 32 + lane) * 4 + e], cm[g * 4 + e]);
+            for (int e = 0; e < EPL; ++e)
+                if (cm[g * EPL + e]) atomicMax(&col_max[(g * 32 + lane) * EPL + e], cm[g * EPL + e]);
         __syncthreads();
-        for (int i = threadIdx.x; i < AMAX_TILE_C; i += AMAX_THREADS) {
+        for (int i = threadIdx.x; i < TILE_C; i += AMAX_THREADS) {
             const int64_t c = c0 + i;
             if (c < cols && col_max[i]) atomicMax(&amax_tr[c], col_max[i]);
         }
@@ -152,9 +195,12 @@ amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, boo
 }
 
 template <typename T>
-static void launch_amax(const void* x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok, uint32_t* amax_rm, bool want_rows,
-                        uint32_t* amax_tr, bool want_cols, unsigned grid, cudaStream_t st) {
+static void launch_amax(const void* x, int64_t rows, int64_t cols, int64_t ld, uint32_t* amax_rm, bool want_rows,
+                        uint32_t* amax_tr, bool want_cols, cudaStream_t st) {
     const T* p = (const T*)x;
+    constexpr int tile_c = 32 * AMAX_GROUPS * (16 / (int)sizeof(T));
+    const unsigned grid = (unsigned)(((cols + tile_c - 1) / tile_c) * ((rows + AMAX_TILE_R - 1) / AMAX_TILE_R));
+    const bool vec_ok = ((uintptr_t)x % 16 == 0) && ((ld * (int64_t)sizeof(T)) % 16 == 0);
     if (want_rows && want_cols) amax_kernel<T, true, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
     else if (want_rows) amax_kernel<T, true, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
     else if (want_cols) amax_kernel<T, false, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
@@ -551,10 +597,9 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
 
     const bool vec_in = ((uintptr_t)a.x % (4 * esize) == 0) && (a.ld % 4 == 0);
     {
-        const unsigned grid = (unsigned)(((cols + AMAX_TILE_C - 1) / AMAX_TILE_C) * ((rows + AMAX_TILE_R - 1) / AMAX_TILE_R));
         const bool want_rows = per_row && want_rm, want_cols = per_row && want_tr;
-        if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, vec_in, amax_rm, want_rows, amax_tr, want_cols, grid, stream);
-        else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, vec_in, amax_rm, want_rows, amax_tr, want_cols, grid, stream);
+        if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, stream);
+        else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, stream);
         ++g_launches;
     }
     {
