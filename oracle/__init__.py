@@ -93,6 +93,17 @@ def lib() -> ctypes.CDLL:
         for name in ("orc_qlinear_fwd", "orc_qlinear_bwd_input", "orc_qlinear_bwd_weight"):
             getattr(L, name).argtypes = [vp, vp, i64, i64, i64, qp, qp, vp, vp, vp, vp, vp, vp]
             getattr(L, name).restype = i64
+        L.orc_e4m3_decode.argtypes = [ctypes.c_uint8]
+        L.orc_e4m3_decode.restype = ctypes.c_double
+        L.orc_quantize_e4m3_scalar.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_int, ctypes.c_uint32]
+        L.orc_quantize_e4m3_scalar.restype = ctypes.c_uint8
+        L.orc_scale_e4m3.argtypes = [ctypes.c_float, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+        L.orc_scale_e4m3.restype = None
+        L.orc_sr_quantize_e4m3.argtypes = [vp, i64, i64, i64, ctypes.c_int, ctypes.c_int,
+                                           ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
+        L.orc_sr_quantize_e4m3.restype = ctypes.c_int
+        L.orc_gemm_e4m3_nt.argtypes = [vp, vp, i64, i64, i64, vp, ctypes.c_int, vp, ctypes.c_int, vp, vp]
+        L.orc_gemm_e4m3_nt.restype = None
         L.orc_num_threads.argtypes = []
         L.orc_num_threads.restype = ctypes.c_int
     return _lib
@@ -249,3 +260,78 @@ def qlinear_bwd_weight(dY, A, qdy: QSpec, qa: QSpec) -> LinearResult:
     T2, K = A.shape
     assert T == T2
     return _qlinear(lib().orc_qlinear_bwd_weight, dY, A, T, N, K, qdy, qa, (N, T), (K, T), (N, K))
+
+
+# ---------------------------------------------------------------------------------------------
+# E4M3 grid
+# ---------------------------------------------------------------------------------------------
+def e4m3_decode(codes) -> np.ndarray:
+    """Values (binary64) of E4M3 code bytes."""
+    table = np.array([lib().orc_e4m3_decode(i) for i in range(256)], dtype=np.float64)
+    return table[np.asarray(codes, dtype=np.uint8)]
+
+
+def scale_e4m3(m: float):
+    d, inv = ctypes.c_float(), ctypes.c_float()
+    lib().orc_scale_e4m3(ctypes.c_float(m), ctypes.byref(d), ctypes.byref(inv))
+    return np.float32(d.value), np.float32(inv.value)
+
+
+def quantize_e4m3_scalar(x: float, inv: float, round_mode: int, u24: int = 0) -> int:
+    return int(lib().orc_quantize_e4m3_scalar(ctypes.c_float(x), ctypes.c_float(inv), round_mode, u24))
+
+
+def sr_quantize_e4m3(x, q: QSpec, want_rm: bool = True, want_tr: bool = False):
+    """Def. 1-3 on the E4M3 grid (q.bits is ignored); returns (codes_rm, scale_rm, codes_tr, scale_tr)."""
+    x = _f32_2d(x)
+    rows, cols = x.shape
+    ld = x.strides[0] // 4
+    per_row = q.scale_mode == PER_ROW
+    crm = srm = ctr = strr = None
+    if want_rm:
+        crm = np.zeros((rows, cols), dtype=np.uint8)
+        srm = np.zeros(rows if per_row else 1, dtype=np.float32)
+    if want_tr:
+        ctr = np.zeros((cols, rows), dtype=np.uint8)
+        strr = np.zeros(cols if per_row else 1, dtype=np.float32)
+    lib().orc_sr_quantize_e4m3(_ptr(x), rows, cols, ld, q.scale_mode, q.round_mode, q.seed, q.tensor_id,
+                               q.index_offset, _ptr(crm), _ptr(srm), _ptr(ctr), _ptr(strr))
+    return crm, srm, ctr, strr
+
+
+def gemm_e4m3_nt(a, b, s_row, s_col):
+    """(acc, out) in binary64: acc[i,j] = sum_k val(a[i,k]) val(b[j,k]), out = acc * (s_row x s_col)."""
+    a = np.ascontiguousarray(a, dtype=np.uint8)
+    b = np.ascontiguousarray(b, dtype=np.uint8)
+    s_row = np.ascontiguousarray(s_row, dtype=np.float32)
+    s_col = np.ascontiguousarray(s_col, dtype=np.float32)
+    M, Kc = a.shape
+    N, Kb = b.shape
+    assert Kc == Kb and s_row.size in (1, M) and s_col.size in (1, N)
+    acc = np.zeros((M, N), dtype=np.float64)
+    out = np.zeros((M, N), dtype=np.float64)
+    lib().orc_gemm_e4m3_nt(_ptr(a), _ptr(b), M, N, Kc, _ptr(s_row), int(s_row.size != 1),
+                           _ptr(s_col), int(s_col.size != 1), _ptr(acc), _ptr(out))
+    return acc, out
+
+
+def _qlinear_e4m3(X0, X1, q0, q1, tr0, tr1):
+    c0 = sr_quantize_e4m3(X0, q0, not tr0, tr0)
+    c1 = sr_quantize_e4m3(X1, q1, not tr1, tr1)
+    ca, sa = (c0[2], c0[3]) if tr0 else (c0[0], c0[1])
+    cb, sb = (c1[2], c1[3]) if tr1 else (c1[0], c1[1])
+    acc, out = gemm_e4m3_nt(ca, cb, sa, sb)
+    return LinearResult(out, acc, ca, sa, cb, sb)
+
+
+def qlinear_fwd_e4m3(A, W, qa: QSpec, qw: QSpec) -> LinearResult:
+    """Alg. 1 on the E4M3 grid: Y = Q(A) Q(W)^T (out and acc in binary64)."""
+    return _qlinear_e4m3(A, W, qa, qw, False, False)
+
+
+def qlinear_bwd_input_e4m3(dY, W, qdy: QSpec, qw: QSpec) -> LinearResult:
+    return _qlinear_e4m3(dY, W, qdy, qw, False, True)
+
+
+def qlinear_bwd_weight_e4m3(dY, A, qdy: QSpec, qa: QSpec) -> LinearResult:
+    return _qlinear_e4m3(dY, A, qdy, qa, True, True)

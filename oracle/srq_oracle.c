@@ -421,3 +421,156 @@ int orc_num_threads(void)
     return 1;
 #endif
 }
+
+/* ====================================================================== */
+/* E4M3 grid (the 8-bit floating-point formats of the paper's experiments  */
+/* section are E4M0 / E4M1 / E4M2; E4M3 is the member of that family the    */
+/* tensor cores multiply natively).  Format: 1 sign bit, 4 exponent bits    */
+/* with bias 7, 3 mantissa bits, subnormals at exponent field 0, no         */
+/* infinities, largest finite value 448 (exponent field 15, mantissa 6).    */
+/* ====================================================================== */
+
+/* Value of an E4M3 code byte, written out from the format's definition.
+ * The two NaN codes (0x7f, 0xff) return NaN. */
+double orc_e4m3_decode(uint8_t code)
+{
+    int sign = code >> 7, ex = (code >> 3) & 15, man = code & 7;
+    double v;
+    if (ex == 15 && man == 7) return NAN;
+    if (ex == 0) v = ldexp((double)man, -9);            /* subnormal: man/8 * 2^-6 */
+    else v = ldexp(1.0 + man / 8.0, ex - 7);
+    return sign ? -v : v;
+}
+
+/* Code byte of a value that lies on the E4M3 grid (|v| <= 448); zero is +0. */
+static uint8_t orc_e4m3_encode_on_grid(double v)
+{
+    if (v == 0.0) return 0;
+    uint8_t sign = v < 0 ? 0x80 : 0;
+    double a = fabs(v);
+    int ex2;
+    double m = frexp(a, &ex2);          /* a = m 2^ex2, m in [0.5, 1) */
+    int e = ex2 - 1;                    /* a in [2^e, 2^(e+1)) */
+    if (e < -6) return (uint8_t)(sign | (int)ldexp(a, 9));            /* subnormal: a / 2^-9 */
+    int man = (int)ldexp(m, 4) - 8;                                   /* (a / 2^e - 1) * 8 */
+    return (uint8_t)(sign | ((e + 7) << 3) | man);
+}
+
+/*
+ * Def. 1 on the E4M3 grid.  The grid is uniform inside each binade, so the
+ * precision level of Def. 1 is taken locally: for t = x * inv with
+ * 2^e <= |t| < 2^(e+1) (e clamped to [-6, 8]; below 2^-6 the subnormal spacing
+ * continues) the step is D = 2^(e-3), and Q_D(t, eps) = D floor(t/D) if
+ * frac(t/D) < eps... i.e. exactly the rule of orc_quantize_scalar applied to
+ * u = t / D: round up (toward +infinity) iff eps < frac(u) for SR, iff
+ * frac(u) >= 1/2 for RTN.  Both neighbours D floor(u) and D (floor(u) + 1) are
+ * E4M3 values (a binade's upper end is the next binade's first value).
+ * Scaling by D is exact, and the comparison is evaluated in binary64 where
+ * every term is exact.  Returns the code byte.
+ */
+uint8_t orc_quantize_e4m3_scalar(float x, float inv, int round_mode, uint32_t u24)
+{
+    float t = x * inv;
+    double td = (double)t, a = fabs(td);
+    if (a == 0.0) return 0;
+    int ex2;
+    (void)frexp(a, &ex2);
+    int e = ex2 - 1;
+    if (e < -6) e = -6;
+    if (e > 8) e = 8;
+    double u = ldexp(td, 3 - e);                 /* t / D, exact */
+    double f = floor(u);
+    int up;
+    if (round_mode == ORC_SR)
+        up = ((double)u24 + f * 0x1p24) < u * 0x1p24;
+    else
+        up = (f * 0x1p24 + 0x1p23) <= u * 0x1p24;
+    double v = ldexp(f + up, e - 3);
+    if (v > 448.0) v = 448.0;                    /* unreachable with inv from orc_scale_e4m3 */
+    if (v < -448.0) v = -448.0;
+    return orc_e4m3_encode_on_grid(v);
+}
+
+/* Step size D = m / 448 (round to nearest) and the reciprocal multiplied in,
+ * 448 / m rounded toward zero, so that |x * inv| <= 448 for the whole group
+ * (same reasoning as orc_scale_from_absmax). */
+void orc_scale_e4m3(float m, float *delta, float *inv)
+{
+    float r = (m == 0.0f) ? 0.0f : 448.0f / m;
+    if (isinf(r) || r != r) r = 0.0f;
+    if (r != 0.0f && (double)r * (double)m > 448.0) r = nextafterf(r, 0.0f);
+    *inv = r;
+    *delta = (r == 0.0f) ? 0.0f : m / 448.0f;
+}
+
+/*
+ * Matrix form, same conventions as orc_sr_quantize (two layouts, per-tensor
+ * or per-row step sizes, one threshold per element by flat source index);
+ * codes are E4M3 bytes.
+ */
+int orc_sr_quantize_e4m3(const float *x, int64_t rows, int64_t cols, int64_t ld,
+                         int scale_mode, int round_mode,
+                         uint64_t seed, uint64_t tensor_id, uint64_t index_offset,
+                         uint8_t *codes_rm, float *scale_rm,
+                         uint8_t *codes_tr, float *scale_tr)
+{
+    float m_tensor = 0.0f;
+    if (scale_mode == ORC_PER_TENSOR) orc_absmax_tensor(x, rows, cols, ld, &m_tensor);
+    if (codes_rm) {
+        if (scale_mode == ORC_PER_ROW) orc_absmax_rows(x, rows, cols, ld, scale_rm);
+#pragma omp parallel for schedule(static)
+        for (int64_t r = 0; r < rows; ++r) {
+            float delta, inv;
+            orc_scale_e4m3(scale_mode == ORC_PER_TENSOR ? m_tensor : scale_rm[r], &delta, &inv);
+            if (scale_mode == ORC_PER_ROW) scale_rm[r] = delta;
+            else if (r == 0) scale_rm[0] = delta;
+            for (int64_t c = 0; c < cols; ++c) {
+                uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
+                uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, i) : 0u;
+                codes_rm[r * cols + c] = orc_quantize_e4m3_scalar(x[r * ld + c], inv, round_mode, u24);
+            }
+        }
+        if (scale_mode == ORC_PER_TENSOR && rows == 0) { float d, iv; orc_scale_e4m3(m_tensor, &d, &iv); scale_rm[0] = d; }
+    }
+    if (codes_tr) {
+        if (scale_mode == ORC_PER_ROW) orc_absmax_cols(x, rows, cols, ld, scale_tr);
+#pragma omp parallel for schedule(static)
+        for (int64_t c = 0; c < cols; ++c) {
+            float delta, inv;
+            orc_scale_e4m3(scale_mode == ORC_PER_TENSOR ? m_tensor : scale_tr[c], &delta, &inv);
+            if (scale_mode == ORC_PER_ROW) scale_tr[c] = delta;
+            else if (c == 0) scale_tr[0] = delta;
+            for (int64_t r = 0; r < rows; ++r) {
+                uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
+                uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, i) : 0u;
+                codes_tr[c * rows + r] = orc_quantize_e4m3_scalar(x[r * ld + c], inv, round_mode, u24);
+            }
+        }
+    }
+    return 0;
+}
+
+/*
+ * Sec. 2.2.2 for E4M3 codes: acc[i,j] = sum_k val(a[i,k]) val(b[j,k]) with the
+ * sum formed in binary64.  Every product of two E4M3 values is exact in
+ * binary64 (8 significant bits), and the partial sums of the lengths used here
+ * stay exact as well (all terms are multiples of 2^-18 below 2^18 each), so
+ * this is the exact product of the two quantized matrices.
+ * out[i,j] = acc[i,j] * (s_row[i] * s_col[j]), the scale product one binary32
+ * multiply, the rest binary64.
+ */
+void orc_gemm_e4m3_nt(const uint8_t *a, const uint8_t *b, int64_t M, int64_t N, int64_t Kc,
+                      const float *s_row, int row_stride, const float *s_col, int col_stride,
+                      double *acc, double *out)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            double s = 0.0;
+            for (int64_t k = 0; k < Kc; ++k)
+                s += orc_e4m3_decode(a[i * Kc + k]) * orc_e4m3_decode(b[j * Kc + k]);
+            acc[i * N + j] = s;
+            float sc = s_row[i * row_stride] * s_col[j * col_stride];
+            out[i * N + j] = s * (double)sc;
+        }
+}
