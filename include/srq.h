@@ -26,6 +26,10 @@
  *     recorded in a status word at the start of the workspace; read it with
  *     srq_poll_status.  After such a condition the outputs are unspecified.
  *   - Outputs are overwritten, never accumulated into.
+ *   - Both operands of a layer pass use the same grid (srq_qspec_t.format).  With the E4M3
+ *     grid the codes are E4M3 bytes, D_g = absmax_g / 448, the products run in kind::f8f6f4
+ *     with binary32 accumulation, and the `acc` member of the debug struct receives binary32
+ *     sums (same size as int32).
  *   - Alignment: input base pointers 16-byte aligned; input pitch `ld` in
  *     elements; fp32 outputs 16-byte aligned; the workspace 256-byte aligned.
  *     Inputs whose pitch or extent is not a multiple of 4 elements take a
@@ -71,6 +75,10 @@ typedef enum {
 typedef enum { SRQ_F32 = 0, SRQ_BF16 = 1 } srq_dtype_t;
 typedef enum { SRQ_PER_TENSOR = 0, SRQ_PER_ROW = 1 } srq_scale_t;
 typedef enum { SRQ_SR = 0, SRQ_RTN = 1 } srq_round_t;
+/* Grid of a quantization point: integers times the step size (bits 2..8), or the E4M3 8-bit
+ * floating-point values times the step size (1 sign, 4 exponent, 3 mantissa bits, bias 7, no
+ * infinities, largest value 448; `bits` is ignored). */
+typedef enum { SRQ_GRID_INT = 0, SRQ_GRID_E4M3 = 1 } srq_grid_t;
 
 /* One quantization point: the paper's (D, eps) pair for one operand of one pass
  * (five per layer: A and W forward; A, W and dY backward). */
@@ -78,7 +86,7 @@ typedef struct {
     int32_t bits;          /* 2..8; codes are stored one per int8 whatever the width */
     int32_t scale;         /* srq_scale_t */
     int32_t round;         /* srq_round_t */
-    int32_t reserved;      /* 0 */
+    int32_t format;        /* srq_grid_t; 0 = integer grid */
     uint64_t seed;         /* Philox key; one per training step */
     uint64_t tensor_id;    /* Philox counter words 2-3; one per (layer, operand, pass) */
     uint64_t index_offset; /* added to the flat index; first_row*cols for a row shard */
@@ -163,6 +171,22 @@ srq_status_t srq_gemm_i8(const int8_t *a, int64_t lda, const int8_t *b, int64_t 
                          const float *s_col, int32_t col_stride,
                          float *out, int64_t ldo, int32_t *acc_out,
                          void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * The same product for E4M3 codes (the 8-bit floating-point grid; the paper's experiments use
+ * the E4M0 / E4M1 / E4M2 members of this family): a[M, Kc], b[N, Kc] are E4M3 bytes, multiplied
+ * on the tensor cores (kind::f8f6f4) with binary32 accumulation, whose summation order is the
+ * hardware's, so results agree with the exact product to about 1e-5 * |row| * |col| rather than
+ * bit for bit.  out[i, j] = acc[i, j] * (s_row[i] * s_col[j]); acc_out, if not NULL, receives
+ * the raw binary32 sums [M, N].  Alignment rules as for srq_gemm_i8; the contraction is never
+ * split, so the workspace only needs its 256-byte header.
+ */
+srq_status_t srq_gemm_e4m3(const uint8_t *a, int64_t lda, const uint8_t *b, int64_t ldb,
+                           int64_t M, int64_t N, int64_t Kc,
+                           const float *s_row, int32_t row_stride,
+                           const float *s_col, int32_t col_stride,
+                           float *out, int64_t ldo, float *acc_out,
+                           void *ws, size_t ws_bytes, void *cuda_stream);
 
 /* Alg. 1: Y[T,N] = Q(A) Q(W)^T.  qA, qW are the forward quantization points of A and W.
  * Per row: A per token, W per output feature. */

@@ -23,9 +23,10 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_ACC_OVERFLOW, ERR_CUDA,
 F32, BF16 = 0, 1
 PER_TENSOR, PER_ROW = 0, 1
 SR, RTN = 0, 1
+GRID_INT, GRID_E4M3 = 0, 1
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
-           "sr_quantize", "sr_quantize_static", "srq_gemm_i8", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
+           "sr_quantize", "sr_quantize_static", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
            "srq_poll_status", "srq_status_string", "srq_launch_count"]
 
 
@@ -37,7 +38,7 @@ class SrqError(RuntimeError):
 
 class _QSpec(ctypes.Structure):
     _fields_ = [("bits", ctypes.c_int32), ("scale", ctypes.c_int32), ("round", ctypes.c_int32),
-                ("reserved", ctypes.c_int32), ("seed", ctypes.c_uint64),
+                ("format", ctypes.c_int32), ("seed", ctypes.c_uint64),
                 ("tensor_id", ctypes.c_uint64), ("index_offset", ctypes.c_uint64)]
 
 
@@ -49,16 +50,17 @@ class _DebugOut(ctypes.Structure):
 
 @dataclass
 class QSpec:
-    """One quantization point (bits, scale mode, rounding mode, seed, tensor_id, index_offset)."""
+    """One quantization point (bits, scale mode, rounding mode, seed, tensor_id, index_offset, grid)."""
     bits: int = 8
     scale: int = PER_TENSOR
     round: int = SR
     seed: int = 0
     tensor_id: int = 0
     index_offset: int = 0
+    format: int = GRID_INT
 
     def c(self) -> _QSpec:
-        return _QSpec(self.bits, self.scale, self.round, 0, self.seed, self.tensor_id,
+        return _QSpec(self.bits, self.scale, self.round, self.format, self.seed, self.tensor_id,
                       self.index_offset)
 
 
@@ -89,6 +91,8 @@ def lib() -> ctypes.CDLL:
     L.sr_quantize_static.restype = ctypes.c_int
     L.srq_gemm_i8.argtypes = [vp, i64, vp, i64, i64, i64, i64, vp, i32, vp, i32, vp, i64, vp, vp, sz, vp]
     L.srq_gemm_i8.restype = ctypes.c_int
+    L.srq_gemm_e4m3.argtypes = L.srq_gemm_i8.argtypes
+    L.srq_gemm_e4m3.restype = ctypes.c_int
     for name in ("qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight"):
         f = getattr(L, name)
         f.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, qp, qp, vp, dp, vp, sz, vp]
@@ -207,6 +211,23 @@ def srq_gemm_i8(a: torch.Tensor, b: torch.Tensor, s_row: torch.Tensor, s_col: to
                            int(s_col.numel() != 1), out.data_ptr(), out.stride(0), _ptr(acc_out),
                            ws.data_ptr(), ws.numel(), _stream())
     _check(st, "srq_gemm_i8")
+
+
+def srq_gemm_e4m3(a: torch.Tensor, b: torch.Tensor, s_row: torch.Tensor, s_col: torch.Tensor,
+                  out: torch.Tensor, acc_out: Optional[torch.Tensor] = None,
+                  ws: Optional[torch.Tensor] = None) -> None:
+    """srq_gemm_i8 for E4M3 code bytes (uint8 tensors); acc_out, if given, is float32 [M, N]."""
+    _dev2d(a, "a")
+    _dev2d(b, "b")
+    M, Kc = a.shape
+    N = b.shape[0]
+    if ws is None:
+        ws = new_workspace(256, a.device)
+    st = lib().srq_gemm_e4m3(a.data_ptr(), a.stride(0), b.data_ptr(), b.stride(0), M, N, Kc,
+                             s_row.data_ptr(), int(s_row.numel() != 1), s_col.data_ptr(),
+                             int(s_col.numel() != 1), out.data_ptr(), out.stride(0), _ptr(acc_out),
+                             ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "srq_gemm_e4m3")
 
 
 @dataclass

@@ -49,7 +49,8 @@ def case_quantize(a):
     dt = torch.float32 if a.dtype == "f32" else torch.bfloat16
     x = synth.with_outliers((a.rows, a.cols), a.seed, dt, "cuda")
     per_row = a.scale == "row"
-    q = B.QSpec(a.bits, B.PER_ROW if per_row else B.PER_TENSOR, B.SR if a.round == "sr" else B.RTN, a.seed, 1)
+    q = B.QSpec(a.bits, B.PER_ROW if per_row else B.PER_TENSOR, B.SR if a.round == "sr" else B.RTN, a.seed, 1,
+                0, B.GRID_E4M3 if getattr(a, "grid", "int") == "e4m3" else B.GRID_INT)
     rm, tr = a.layouts in ("rm", "both"), a.layouts in ("tr", "both")
     crm = torch.empty((a.rows, a.cols), dtype=torch.int8, device="cuda") if rm else None
     ctr = torch.empty((a.cols, a.rows), dtype=torch.int8, device="cuda") if tr else None
@@ -63,7 +64,7 @@ def case_quantize(a):
     assert B.srq_poll_status(ws) == 0
     nbytes = n * (2 * e + int(rm) + int(tr))       # absmax read + quantize read + code layouts written
     return {"op": "sr_quantize", "rows": a.rows, "cols": a.cols, "dtype": a.dtype, "bits": a.bits, "scale": a.scale,
-            "round": a.round, "layouts": a.layouts, "ms": med, "ms_best": best, "algorithmic_bytes": nbytes,
+            "round": a.round, "layouts": a.layouts, "grid": getattr(a, "grid", "int"), "ms": med, "ms_best": best, "algorithmic_bytes": nbytes,
             "GBps": nbytes / med / 1e6}
 
 
@@ -74,12 +75,18 @@ def case_gemm(a):
     one = torch.ones(1, device="cuda")
     out = torch.empty((a.M, a.N), device="cuda")
     ws = B.new_workspace(B.srq_gemm_workspace_bytes(a.M, a.N))
-    fn = lambda: B.srq_gemm_i8(A, Bm, one, one, out, None, ws)
+    if getattr(a, "grid", "int") == "e4m3":
+        A, Bm = A.view(torch.uint8), Bm.view(torch.uint8)
+        A[(A & 0x7F) == 0x7F] = 0x38          # no NaN codes
+        Bm[(Bm & 0x7F) == 0x7F] = 0x38
+        fn = lambda: B.srq_gemm_e4m3(A, Bm, one, one, out, None, ws)
+    else:
+        fn = lambda: B.srq_gemm_i8(A, Bm, one, one, out, None, ws)
     small = (a.M + a.N) * a.K + 4 * a.M * a.N < 2 * L2_BYTES
     med, best = _time(fn, a.iters, a.warmup, flush=small)
     assert B.srq_poll_status(ws) == 0
     ops = 2.0 * a.M * a.N * a.K
-    return {"op": "srq_gemm_i8", "M": a.M, "N": a.N, "K": a.K, "ms": med, "ms_best": best, "TOPS": ops / med / 1e9,
+    return {"op": "srq_gemm_e4m3" if getattr(a, "grid", "int") == "e4m3" else "srq_gemm_i8", "M": a.M, "N": a.N, "K": a.K, "ms": med, "ms_best": best, "TOPS": ops / med / 1e9,
             "out_GBps": 4.0 * a.M * a.N / med / 1e6}
 
 
@@ -90,8 +97,9 @@ def _layer_fn(A, W, dY, q, Y, dA, dW, ws):
     return fn
 
 
-def _layer_specs(bits_fwd, bits_bwd, sc, rd, seed):
-    return {k: B.QSpec(b, sc, rd, seed, i) for i, (k, b) in enumerate(
+def _layer_specs(bits_fwd, bits_bwd, sc, rd, seed, grid="int"):
+    fmt = B.GRID_E4M3 if grid == "e4m3" else B.GRID_INT
+    return {k: B.QSpec(b, sc, rd, seed, i, 0, fmt) for i, (k, b) in enumerate(
         [("a_fwd", bits_fwd), ("w_fwd", bits_fwd), ("a_bwd", bits_bwd), ("w_bwd", bits_bwd), ("dy", bits_bwd)])}
 
 
@@ -100,7 +108,7 @@ def case_layer(a):
     A, W, dY = synth.layer_inputs(a.T, a.N, a.K, a.seed, dt, "cuda", std_dy=1e-3)
     sc = B.PER_ROW if a.scale == "row" else B.PER_TENSOR
     rd = B.SR if a.round == "sr" else B.RTN
-    q = _layer_specs(a.bits_fwd, a.bits_bwd, sc, rd, a.seed)
+    q = _layer_specs(a.bits_fwd, a.bits_bwd, sc, rd, a.seed, getattr(a, "grid", "int"))
     Y = torch.empty((a.T, a.N), device="cuda")
     dA = torch.empty((a.T, a.K), device="cuda")
     dW = torch.empty((a.N, a.K), device="cuda")
@@ -111,7 +119,7 @@ def case_layer(a):
     assert B.srq_poll_status(ws) == 0
     ops = 6.0 * a.T * a.N * a.K
     return {"op": "layer fwd+bwd", "T": a.T, "N": a.N, "K": a.K, "dtype": a.dtype, "bits_fwd": a.bits_fwd,
-            "bits_bwd": a.bits_bwd, "scale": a.scale, "round": a.round, "ms": med, "ms_best": best,
+            "bits_bwd": a.bits_bwd, "scale": a.scale, "round": a.round, "grid": getattr(a, "grid", "int"), "ms": med, "ms_best": best,
             "TOPS": ops / med / 1e9}
 
 
@@ -223,6 +231,7 @@ def main(argv=None):
         p.add_argument("--iters", type=int, default=20)
         p.add_argument("--warmup", type=int, default=3)
         p.add_argument("--seed", type=int, default=0)
+        p.add_argument("--grid", default="int", choices=["int", "e4m3"])
         if name == "quantize":
             p.add_argument("--rows", type=int, default=16384)
             p.add_argument("--cols", type=int, default=4096)

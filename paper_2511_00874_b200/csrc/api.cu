@@ -10,7 +10,8 @@ inline int qmax_of(int bits) { return (1 << (bits - 1)) - 1; }
 
 srq_status_t check_qspec(const srq_qspec_t* q) {
     if (!q) return SRQ_ERR_INVALID_ARG;
-    if (q->bits < 2 || q->bits > 8) return SRQ_ERR_UNSUPPORTED;
+    if (q->format != SRQ_GRID_INT && q->format != SRQ_GRID_E4M3) return SRQ_ERR_INVALID_ARG;
+    if (q->format == SRQ_GRID_INT && (q->bits < 2 || q->bits > 8)) return SRQ_ERR_UNSUPPORTED;
     if (q->scale != SRQ_PER_TENSOR && q->scale != SRQ_PER_ROW) return SRQ_ERR_INVALID_ARG;
     if (q->round != SRQ_SR && q->round != SRQ_RTN) return SRQ_ERR_INVALID_ARG;
     return SRQ_OK;
@@ -63,7 +64,8 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
     if (!aligned_to(a.x, 16) || !aligned_to(b.x, 16) || !aligned_to(out, 16) || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
     const int64_t M = a.out_rows(), Nn = b.out_rows(), Kc = a.out_cols();
     if (Kc != b.out_cols()) return SRQ_ERR_INVALID_ARG;
-    if ((double)Kc * qmax_of(a.q->bits) * qmax_of(b.q->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
+    if (a.q->format != b.q->format) return SRQ_ERR_INVALID_ARG;          // one product, one kind of code
+    if (a.q->format == SRQ_GRID_INT && (double)Kc * qmax_of(a.q->bits) * qmax_of(b.q->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
     const LayerPlan p = plan_layer(a, b);
     if (ws_bytes < p.total) return SRQ_ERR_WORKSPACE;
     if (M == 0 || Nn == 0) return SRQ_OK;
@@ -92,7 +94,7 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
 
     GemmArgs g;
     g.a = codes[0]; g.lda = p.pitch; g.b = codes[1]; g.ldb = p.pitch;
-    g.M = M; g.N = Nn; g.Kc = Kc;
+    g.M = M; g.N = Nn; g.Kc = Kc; g.kind = a.q->format == SRQ_GRID_E4M3;
     g.s_row = scales[0]; g.row_stride = a.q->scale == SRQ_PER_ROW;
     g.s_col = scales[1]; g.col_stride = b.q->scale == SRQ_PER_ROW;
     g.out = out; g.ldo = Nn; g.acc_out = dbg ? dbg->acc : nullptr;
@@ -162,8 +164,10 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
     if ((s = check_qspec(qW)) != SRQ_OK) return s;
     if (!aligned_to(dY, 16) || !aligned_to(A, 16) || !aligned_to(W, 16) || !aligned_to(dA, 16) || !aligned_to(dW, 16) || !aligned_to(ws, 256))
         return SRQ_ERR_INVALID_ARG;
-    if ((double)N * qmax_of(qdY->bits) * qmax_of(qW->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
-    if ((double)T * qmax_of(qdY->bits) * qmax_of(qA->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
+    if (qdY->format != qW->format || qdY->format != qA->format) return SRQ_ERR_INVALID_ARG;
+    const int kind = qdY->format == SRQ_GRID_E4M3;
+    if (!kind && (double)N * qmax_of(qdY->bits) * qmax_of(qW->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
+    if (!kind && (double)T * qmax_of(qdY->bits) * qmax_of(qA->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
     const BwdPlan p = plan_bwd(T, N, K);
     if (ws_bytes < p.total) return SRQ_ERR_WORKSPACE;
 
@@ -198,7 +202,7 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
             if (cudaMemset2DAsync(dA, (size_t)K * 4, 0, (size_t)K * 4, (size_t)T, st) != cudaSuccess) return SRQ_ERR_CUDA;
         } else {
             GemmArgs g;
-            g.a = cd[0]; g.lda = p.pitch_n; g.b = cd[2]; g.ldb = p.pitch_n; g.M = T; g.N = K; g.Kc = N;
+            g.a = cd[0]; g.lda = p.pitch_n; g.b = cd[2]; g.ldb = p.pitch_n; g.M = T; g.N = K; g.Kc = N; g.kind = kind;
             g.s_row = sc[0]; g.row_stride = qdY->scale == SRQ_PER_ROW; g.s_col = sc[2]; g.col_stride = qW->scale == SRQ_PER_ROW;
             g.out = dA; g.ldo = K; g.acc_out = dbg_in ? dbg_in->acc : nullptr;
             g.splitk_ws = base + p.off_split[0]; g.splitk_ws_bytes = p.off_split[1] - p.off_split[0];
@@ -212,7 +216,7 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
             if (cudaMemset2DAsync(dW, (size_t)K * 4, 0, (size_t)K * 4, (size_t)N, st) != cudaSuccess) return SRQ_ERR_CUDA;
         } else {
             GemmArgs g;
-            g.a = cd[1]; g.lda = p.pitch_t; g.b = cd[3]; g.ldb = p.pitch_t; g.M = N; g.N = K; g.Kc = T;
+            g.a = cd[1]; g.lda = p.pitch_t; g.b = cd[3]; g.ldb = p.pitch_t; g.M = N; g.N = K; g.Kc = T; g.kind = kind;
             g.s_row = sc[1]; g.row_stride = qdY->scale == SRQ_PER_ROW; g.s_col = sc[3]; g.col_stride = qA->scale == SRQ_PER_ROW;
             g.out = dW; g.ldo = K; g.acc_out = dbg_w ? dbg_w->acc : nullptr;
             g.splitk_ws = base + p.off_split[1]; g.splitk_ws_bytes = p.total - p.off_split[1];
@@ -290,10 +294,30 @@ srq_status_t srq_gemm_i8(const int8_t* a, int64_t lda, const int8_t* b, int64_t 
     uint32_t* status = &((WsHeader*)ws)->status;
     if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
     GemmArgs g;
-    g.a = a; g.lda = lda; g.b = b; g.ldb = ldb; g.M = M; g.N = N; g.Kc = Kc;
+    g.a = a; g.lda = lda; g.b = b; g.ldb = ldb; g.M = M; g.N = N; g.Kc = Kc; g.kind = 0;
     g.s_row = s_row; g.row_stride = row_stride; g.s_col = s_col; g.col_stride = col_stride;
     g.out = out; g.ldo = ldo; g.acc_out = acc_out;
     g.splitk_ws = (char*)ws + sizeof(WsHeader); g.splitk_ws_bytes = ws_bytes - sizeof(WsHeader);
+    return launch_gemm_i8(g, status, st);
+}
+
+srq_status_t srq_gemm_e4m3(const uint8_t* a, int64_t lda, const uint8_t* b, int64_t ldb, int64_t M, int64_t N, int64_t Kc,
+                           const float* s_row, int32_t row_stride, const float* s_col, int32_t col_stride,
+                           float* out, int64_t ldo, float* acc_out, void* ws, size_t ws_bytes, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!a || !b || !s_row || !s_col || !out || !ws) return SRQ_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || Kc <= 0 || lda < Kc || ldb < Kc || ldo < N) return SRQ_ERR_INVALID_ARG;
+    if ((row_stride != 0 && row_stride != 1) || (col_stride != 0 && col_stride != 1)) return SRQ_ERR_INVALID_ARG;
+    if (!aligned_to(a, 16) || !aligned_to(b, 16) || lda % 16 || ldb % 16 || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
+    if (ws_bytes < sizeof(WsHeader)) return SRQ_ERR_WORKSPACE;
+    if (M == 0 || N == 0) return SRQ_OK;
+    uint32_t* status = &((WsHeader*)ws)->status;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    GemmArgs g;
+    g.a = (const int8_t*)a; g.lda = lda; g.b = (const int8_t*)b; g.ldb = ldb; g.M = M; g.N = N; g.Kc = Kc; g.kind = 1;
+    g.s_row = s_row; g.row_stride = row_stride; g.s_col = s_col; g.col_stride = col_stride;
+    g.out = out; g.ldo = ldo; g.acc_out = (int32_t*)acc_out;       // raw binary32 sums, copied bit for bit
+    g.splitk_ws = nullptr; g.splitk_ws_bytes = 0;
     return launch_gemm_i8(g, status, st);
 }
 

@@ -57,6 +57,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& scratch, uin
 struct GemmArgs {
     const int8_t* a; int64_t lda; const int8_t* b; int64_t ldb;
     int64_t M, N, Kc;
+    int kind;                                   // 0: int8 codes, int32 sums; 1: E4M3 codes, binary32 sums
     const float* s_row; int32_t row_stride; const float* s_col; int32_t col_stride;
     float* out; int64_t ldo; int32_t* acc_out;
     void* splitk_ws; size_t splitk_ws_bytes;   // int32 [M,N] partial sums

@@ -186,21 +186,20 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
     else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem], int8 operands, int32 accumulators, issued by one thread (of the
-// leader CTA when CTAS = 2; the descriptors then address the same offsets in both CTAs).
-template <int CTAS>
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    if constexpr (CTAS == 1) {
-        asm volatile(
-            "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
-            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-    } else {
-        asm volatile(
-            "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n}"
-            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-    }
+// D[tmem] (+)= A[smem] * B[smem], issued by one thread (of the leader CTA when CTAS = 2; the
+// descriptors then address the same offsets in both CTAs).  KIND 0: int8 operands, int32
+// accumulators (kind::i8); KIND 1: E4M3 operands, binary32 accumulators (kind::f8f6f4).
+template <int CTAS, int KIND>
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+#define SRQ_UMMA(GROUP, KINDSTR)                                                                   \
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"                                        \
+                 "tcgen05.mma.cta_group::" GROUP ".kind::" KINDSTR " [%0], %1, %2, %3, p;\n}"        \
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory")
+    if constexpr (CTAS == 1 && KIND == 0) SRQ_UMMA("1", "i8");
+    else if constexpr (CTAS == 2 && KIND == 0) SRQ_UMMA("2", "i8");
+    else if constexpr (CTAS == 1 && KIND == 1) SRQ_UMMA("1", "f8f6f4");
+    else SRQ_UMMA("2", "f8f6f4");
+#undef SRQ_UMMA
 }
 // The mbarrier gets one arrival once every MMA issued so far by this thread has completed.
 // CTAS = 2, both = true: the barrier at the same offset in both CTAs of the pair gets it.
@@ -246,9 +245,19 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
     return d;
 }
 
-// Instruction descriptor: dense, no saturation, D = s32, A = B = s8, both K-major, N x M.
-__device__ __forceinline__ constexpr uint32_t make_idesc_i8(int m, int n) {
-    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+// Instruction descriptor: dense, no saturation, both operands K-major, N x M; KIND 0: D = s32,
+// A = B = s8; KIND 1: D = f32, A = B = E4M3 (format 0).
+__device__ __forceinline__ constexpr uint32_t make_idesc(int kind, int m, int n) {
+    const uint32_t types = kind == 0 ? ((2u << 4) | (1u << 7) | (1u << 10)) : (1u << 4);
+    return types | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// Accumulator word to binary32: an exact int32 -> float conversion for integer codes, the bits
+// themselves for binary32 accumulators.
+template <int KIND>
+__device__ __forceinline__ float acc_to_float(uint32_t v) {
+    if constexpr (KIND == 0) return __int2float_rn((int)v);
+    else return __uint_as_float(v);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -276,7 +285,7 @@ __device__ __forceinline__ void give_up(SharedTail<STAGES>* T, uint32_t* status)
     record_status(status, SRQ_ERR_TIMEOUT);
 }
 
-template <int CTAS>
+template <int CTAS, int KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_part, const GemmParams P) {
@@ -354,7 +363,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && leader) {
-            const uint32_t idesc = make_idesc_i8(BM * CTAS, BN);
+            const uint32_t idesc = make_idesc(KIND, BM * CTAS, BN);
             uint32_t it = 0, lt = 0;
             bool ok = true;
             for (int64_t u = group; u < units && ok; u += groups, ++lt) {
@@ -374,7 +383,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         // advancing K inside the swizzle atom = advancing the start address
-                        umma_i8<CTAS>(d_tmem, da + (uint64_t)((k * UMMA_K) >> 4), db + (uint64_t)((k * UMMA_K) >> 4), idesc,
+                        umma<CTAS, KIND>(d_tmem, da + (uint64_t)((k * UMMA_K) >> 4), db + (uint64_t)((k * UMMA_K) >> 4), idesc,
                                       (kb > kb0 || k > 0) ? 1u : 0u);
                     }
                     umma_commit<CTAS>(&T->empty[s], true);       // stage reusable (in every CTA) once these MMAs have read it
@@ -430,10 +439,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
                         const float4 c4 = *reinterpret_cast<const float4*>(sc + 4 * q);
-                        v[4 * q + 0] = __float_as_uint(__fmul_rn(__int2float_rn((int)v[4 * q + 0]), __fmul_rn(sr, c4.x)));
-                        v[4 * q + 1] = __float_as_uint(__fmul_rn(__int2float_rn((int)v[4 * q + 1]), __fmul_rn(sr, c4.y)));
-                        v[4 * q + 2] = __float_as_uint(__fmul_rn(__int2float_rn((int)v[4 * q + 2]), __fmul_rn(sr, c4.z)));
-                        v[4 * q + 3] = __float_as_uint(__fmul_rn(__int2float_rn((int)v[4 * q + 3]), __fmul_rn(sr, c4.w)));
+                        v[4 * q + 0] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 0]), __fmul_rn(sr, c4.x)));
+                        v[4 * q + 1] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 1]), __fmul_rn(sr, c4.y)));
+                        v[4 * q + 2] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 2]), __fmul_rn(sr, c4.z)));
+                        v[4 * q + 3] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 3]), __fmul_rn(sr, c4.w)));
                     }
                     if (lane == 0) bulk_wait_read();          // the previous block has left the staging buffer
                     __syncwarp();
@@ -461,16 +470,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             for (int q = 0; q < 8; ++q) {
                                 const float4 c4 = *reinterpret_cast<const float4*>(sc + 4 * q);
                                 float4 o;
-                                o.x = __fmul_rn(__int2float_rn((int)v[4 * q + 0]), __fmul_rn(sr, c4.x));
-                                o.y = __fmul_rn(__int2float_rn((int)v[4 * q + 1]), __fmul_rn(sr, c4.y));
-                                o.z = __fmul_rn(__int2float_rn((int)v[4 * q + 2]), __fmul_rn(sr, c4.z));
-                                o.w = __fmul_rn(__int2float_rn((int)v[4 * q + 3]), __fmul_rn(sr, c4.w));
+                                o.x = __fmul_rn(acc_to_float<KIND>(v[4 * q + 0]), __fmul_rn(sr, c4.x));
+                                o.y = __fmul_rn(acc_to_float<KIND>(v[4 * q + 1]), __fmul_rn(sr, c4.y));
+                                o.z = __fmul_rn(acc_to_float<KIND>(v[4 * q + 2]), __fmul_rn(sr, c4.z));
+                                o.w = __fmul_rn(acc_to_float<KIND>(v[4 * q + 3]), __fmul_rn(sr, c4.w));
                                 __stcs(reinterpret_cast<float4*>(dst + 4 * q), o);
                             }
                         } else {
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
-                                if (col0 + i < P.N) dst[i] = __fmul_rn(__int2float_rn((int)v[i]), __fmul_rn(sr, sc[i]));
+                                if (col0 + i < P.N) dst[i] = __fmul_rn(acc_to_float<KIND>(v[i]), __fmul_rn(sr, sc[i]));
                         }
                         if (P.acc_out) {
                             int32_t* ad = P.acc_out + row * P.N + col0;
@@ -610,15 +619,17 @@ static bool device_info(DeviceInfo** out) {
     DeviceInfo& d = info[dev];
     if (!d.ready) {
         if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || d.sms <= 0) return false;
-        if (cudaFuncSetAttribute(gemm_i8_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<1>()) != cudaSuccess) return false;
-        if (cudaFuncSetAttribute(gemm_i8_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<2>()) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_i8_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<1>()) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_i8_kernel<2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<2>()) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_i8_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<1>()) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_i8_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<2>()) != cudaSuccess) return false;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(d.sms / 2 * 2)); cfg.blockDim = dim3(GEMM_THREADS); cfg.dynamicSmemBytes = gemm_smem<2>();
         cudaLaunchAttribute at;
         at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
         cfg.attrs = &at; cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<2>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<2, 0>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
         d.pairs = n < d.sms / 2 ? n : d.sms / 2;
         d.ready = true;
     }
@@ -648,7 +659,7 @@ size_t gemm_splitk_bytes(int64_t M, int64_t N) {
     return align_up((size_t)M * N * 4);
 }
 
-template <int CTAS>
+template <int CTAS, int KIND>
 static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out,
                                  const CUtensorMap& map_part, const GemmParams& P, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
@@ -657,7 +668,7 @@ static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, cons
     cudaLaunchAttribute at;
     at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = CTAS; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
     cfg.attrs = &at; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_i8_kernel<CTAS>, map_a, map_b, map_out, map_part, P);
+    return cudaLaunchKernelEx(&cfg, gemm_i8_kernel<CTAS, KIND>, map_a, map_b, map_out, map_part, P);
 }
 
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream) {
@@ -677,7 +688,8 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.tiles_m = (int32_t)((g.M + BM * ctas - 1) / (BM * ctas));
     P.tiles_n = (int32_t)((g.N + BN - 1) / BN);
     const int64_t tiles = (int64_t)P.tiles_m * P.tiles_n;
-    P.splits = choose_splits(tiles, P.num_kb, groups_max);
+    // binary32 accumulators do not add exactly: the E4M3 product is never split
+    P.splits = g.kind == 0 ? choose_splits(tiles, P.num_kb, groups_max) : 1;
     P.part = nullptr;
     if (P.splits > 1) {
         const size_t part_bytes = align_up((size_t)g.M * g.N * 4);
@@ -703,8 +715,11 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
 
     const int64_t units = tiles * P.splits;
     const unsigned groups = (unsigned)(units < groups_max ? units : groups_max);
-    const cudaError_t e = ctas == 2 ? launch_kernel<2>(groups, map_a, map_b, map_out, map_part, P, stream)
-                                    : launch_kernel<1>(groups, map_a, map_b, map_out, map_part, P, stream);
+    cudaError_t e;
+    if (g.kind == 0) e = ctas == 2 ? launch_kernel<2, 0>(groups, map_a, map_b, map_out, map_part, P, stream)
+                                   : launch_kernel<1, 0>(groups, map_a, map_b, map_out, map_part, P, stream);
+    else e = ctas == 2 ? launch_kernel<2, 1>(groups, map_a, map_b, map_out, map_part, P, stream)
+                       : launch_kernel<1, 1>(groups, map_a, map_b, map_out, map_part, P, stream);
     ++g_launches;
     if (e != cudaSuccess) return SRQ_ERR_CUDA;
     if (P.splits > 1) {

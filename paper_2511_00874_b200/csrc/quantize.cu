@@ -280,12 +280,14 @@ __device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, const Ph
 //        (floor(S) + 2^23) >> 24.
 // |t| <= qmax for every element of a group (the reciprocal step is rounded toward zero), so
 // |C| <= qmax 2^24, the sum stays inside int32 and the code inside [-qmax, qmax] without a clamp.
-// quantize_sum returns the 32-bit sum whose top byte is the code (two's complement); pack4 takes
-// the top bytes, so the final shift costs nothing.
-template <bool SRM>
+// MODE: bit 0 = stochastic rounding (else round to nearest), bit 1 = E4M3 grid (else integer grid).
+constexpr int MODE_SR = 1, MODE_E4M3 = 2;
+
+// Integer grid: returns the 32-bit sum whose top byte is the code (two's complement).
+template <int MODE>
 __device__ __forceinline__ uint32_t quantize_sum(float x, float inv, uint32_t word) {
     const float s = __fmul_rn(__fmul_rn(x, inv), 16777216.0f);
-    if constexpr (SRM) {
+    if constexpr ((MODE & MODE_SR) != 0) {
         const int c = __float2int_ru(s);
         uint32_t sum;   // (~word >> 8) + c = (2^24 - 1 - u24) + c in one multiply-add (high half)
         asm("mad.hi.u32 %0, %1, 16777216, %2;" : "=r"(sum) : "r"(~word), "r"((uint32_t)c));
@@ -295,15 +297,52 @@ __device__ __forceinline__ uint32_t quantize_sum(float x, float inv, uint32_t wo
     }
 }
 
-__device__ __forceinline__ uint32_t pack4(uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3) {
-    return __byte_perm(__byte_perm(s0, s1, 0x0073), __byte_perm(s2, s3, 0x0073), 0x5410);
+// E4M3 grid: Def. 1 with the step of the binade of t = x * (1/D): for 2^e <= |t| < 2^(e+1) (e >= -6;
+// smaller |t| use e = -6, the subnormal spacing) the step is 2^(e-3) and u = t 2^(3-e) is rounded to
+// an integer q in [-16, 16] by the same exact fixed-point rule as above.  With E = e + 127 the biased
+// exponent of t, the code is sign | ((E - 120) << 3) + |q| - 8: |q| = 16 carries into the exponent
+// field (next binade), |q| < 8 only occurs for E = 121 and gives the subnormal codes, q = 0 gives +0.
+// Returns the code in the low byte.
+template <int MODE>
+__device__ __forceinline__ uint32_t quantize_e4m3(float x, float inv, uint32_t word) {
+    const float t = __fmul_rn(x, inv);
+    const uint32_t E = max((__float_as_uint(t) >> 23) & 0xFFu, 121u);          // |t| <= 448: E <= 135
+    const float s = __fmul_rn(t, __uint_as_float((281u - E) << 23));            // t 2^(3-e) 2^24, exact
+    uint32_t sum;
+    if constexpr ((MODE & MODE_SR) != 0) {
+        const int c = __float2int_ru(s);
+        asm("mad.hi.u32 %0, %1, 16777216, %2;" : "=r"(sum) : "r"(~word), "r"((uint32_t)c));
+    } else {
+        sum = (uint32_t)__float2int_rd(s) + 0x00800000u;
+    }
+    const int q = (int)sum >> 24;
+    return ((uint32_t)q & 0x80u) | ((E << 3) + (uint32_t)abs(q) - 968u);
 }
 
-template <bool SRM>
+// Four codes packed into one word, first element in the low byte.
+template <int MODE>
 __device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3,
                                               const uint32_t rnd[4]) {
-    return pack4(quantize_sum<SRM>(v[0], i0, rnd[0]), quantize_sum<SRM>(v[1], i1, rnd[1]),
-                 quantize_sum<SRM>(v[2], i2, rnd[2]), quantize_sum<SRM>(v[3], i3, rnd[3]));
+    if constexpr ((MODE & MODE_E4M3) != 0) {
+        const uint32_t c0 = quantize_e4m3<MODE>(v[0], i0, rnd[0]), c1 = quantize_e4m3<MODE>(v[1], i1, rnd[1]);
+        const uint32_t c2 = quantize_e4m3<MODE>(v[2], i2, rnd[2]), c3 = quantize_e4m3<MODE>(v[3], i3, rnd[3]);
+        return __byte_perm(__byte_perm(c0, c1, 0x0040), __byte_perm(c2, c3, 0x0040), 0x5410);
+    } else {
+        const uint32_t s0 = quantize_sum<MODE>(v[0], i0, rnd[0]), s1 = quantize_sum<MODE>(v[1], i1, rnd[1]);
+        const uint32_t s2 = quantize_sum<MODE>(v[2], i2, rnd[2]), s3 = quantize_sum<MODE>(v[3], i3, rnd[3]);
+        return __byte_perm(__byte_perm(s0, s1, 0x0073), __byte_perm(s2, s3, 0x0073), 0x5410);   // top bytes
+    }
+}
+
+// Same with the mode chosen at run time (general path).
+__device__ __forceinline__ uint32_t quantize4_rt(int mode, const float v[4], float i0, float i1, float i2, float i3,
+                                                 const uint32_t rnd[4]) {
+    switch (mode) {
+        case 0: return quantize4<0>(v, i0, i1, i2, i3, rnd);
+        case 1: return quantize4<1>(v, i0, i1, i2, i3, rnd);
+        case 2: return quantize4<2>(v, i0, i1, i2, i3, rnd);
+        default: return quantize4<3>(v, i0, i1, i2, i3, rnd);
+    }
 }
 
 // 4x4 byte transpose: w[i] holds columns c..c+3 of row i -> o[e] holds rows 0..3 of column c+e
@@ -322,6 +361,7 @@ struct QuantParams {
     uint64_t index_offset;
     PhiloxKeys keys;
     int sr;                       // 1 = SR, 0 = RTN
+    int mode;                     // MODE_SR | MODE_E4M3
     int per_row;                  // step size per row of each layout
     int8_t* codes_rm; int64_t ld_rm;
     int8_t* codes_tr; int64_t ld_tr;
@@ -368,12 +408,13 @@ __device__ __forceinline__ void widen(const uint2& q, float v[4]) {
 // current one is processed, which keeps two quads of loads in flight per thread.
 // FULL: the 128 x 128 tile lies inside the matrix and its Philox block indices do not carry into the
 // upper counter word, so rows need no bounds checks and the counter is one 32-bit multiply-add.
-template <typename T, bool SRM, int LAYOUT, bool PER_ROW, bool FULL>
+template <typename T, int MODE, int LAYOUT, bool PER_ROW, bool FULL>
 __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const QuantParams& P, uint32_t* tileT,
                                               int64_t r0, int64_t c0) {
     using Raw = typename Raw4<T>::type;
     constexpr bool WANT_RM = (LAYOUT & 1) != 0, WANT_TR = (LAYOUT & 2) != 0;
     constexpr bool TWO_STEPS = WANT_TR && PER_ROW;     // transposed layout has its own step sizes
+    constexpr bool SRM = (MODE & MODE_SR) != 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t c = c0 + lane * 4;
     const bool col_ok = FULL || c < P.cols;             // cols % 4 == 0: a group is all in or all out
@@ -432,9 +473,9 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
             }
             if constexpr (WANT_RM || !TWO_STEPS) {
                 const float ir = (PER_ROW && WANT_RM) ? inv_cur[i] : inv_tensor;
-                wr[i] = quantize4<SRM>(v, ir, ir, ir, ir, rnd);
+                wr[i] = quantize4<MODE>(v, ir, ir, ir, ir, rnd);
             }
-            if constexpr (TWO_STEPS) wt[i] = quantize4<SRM>(v, ic[0], ic[1], ic[2], ic[3], rnd);
+            if constexpr (TWO_STEPS) wt[i] = quantize4<MODE>(v, ic[0], ic[1], ic[2], ic[3], rnd);
             else wt[i] = wr[i];
             if constexpr (WANT_RM) {
                 if (FULL || (col_ok && r0 + tr < P.rows)) *reinterpret_cast<uint32_t*>(out_rm + tr * ld_rm) = wr[i];
@@ -455,7 +496,7 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
     }
 }
 
-template <typename T, bool SRM, int LAYOUT, bool PER_ROW>
+template <typename T, int MODE, int LAYOUT, bool PER_ROW>
 __global__ void __launch_bounds__(Q_THREADS)
 quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P) {
     __shared__ uint32_t tileT[(LAYOUT & 2) ? Q_TILE * (Q_TILE / 4) : 1];
@@ -466,8 +507,8 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
     const uint64_t j_first = (P.index_offset + (uint64_t)r0 * (uint64_t)P.cols + (uint64_t)c0) >> 2;
     const uint64_t j_span = (uint64_t)(Q_TILE - 1) * ((uint64_t)P.cols >> 2) + (Q_TILE / 4 - 1);
     const bool full = r0 + Q_TILE <= P.rows && c0 + Q_TILE <= P.cols && (j_first & 0xFFFFFFFFull) + j_span <= 0xFFFFFFFFull;
-    if (full) quantize_tile<T, SRM, LAYOUT, PER_ROW, true>(x, P, tileT, r0, c0);
-    else quantize_tile<T, SRM, LAYOUT, PER_ROW, false>(x, P, tileT, r0, c0);
+    if (full) quantize_tile<T, MODE, LAYOUT, PER_ROW, true>(x, P, tileT, r0, c0);
+    else quantize_tile<T, MODE, LAYOUT, PER_ROW, false>(x, P, tileT, r0, c0);
 }
 
 // General path: any extent, pitch, alignment and index offset; one Philox block per element
@@ -520,11 +561,9 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
                 }
                 const float inv_r = P.per_row ? P.inv_rm[want_rm ? r : 0] : inv_tensor;
                 if (want_rm || !two_steps)
-                    wr[i] = sr ? quantize4<true>(v, inv_r, inv_r, inv_r, inv_r, rnd)
-                               : quantize4<false>(v, inv_r, inv_r, inv_r, inv_r, rnd);
+                    wr[i] = quantize4_rt(P.mode, v, inv_r, inv_r, inv_r, inv_r, rnd);
                 if (two_steps)
-                    wt[i] = sr ? quantize4<true>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], rnd)
-                               : quantize4<false>(v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], rnd);
+                    wt[i] = quantize4_rt(P.mode, v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], rnd);
                 else
                     wt[i] = wr[i];
                 if (want_rm) {
@@ -554,26 +593,30 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
-template <typename T, bool SRM, int LAYOUT>
+template <typename T, int MODE, int LAYOUT>
 static void launch_fast_pr(bool per_row, const void* x, const QuantParams& P, unsigned grid, cudaStream_t st) {
-    if (per_row) quantize_fast_kernel<T, SRM, LAYOUT, true><<<grid, Q_THREADS, 0, st>>>((const T*)x, P);
-    else quantize_fast_kernel<T, SRM, LAYOUT, false><<<grid, Q_THREADS, 0, st>>>((const T*)x, P);
+    if (per_row) quantize_fast_kernel<T, MODE, LAYOUT, true><<<grid, Q_THREADS, 0, st>>>((const T*)x, P);
+    else quantize_fast_kernel<T, MODE, LAYOUT, false><<<grid, Q_THREADS, 0, st>>>((const T*)x, P);
 }
-template <typename T, bool SRM>
+template <typename T, int MODE>
 static void launch_fast_layout(int layout, bool per_row, const void* x, const QuantParams& P, unsigned grid, cudaStream_t st) {
-    if (layout == 1) launch_fast_pr<T, SRM, 1>(per_row, x, P, grid, st);
-    else if (layout == 2) launch_fast_pr<T, SRM, 2>(per_row, x, P, grid, st);
-    else launch_fast_pr<T, SRM, 3>(per_row, x, P, grid, st);
+    if (layout == 1) launch_fast_pr<T, MODE, 1>(per_row, x, P, grid, st);
+    else if (layout == 2) launch_fast_pr<T, MODE, 2>(per_row, x, P, grid, st);
+    else launch_fast_pr<T, MODE, 3>(per_row, x, P, grid, st);
 }
-static void launch_fast(srq_dtype_t dt, bool sr, int layout, bool per_row, const void* x, const QuantParams& P, unsigned grid,
-                        cudaStream_t st) {
-    if (dt == SRQ_F32) {
-        if (sr) launch_fast_layout<float, true>(layout, per_row, x, P, grid, st);
-        else launch_fast_layout<float, false>(layout, per_row, x, P, grid, st);
-    } else {
-        if (sr) launch_fast_layout<__nv_bfloat16, true>(layout, per_row, x, P, grid, st);
-        else launch_fast_layout<__nv_bfloat16, false>(layout, per_row, x, P, grid, st);
+template <typename T>
+static void launch_fast_mode(int mode, int layout, bool per_row, const void* x, const QuantParams& P, unsigned grid, cudaStream_t st) {
+    switch (mode) {
+        case 0: launch_fast_layout<T, 0>(layout, per_row, x, P, grid, st); break;
+        case 1: launch_fast_layout<T, 1>(layout, per_row, x, P, grid, st); break;
+        case 2: launch_fast_layout<T, 2>(layout, per_row, x, P, grid, st); break;
+        default: launch_fast_layout<T, 3>(layout, per_row, x, P, grid, st); break;
     }
+}
+static void launch_fast(srq_dtype_t dt, int mode, int layout, bool per_row, const void* x, const QuantParams& P, unsigned grid,
+                        cudaStream_t st) {
+    if (dt == SRQ_F32) launch_fast_mode<float>(mode, layout, per_row, x, P, grid, st);
+    else launch_fast_mode<__nv_bfloat16>(mode, layout, per_row, x, P, grid, st);
 }
 
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream) {
@@ -581,7 +624,8 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     const bool per_row = a.q.scale == SRQ_PER_ROW;
     const int64_t rows = a.rows, cols = a.cols;
     if (rows == 0 || cols == 0 || (!want_rm && !want_tr)) return cudaSuccess;
-    const float qmax = (float)((1 << (a.q.bits - 1)) - 1);
+    const bool e4m3 = a.q.format == SRQ_GRID_E4M3;
+    const float qmax = e4m3 ? 448.0f : (float)((1 << (a.q.bits - 1)) - 1);
     const size_t esize = a.dt == SRQ_F32 ? 4 : 2;
 
     // group counts and where each layout's absmax lives; per tensor both layouts share word 0
@@ -623,6 +667,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         }
         P.keys.tid0 = (uint32_t)a.q.tensor_id; P.keys.tid1 = (uint32_t)(a.q.tensor_id >> 32);
         P.sr = a.q.round == SRQ_SR;
+        P.mode = (P.sr ? MODE_SR : 0) | (e4m3 ? MODE_E4M3 : 0);
         P.per_row = per_row;
         P.codes_rm = a.codes_rm; P.ld_rm = a.ld_rm;
         P.codes_tr = a.codes_tr; P.ld_tr = a.ld_tr;
@@ -633,7 +678,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) &&
                           (!want_tr || (P.vec_tr && rows % 4 == 0));
         const unsigned grid = (unsigned)(((cols + Q_TILE - 1) / Q_TILE) * ((rows + Q_TILE - 1) / Q_TILE));
-        if (fast) launch_fast(a.dt, P.sr != 0, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);
+        if (fast) launch_fast(a.dt, P.mode, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);
         else if (a.dt == SRQ_F32) quantize_kernel<float><<<grid, Q_THREADS, 0, stream>>>((const float*)a.x, P);
         else quantize_kernel<__nv_bfloat16><<<grid, Q_THREADS, 0, stream>>>((const __nv_bfloat16*)a.x, P);
         ++g_launches;
