@@ -78,7 +78,7 @@ typedef enum { SRQ_SR = 0, SRQ_RTN = 1 } srq_round_t;
 /* Grid of a quantization point: integers times the step size (bits 2..8), or the E4M3 8-bit
  * floating-point values times the step size (1 sign, 4 exponent, 3 mantissa bits, bias 7, no
  * infinities, largest value 448; `bits` is ignored). */
-typedef enum { SRQ_GRID_INT = 0, SRQ_GRID_E4M3 = 1 } srq_grid_t;
+typedef enum { SRQ_GRID_INT = 0, SRQ_GRID_E4M3 = 1, SRQ_GRID_NONE = 2 /* operand left unquantized */ } srq_grid_t;
 
 /* One quantization point: the paper's (D, eps) pair for one operand of one pass
  * (five per layer: A and W forward; A, W and dY backward). */
@@ -189,7 +189,13 @@ srq_status_t srq_gemm_e4m3(const uint8_t *a, int64_t lda, const uint8_t *b, int6
                            void *ws, size_t ws_bytes, void *cuda_stream);
 
 /* Alg. 1: Y[T,N] = Q(A) Q(W)^T.  qA, qW are the forward quantization points of A and W.
- * Per row: A per token, W per output feature. */
+ * Per row: A per token, W per output feature.
+ * qA->format == SRQ_GRID_NONE gives the forward pass of the paper's mixed-precision SGD for the
+ * quantization-aware objective, which leaves the forward activations unquantized (D_A^fwd = 0):
+ * Y = A Q(W)^T with A used as the bfloat16 numbers it holds (dt must be SRQ_BF16, K a multiple
+ * of 8, W on the integer grid).  The product then runs in bfloat16 with binary32 accumulation,
+ * so Y agrees with the exact product to about 1e-5 * |row| * |col| rather than bit for bit; dbg
+ * is ignored. */
 srq_status_t qlinear_fwd(const void *A, const void *W, srq_dtype_t dt,
                          int64_t T, int64_t N, int64_t K,
                          const srq_qspec_t *qA, const srq_qspec_t *qW,

@@ -335,3 +335,14 @@ def qlinear_bwd_input_e4m3(dY, W, qdy: QSpec, qw: QSpec) -> LinearResult:
 
 def qlinear_bwd_weight_e4m3(dY, A, qdy: QSpec, qa: QSpec) -> LinearResult:
     return _qlinear_e4m3(dY, A, qdy, qa, True, True)
+
+
+def qlinear_fwd_fp_act(A, W, qw: QSpec) -> LinearResult:
+    """Forward pass of the paper's mixed-precision SGD for the quantization-aware objective
+    (Sec. 3.3: D_A^fwd = 0, only W is quantized): Y = A Q(W)^T with A as given, in binary64.
+    acc holds A codes(W)^T, out = acc * D_W."""
+    A = np.ascontiguousarray(A, dtype=np.float32)
+    cw, sw, _, _ = sr_quantize(W, qw, True, False)
+    acc = A.astype(np.float64) @ cw.astype(np.float64).T          # library matmul as one step
+    out = acc * np.broadcast_to(sw.astype(np.float64), (cw.shape[0],))[None, :]
+    return LinearResult(out, acc, None, None, cw, sw)

@@ -23,7 +23,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_ACC_OVERFLOW, ERR_CUDA,
 F32, BF16 = 0, 1
 PER_TENSOR, PER_ROW = 0, 1
 SR, RTN = 0, 1
-GRID_INT, GRID_E4M3 = 0, 1
+GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
            "sr_quantize", "sr_quantize_static", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",

@@ -117,6 +117,57 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
     return SRQ_OK;
 }
 
+// Forward pass with unquantized activations (the paper's SR-MP-SGD for the QAT objective keeps
+// D_A^fwd = 0): Y = A Q(W)^T with A taken as the bfloat16 numbers it holds.  Q(W) is quantized as
+// usual, its integer codes are widened to bfloat16 (exact) and the product runs in kind::f16 with
+// binary32 accumulation; Y[t, n] = acc[t, n] * D_W[n].
+struct FpActPlan { size_t off_scratch, off_scale, off_one, off_codes8, off_codes16, total; int64_t pitch8, pitch16; };
+
+FpActPlan plan_fp_act(int64_t N, int64_t K) {
+    FpActPlan p;
+    size_t o = sizeof(WsHeader);
+    p.off_scratch = o; o += quant_scratch_bytes(N, K);
+    p.off_scale = o; o += f32_block(N);
+    p.off_one = o; o += f32_block(1);
+    p.pitch8 = pitch16(K); p.pitch16 = pitch16(2 * K) / 2;       // elements; rows start on 16-byte boundaries
+    p.off_codes8 = o; o += align_up((size_t)N * p.pitch8);
+    p.off_codes16 = o; o += align_up((size_t)N * p.pitch16 * 2);
+    p.total = o;
+    return p;
+}
+
+srq_status_t run_fwd_fp_act(const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
+                            const srq_qspec_t* qW, float* Y, void* ws, size_t ws_bytes, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!A || !W || !Y || !ws || T < 0 || N < 0 || K < 0) return SRQ_ERR_INVALID_ARG;
+    if (dt != SRQ_BF16) return SRQ_ERR_UNSUPPORTED;                  // the activations feed the tensor cores as they are
+    srq_status_t s = check_qspec(qW);
+    if (s != SRQ_OK) return s;
+    if (qW->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;
+    if (K % 8 != 0) return SRQ_ERR_INVALID_ARG;                      // rows of A must start on 16-byte boundaries (TMA)
+    if (!aligned_to(A, 16) || !aligned_to(W, 16) || !aligned_to(Y, 16) || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
+    const FpActPlan p = plan_fp_act(N, K);
+    if (ws_bytes < p.total) return SRQ_ERR_WORKSPACE;
+    if (T == 0 || N == 0) return SRQ_OK;
+    if (K == 0) return cudaMemset2DAsync(Y, (size_t)N * 4, 0, (size_t)N * 4, (size_t)T, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+    char* base = (char*)ws;
+    uint32_t* status = &((WsHeader*)ws)->status;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    int8_t* c8 = (int8_t*)(base + p.off_codes8);
+    float* scale = (float*)(base + p.off_scale);
+    float* one = (float*)(base + p.off_one);
+    QuantArgs q; q.x = W; q.dt = dt; q.rows = N; q.cols = K; q.ld = K; q.q = *qW;
+    q.codes_rm = c8; q.ld_rm = p.pitch8; q.scale_rm = scale; q.codes_tr = nullptr; q.ld_tr = 0; q.scale_tr = nullptr;
+    if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch, N, K), status, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    if (launch_widen_codes(c8, N, K, p.pitch8, base + p.off_codes16, p.pitch16, one, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    GemmArgs g;
+    g.a = (const int8_t*)A; g.lda = 2 * K; g.b = (const int8_t*)(base + p.off_codes16); g.ldb = 2 * p.pitch16;
+    g.M = T; g.N = N; g.Kc = 2 * K; g.kind = 2;
+    g.s_row = one; g.row_stride = 0; g.s_col = scale; g.col_stride = qW->scale == SRQ_PER_ROW;
+    g.out = Y; g.ldo = N; g.acc_out = nullptr; g.splitk_ws = nullptr; g.splitk_ws_bytes = 0;
+    return launch_gemm_i8(g, status, st);
+}
+
 // Alg. 2 as one call: dY is read once and written in both code layouts, then both products run.
 struct BwdPlan {
     size_t off_scratch[3], off_scale[4], off_codes[4], off_split[2], total;
@@ -251,8 +302,9 @@ size_t srq_workspace_bytes(int64_t T, int64_t N, int64_t K) {
     const size_t m1 = plan_layer(iy, iw).total, m2 = plan_layer(wy, wa).total;
     if (m1 > m) m = m1;
     if (m2 > m) m = m2;
-    const size_t m3 = plan_bwd(T, N, K).total;
+    const size_t m3 = plan_bwd(T, N, K).total, m4 = plan_fp_act(N, K).total;
     if (m3 > m) m = m3;
+    if (m4 > m) m = m4;
     return m;
 }
 
@@ -324,6 +376,7 @@ srq_status_t srq_gemm_e4m3(const uint8_t* a, int64_t lda, const uint8_t* b, int6
 srq_status_t qlinear_fwd(const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
                          const srq_qspec_t* qA, const srq_qspec_t* qW, float* Y, const srq_debug_out_t* dbg,
                          void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (qA && qA->format == SRQ_GRID_NONE) return run_fwd_fp_act(A, W, dt, T, N, K, qW, Y, ws, ws_bytes, cuda_stream);
     const Operand a{A, T, K, false, qA}, b{W, N, K, false, qW};
     return run_layer(a, b, dt, Y, dbg, ws, ws_bytes, cuda_stream);
 }

@@ -51,13 +51,18 @@ struct QuantArgs {
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& scratch, uint32_t* status,
                             cudaStream_t stream);
 
+// int8 codes as bfloat16 integers (pitches in elements); *one receives 1.0f.
+cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, int64_t ld, void* out_bf16, int64_t ld_out,
+                               float* one, cudaStream_t stream);
+
 // ------------------------------------------------------------------------------------------
 // int8 GEMM (gemm_i8.cu)
 // ------------------------------------------------------------------------------------------
 struct GemmArgs {
     const int8_t* a; int64_t lda; const int8_t* b; int64_t ldb;
     int64_t M, N, Kc;
-    int kind;                                   // 0: int8 codes, int32 sums; 1: E4M3 codes, binary32 sums
+    int kind;                                   // 0: int8 codes, int32 sums; 1: E4M3 codes, binary32 sums;
+                                                // 2: bfloat16 operands, binary32 sums (Kc, lda, ldb in BYTES)
     const float* s_row; int32_t row_stride; const float* s_col; int32_t col_stride;
     float* out; int64_t ldo; int32_t* acc_out;
     void* splitk_ws; size_t splitk_ws_bytes;   // int32 [M,N] partial sums

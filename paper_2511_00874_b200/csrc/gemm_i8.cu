@@ -188,7 +188,8 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
 
 // D[tmem] (+)= A[smem] * B[smem], issued by one thread (of the leader CTA when CTAS = 2; the
 // descriptors then address the same offsets in both CTAs).  KIND 0: int8 operands, int32
-// accumulators (kind::i8); KIND 1: E4M3 operands, binary32 accumulators (kind::f8f6f4).
+// accumulators (kind::i8); KIND 1: E4M3 operands, binary32 accumulators (kind::f8f6f4); KIND 2:
+// bfloat16 operands, binary32 accumulators (kind::f16; 16 elements = 32 bytes of K per instruction).
 template <int CTAS, int KIND>
 __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
 #define SRQ_UMMA(GROUP, KINDSTR)                                                                   \
@@ -198,7 +199,9 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
     if constexpr (CTAS == 1 && KIND == 0) SRQ_UMMA("1", "i8");
     else if constexpr (CTAS == 2 && KIND == 0) SRQ_UMMA("2", "i8");
     else if constexpr (CTAS == 1 && KIND == 1) SRQ_UMMA("1", "f8f6f4");
-    else SRQ_UMMA("2", "f8f6f4");
+    else if constexpr (CTAS == 2 && KIND == 1) SRQ_UMMA("2", "f8f6f4");
+    else if constexpr (CTAS == 1 && KIND == 2) SRQ_UMMA("1", "f16");
+    else SRQ_UMMA("2", "f16");
 #undef SRQ_UMMA
 }
 // The mbarrier gets one arrival once every MMA issued so far by this thread has completed.
@@ -246,9 +249,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
 }
 
 // Instruction descriptor: dense, no saturation, both operands K-major, N x M; KIND 0: D = s32,
-// A = B = s8; KIND 1: D = f32, A = B = E4M3 (format 0).
+// A = B = s8; KIND 1: D = f32, A = B = E4M3 (format 0); KIND 2: D = f32, A = B = bfloat16.
 __device__ __forceinline__ constexpr uint32_t make_idesc(int kind, int m, int n) {
-    const uint32_t types = kind == 0 ? ((2u << 4) | (1u << 7) | (1u << 10)) : (1u << 4);
+    const uint32_t types = kind == 0 ? ((2u << 4) | (1u << 7) | (1u << 10))          // s32 <- s8 x s8
+                         : kind == 1 ? (1u << 4)                                   // f32 <- e4m3 x e4m3
+                                     : ((1u << 4) | (1u << 7) | (1u << 10));       // f32 <- bf16 x bf16
     return types | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
@@ -623,6 +628,8 @@ static bool device_info(DeviceInfo** out) {
         if (cudaFuncSetAttribute(gemm_i8_kernel<2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<2>()) != cudaSuccess) return false;
         if (cudaFuncSetAttribute(gemm_i8_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<1>()) != cudaSuccess) return false;
         if (cudaFuncSetAttribute(gemm_i8_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<2>()) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_i8_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<1>()) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_i8_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem<2>()) != cudaSuccess) return false;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(d.sms / 2 * 2)); cfg.blockDim = dim3(GEMM_THREADS); cfg.dynamicSmemBytes = gemm_smem<2>();
         cudaLaunchAttribute at;
@@ -718,8 +725,10 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     cudaError_t e;
     if (g.kind == 0) e = ctas == 2 ? launch_kernel<2, 0>(groups, map_a, map_b, map_out, map_part, P, stream)
                                    : launch_kernel<1, 0>(groups, map_a, map_b, map_out, map_part, P, stream);
-    else e = ctas == 2 ? launch_kernel<2, 1>(groups, map_a, map_b, map_out, map_part, P, stream)
-                       : launch_kernel<1, 1>(groups, map_a, map_b, map_out, map_part, P, stream);
+    else if (g.kind == 1) e = ctas == 2 ? launch_kernel<2, 1>(groups, map_a, map_b, map_out, map_part, P, stream)
+                                        : launch_kernel<1, 1>(groups, map_a, map_b, map_out, map_part, P, stream);
+    else e = ctas == 2 ? launch_kernel<2, 2>(groups, map_a, map_b, map_out, map_part, P, stream)
+                       : launch_kernel<1, 2>(groups, map_a, map_b, map_out, map_part, P, stream);
     ++g_launches;
     if (e != cudaSuccess) return SRQ_ERR_CUDA;
     if (P.splits > 1) {

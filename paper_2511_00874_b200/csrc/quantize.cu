@@ -619,6 +619,26 @@ static void launch_fast(srq_dtype_t dt, int mode, int layout, bool per_row, cons
     else launch_fast_mode<__nv_bfloat16>(mode, layout, per_row, x, P, grid, st);
 }
 
+// int8 codes [rows, cols] -> the same integers as bfloat16 (exact: |code| <= 127), for the product
+// of unquantized bfloat16 activations with a quantized weight.  Also writes 1.0f to *one.
+__global__ void widen_codes_kernel(const int8_t* __restrict__ codes, int64_t rows, int64_t cols, int64_t ld,
+                                   uint16_t* __restrict__ out, int64_t ld_out, float* one) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) *one = 1.0f;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < rows * cols; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / cols, c = i % cols;
+        out[r * ld_out + c] = (uint16_t)(__float_as_uint(__int2float_rn((int)codes[r * ld + c])) >> 16);
+    }
+}
+
+cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, int64_t ld, void* out_bf16, int64_t ld_out,
+                               float* one, cudaStream_t stream) {
+    const int64_t n = rows * cols;
+    const unsigned grid = (unsigned)(n / 256 + 1 < 4096 ? n / 256 + 1 : 4096);
+    widen_codes_kernel<<<grid, 256, 0, stream>>>(codes, rows, cols, ld, (uint16_t*)out_bf16, ld_out, one);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream) {
     const bool want_rm = a.codes_rm != nullptr, want_tr = a.codes_tr != nullptr;
     const bool per_row = a.q.scale == SRQ_PER_ROW;

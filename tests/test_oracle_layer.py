@@ -180,3 +180,22 @@ def test_one_bit_less_costs_about_four_times_the_variance():
         v[bits] = outs.var(0).mean()
     ratio = v[7] / v[8]
     assert abs(ratio - (127 / 63) ** 2) < 0.6
+
+
+def test_forward_with_unquantized_activations_reduces_to_known_cases():
+    """Sec. 3.3 variant (D_A^fwd = 0): unit-vector activations read out the dequantized weight, and
+    activations that already lie on the 8-bit grid give what the fully quantized forward gives."""
+    rng = np.random.default_rng(11)
+    W = rng.normal(0, 0.02, (12, 16)).astype(np.float32)
+    qw = QSpec(8, PER_ROW, SR, 3, 1)
+    eye = np.eye(16, dtype=np.float32)
+    r = oracle.qlinear_fwd_fp_act(eye, W, qw)
+    cw, sw, _, _ = oracle.sr_quantize(W, qw)
+    assert np.array_equal(r.out, (cw.astype(np.float64) * sw.astype(np.float64)[:, None]).T)
+    A = rng.integers(-127, 128, (9, 16)).astype(np.float32)
+    A[0, 0] = 127                                   # absmax 127: step size 1, codes = A
+    full = oracle.qlinear_fwd(A, W, QSpec(8, PER_TENSOR, RTN), qw)
+    assert full.scale_a[0] == 1 and np.array_equal(full.codes_a, A.astype(np.int8))
+    part = oracle.qlinear_fwd_fp_act(A, W, qw)
+    assert np.array_equal(part.acc, full.acc.astype(np.float64))
+    assert np.array_equal(part.out.astype(np.float32), full.out)
