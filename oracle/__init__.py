@@ -104,6 +104,11 @@ def lib() -> ctypes.CDLL:
         L.orc_sr_quantize_e4m3.restype = ctypes.c_int
         L.orc_gemm_e4m3_nt.argtypes = [vp, vp, i64, i64, i64, vp, ctypes.c_int, vp, ctypes.c_int, vp, vp]
         L.orc_gemm_e4m3_nt.restype = None
+        L.orc_requantize.argtypes = [vp, i64, i64, ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_uint64,
+                                     ctypes.c_uint64, ctypes.c_uint64, vp, ctypes.POINTER(ctypes.c_float)]
+        L.orc_requantize.restype = None
+        L.orc_accumulate.argtypes = [vp, vp, i64]
+        L.orc_accumulate.restype = None
         L.orc_num_threads.argtypes = []
         L.orc_num_threads.restype = ctypes.c_int
     return _lib
@@ -346,3 +351,23 @@ def qlinear_fwd_fp_act(A, W, qw: QSpec) -> LinearResult:
     acc = A.astype(np.float64) @ cw.astype(np.float64).T          # library matmul as one step
     out = acc * np.broadcast_to(sw.astype(np.float64), (cw.shape[0],))[None, :]
     return LinearResult(out, acc, None, None, cw, sw)
+
+
+def requantize(out, step: float, q: QSpec):
+    """(codes int8 [M, N], max |out|) of a product's output quantized with a caller-supplied step."""
+    out = np.ascontiguousarray(out, dtype=np.float32)
+    M, N = out.shape
+    codes = np.zeros((M, N), dtype=np.int8)
+    m = ctypes.c_float()
+    lib().orc_requantize(_ptr(out), M, N, ctypes.c_float(step), q.bits, q.round_mode, q.seed, q.tensor_id,
+                         q.index_offset, _ptr(codes), ctypes.byref(m))
+    return codes, np.float32(m.value)
+
+
+def accumulate(dst, src) -> np.ndarray:
+    """dst + src in binary32 (one addition per element), as a new array."""
+    d = np.array(dst, dtype=np.float32, order="C", copy=True)
+    s = np.ascontiguousarray(src, dtype=np.float32)
+    assert d.shape == s.shape
+    lib().orc_accumulate(_ptr(d), _ptr(s), d.size)
+    return d

@@ -574,3 +574,45 @@ void orc_gemm_e4m3_nt(const uint8_t *a, const uint8_t *b, int64_t M, int64_t N, 
             out[i * N + j] = s * (double)sc;
         }
 }
+
+/* ====================================================================== */
+/* Output options of a product                                              */
+/* ====================================================================== */
+/*
+ * Quantization of a product's output for the layer that consumes it (the
+ * next layer's Q(A_in), Alg. 1; or the previous layer's Q(dA_out), Alg. 2)
+ * with a step size D that the caller supplies, because the absmax of the
+ * output is not known before the product has finished.  1/D is one binary32
+ * division; t = out * (1/D) is SATURATED to [-qmax, qmax] (a step size taken
+ * from an earlier tensor does not bound this one), then rounded by the rule of
+ * orc_quantize_scalar with the threshold of flat index
+ * index_offset + i * N + j.  D = 0 (or a reciprocal that overflows) gives
+ * codes 0.  Also returns max |out| through absmax.
+ */
+void orc_requantize(const float *out, int64_t M, int64_t N, float step, int bits, int round_mode,
+                    uint64_t seed, uint64_t tensor_id, uint64_t index_offset,
+                    int8_t *codes, float *absmax)
+{
+    float qmax = (float)orc_qmax(bits);
+    float inv = (step == 0.0f) ? 0.0f : 1.0f / step;
+    if (isinf(inv) || inv != inv) inv = 0.0f;
+    float best = 0.0f;
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            float o = out[i * N + j];
+            if (fabsf(o) > best) best = fabsf(o);
+            float t = o * inv;
+            if (t > qmax) t = qmax;
+            if (t < -qmax) t = -qmax;
+            uint64_t idx = index_offset + (uint64_t)i * (uint64_t)N + (uint64_t)j;
+            uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, idx) : 0u;
+            codes[i * N + j] = (int8_t)orc_quantize_scalar(t, 1.0f, bits, round_mode, u24);
+        }
+    if (absmax) *absmax = best;
+}
+
+/* Gradient accumulation over micro-batches: dst += src, one binary32 addition per element. */
+void orc_accumulate(float *dst, const float *src, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) dst[i] = dst[i] + src[i];
+}

@@ -26,6 +26,41 @@ __device__ __forceinline__ void record_status(uint32_t* status, uint32_t code) {
 }
 
 // ------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds, two 32x32->64 multiplies per round.
+// The ten round keys (key + r * Weyl constants) are the same for every thread; the host
+// computes them once and passes them in the kernel parameters.
+// ------------------------------------------------------------------------------------------
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+    uint32_t tid0, tid1;     // counter words 2 and 3 (tensor_id)
+};
+
+__device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, const PhiloxKeys& K, uint32_t out[4]) {
+    uint32_t c2 = K.tid0, c3 = K.tid1;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;    // one wide multiply: hi and lo
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
+        c3 = (uint32_t)p0;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Round keys and upper counter words for one quantization point.
+inline PhiloxKeys make_philox_keys(uint64_t seed, uint64_t tensor_id) {
+    PhiloxKeys k;
+    for (int r = 0; r < 10; ++r) {
+        k.k0[r] = (uint32_t)seed + (uint32_t)r * 0x9E3779B9u;
+        k.k1[r] = (uint32_t)(seed >> 32) + (uint32_t)r * 0xBB67AE85u;
+    }
+    k.tid0 = (uint32_t)tensor_id; k.tid1 = (uint32_t)(tensor_id >> 32);
+    return k;
+}
+
+// ------------------------------------------------------------------------------------------
 // Quantizer (quantize.cu)
 // ------------------------------------------------------------------------------------------
 // Scratch carved from a workspace for one sr_quantize: absmax words and reciprocal steps for

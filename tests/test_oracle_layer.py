@@ -199,3 +199,35 @@ def test_forward_with_unquantized_activations_reduces_to_known_cases():
     part = oracle.qlinear_fwd_fp_act(A, W, qw)
     assert np.array_equal(part.acc, full.acc.astype(np.float64))
     assert np.array_equal(part.out.astype(np.float32), full.out)
+
+
+def test_requantization_of_an_output_with_a_supplied_step():
+    from fractions import Fraction
+    from _independent import thresholds_u24
+    rng = np.random.default_rng(12)
+    out = (rng.normal(0, 3, (11, 20))).astype(np.float32)
+    out[0, :5] = [1000.0, -1000.0, 31.75, -31.75, 0.0]          # far outside, and on the edge of, the range
+    step = np.float32(0.25)
+    for bits, rnd in ((8, SR), (8, RTN), (4, SR)):
+        q = QSpec(bits, PER_TENSOR, rnd, seed=9, tensor_id=4, index_offset=6)
+        codes, m = oracle.requantize(out, float(step), q)
+        assert m == np.abs(out).max()
+        qmax = 2 ** (bits - 1) - 1
+        u = thresholds_u24(9, 4, 6, 11, 20)
+        inv = np.float32(1) / step
+        for idx in np.ndindex(out.shape):                      # Def. 1 in exact rationals after saturation
+            t = Fraction(float(np.float32(out[idx] * inv)))
+            t = max(Fraction(-qmax), min(Fraction(qmax), t))
+            f = t.numerator // t.denominator
+            p = t - f
+            up = (Fraction(int(u[idx]), 2 ** 24) < p) if rnd == SR else (p >= Fraction(1, 2))
+            assert codes[idx] == f + int(up), idx
+        assert codes[0, 0] == qmax and codes[0, 1] == -qmax and codes[0, 4] == 0
+    # grid values with a power-of-two step are reproduced; a zero step gives zero codes
+    grid = (rng.integers(-127, 128, (5, 8)) * 0.5).astype(np.float32)
+    codes, _ = oracle.requantize(grid, 0.5, QSpec(8, PER_TENSOR, SR, 1, 1))
+    assert np.array_equal(codes, (grid * 2).astype(np.int8))
+    assert not oracle.requantize(grid, 0.0, QSpec(8, PER_TENSOR, SR, 1, 1))[0].any()
+    # accumulation is one binary32 addition per element
+    a, b = rng.normal(0, 1, 50).astype(np.float32), rng.normal(0, 1e-3, 50).astype(np.float32)
+    assert np.array_equal(oracle.accumulate(a, b), a + b)
