@@ -232,6 +232,56 @@ srq_status_t qlinear_bwd(const void *dY, const void *A, const void *W, srq_dtype
                          const srq_debug_out_t *dbg_input, const srq_debug_out_t *dbg_weight,
                          void *ws, size_t ws_bytes, void *cuda_stream);
 
+/*
+ * What else a product does with its results; every member is optional (zero / NULL).
+ *   accumulate  1: out += result (one binary32 addition per element) instead of out = result.
+ *               The paper emulates large batches by accumulating gradients over micro-batches
+ *               (hardware-considerations section); this is that accumulation for dW.
+ *   q, step, codes, ld_codes
+ *               also write Q(result) as int8 codes [M, ld_codes] for the layer that consumes the
+ *               result (the next layer's Q(A_in) of Alg. 1, the previous layer's Q(dA_out) of
+ *               Alg. 2), fused into the product's epilogue so that the result is not read again.
+ *               The absmax of a result is not known until the product has finished, so the step
+ *               size comes from the caller: *step (device, [1]); x / D is out * (1 / D) with one
+ *               binary32 division, SATURATED to [-qmax, qmax], then rounded by q->round with the
+ *               thresholds of (q->seed, q->tensor_id, q->index_offset + i * N + j).  q must be on
+ *               the integer grid; q->scale is ignored (one step for the whole result).  With
+ *               codes given, the fp32 output pointer of the call may be NULL.
+ *   absmax      device [1], holding a non-negative number (usually 0) on entry: raised to
+ *               max |result|, from which the caller derives the step size of its next step.
+ * Products with q or absmax set are never split along the contraction.
+ */
+typedef struct {
+    int32_t accumulate;
+    int32_t reserved;
+    const srq_qspec_t *q;
+    const float *step;
+    int8_t *codes;
+    int64_t ld_codes;
+    float *absmax;
+} srq_output_t;
+
+/* srq_gemm_i8, qlinear_fwd and qlinear_bwd with output options (NULL = none, i.e. the plain call).
+ * In qlinear_bwd_ex, output_dA applies to dA[T,K] and output_dW to dW[N,K]. */
+srq_status_t srq_gemm_i8_ex(const int8_t *a, int64_t lda, const int8_t *b, int64_t ldb,
+                            int64_t M, int64_t N, int64_t Kc,
+                            const float *s_row, int32_t row_stride,
+                            const float *s_col, int32_t col_stride,
+                            float *out, int64_t ldo, int32_t *acc_out, const srq_output_t *output,
+                            void *ws, size_t ws_bytes, void *cuda_stream);
+srq_status_t qlinear_fwd_ex(const void *A, const void *W, srq_dtype_t dt,
+                            int64_t T, int64_t N, int64_t K,
+                            const srq_qspec_t *qA, const srq_qspec_t *qW, float *Y,
+                            const srq_output_t *output, const srq_debug_out_t *dbg,
+                            void *ws, size_t ws_bytes, void *cuda_stream);
+srq_status_t qlinear_bwd_ex(const void *dY, const void *A, const void *W, srq_dtype_t dt,
+                            int64_t T, int64_t N, int64_t K,
+                            const srq_qspec_t *qdY, const srq_qspec_t *qA, const srq_qspec_t *qW,
+                            float *dA, float *dW,
+                            const srq_output_t *output_dA, const srq_output_t *output_dW,
+                            const srq_debug_out_t *dbg_input, const srq_debug_out_t *dbg_weight,
+                            void *ws, size_t ws_bytes, void *cuda_stream);
+
 /* Waits for the stream, then returns the device status word of the workspace: SRQ_OK, or the
  * first device-side condition recorded by the calls that used this workspace since its header
  * was last cleared (every entry point clears it when it starts). */

@@ -27,6 +27,7 @@ GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
            "sr_quantize", "sr_quantize_static", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
+           "srq_gemm_i8_ex", "qlinear_fwd_ex", "qlinear_bwd_ex",
            "srq_poll_status", "srq_status_string", "srq_launch_count"]
 
 
@@ -46,6 +47,12 @@ class _DebugOut(ctypes.Structure):
     _fields_ = [("codes_a", ctypes.c_void_p), ("scale_a", ctypes.c_void_p),
                 ("codes_b", ctypes.c_void_p), ("scale_b", ctypes.c_void_p),
                 ("acc", ctypes.c_void_p)]
+
+
+class _Output(ctypes.Structure):
+    _fields_ = [("accumulate", ctypes.c_int32), ("reserved", ctypes.c_int32), ("q", ctypes.POINTER(_QSpec)),
+                ("step", ctypes.c_void_p), ("codes", ctypes.c_void_p), ("ld_codes", ctypes.c_int64),
+                ("absmax", ctypes.c_void_p)]
 
 
 @dataclass
@@ -99,6 +106,13 @@ def lib() -> ctypes.CDLL:
         f.restype = ctypes.c_int
     L.qlinear_bwd.argtypes = [vp, vp, vp, ctypes.c_int, i64, i64, i64, qp, qp, qp, vp, vp, dp, dp, vp, sz, vp]
     L.qlinear_bwd.restype = ctypes.c_int
+    op = ctypes.POINTER(_Output)
+    L.srq_gemm_i8_ex.argtypes = [vp, i64, vp, i64, i64, i64, i64, vp, i32, vp, i32, vp, i64, vp, op, vp, sz, vp]
+    L.srq_gemm_i8_ex.restype = ctypes.c_int
+    L.qlinear_fwd_ex.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, qp, qp, vp, op, dp, vp, sz, vp]
+    L.qlinear_fwd_ex.restype = ctypes.c_int
+    L.qlinear_bwd_ex.argtypes = [vp, vp, vp, ctypes.c_int, i64, i64, i64, qp, qp, qp, vp, vp, op, op, dp, dp, vp, sz, vp]
+    L.qlinear_bwd_ex.restype = ctypes.c_int
     L.srq_poll_status.argtypes = [vp, vp]
     L.srq_poll_status.restype = ctypes.c_int
     L.srq_status_string.argtypes = [ctypes.c_int]
@@ -324,6 +338,81 @@ def qlinear_bwd(dY: torch.Tensor, A: torch.Tensor, W: torch.Tensor, qdY: QSpec, 
                            ctypes.byref(d1) if d1 is not None else None,
                            ws.data_ptr(), ws.numel(), _stream())
     _check(st, "qlinear_bwd")
+
+
+@dataclass
+class Output:
+    """Output options of a product (srq_output_t): accumulate into out, codes of Q(result) with a
+    caller-supplied step (q, step, codes), absmax of the result."""
+    accumulate: bool = False
+    q: Optional[QSpec] = None
+    step: Optional[torch.Tensor] = None
+    codes: Optional[torch.Tensor] = None
+    absmax: Optional[torch.Tensor] = None
+
+    def c(self):
+        cq = self.q.c() if self.q is not None else None
+        o = _Output(int(self.accumulate), 0, ctypes.pointer(cq) if cq is not None else None, _ptr(self.step),
+                    _ptr(self.codes), self.codes.stride(0) if self.codes is not None else 0, _ptr(self.absmax))
+        o._keep = cq                      # the struct points into cq
+        return o
+
+
+def _opt(o: Optional[Output]):
+    return None if o is None else o.c()
+
+
+def srq_gemm_i8_ex(a: torch.Tensor, b: torch.Tensor, s_row: torch.Tensor, s_col: torch.Tensor,
+                   out: Optional[torch.Tensor], output: Optional[Output] = None,
+                   acc_out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None) -> None:
+    """srq_gemm_i8 with output options; out may be None when codes are requested."""
+    _dev2d(a, "a")
+    _dev2d(b, "b")
+    M, Kc = a.shape
+    N = b.shape[0]
+    if ws is None:
+        ws = new_workspace(srq_gemm_workspace_bytes(M, N), a.device)
+    co = _opt(output)
+    st = lib().srq_gemm_i8_ex(a.data_ptr(), a.stride(0), b.data_ptr(), b.stride(0), M, N, Kc,
+                              s_row.data_ptr(), int(s_row.numel() != 1), s_col.data_ptr(), int(s_col.numel() != 1),
+                              _ptr(out), out.stride(0) if out is not None else 0, _ptr(acc_out),
+                              ctypes.byref(co) if co is not None else None, ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "srq_gemm_i8_ex")
+
+
+def qlinear_fwd_ex(A: torch.Tensor, W: torch.Tensor, qA: QSpec, qW: QSpec, Y: Optional[torch.Tensor],
+                   output: Optional[Output] = None, dbg: Optional[DebugOut] = None,
+                   ws: Optional[torch.Tensor] = None) -> None:
+    """qlinear_fwd with output options; Y may be None when codes are requested."""
+    T, K = A.shape
+    N = W.shape[0]
+    if ws is None:
+        ws = new_workspace(srq_workspace_bytes(T, N, K), A.device)
+    c0, c1 = qA.c(), qW.c()
+    cd = dbg.c() if dbg is not None else None
+    co = _opt(output)
+    st = lib().qlinear_fwd_ex(A.data_ptr(), W.data_ptr(), _dtype_of(A), T, N, K, ctypes.byref(c0), ctypes.byref(c1),
+                              _ptr(Y), ctypes.byref(co) if co is not None else None,
+                              ctypes.byref(cd) if cd is not None else None, ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "qlinear_fwd_ex")
+
+
+def qlinear_bwd_ex(dY: torch.Tensor, A: torch.Tensor, W: torch.Tensor, qdY: QSpec, qA: QSpec, qW: QSpec,
+                   dA: Optional[torch.Tensor], dW: Optional[torch.Tensor], output_dA: Optional[Output] = None,
+                   output_dW: Optional[Output] = None, ws: Optional[torch.Tensor] = None) -> None:
+    """qlinear_bwd with output options for dA and dW."""
+    T, N = dY.shape
+    K = A.shape[1]
+    if ws is None:
+        ws = new_workspace(srq_workspace_bytes(T, N, K), dY.device)
+    c0, c1, c2 = qdY.c(), qA.c(), qW.c()
+    o0, o1 = _opt(output_dA), _opt(output_dW)
+    st = lib().qlinear_bwd_ex(dY.data_ptr(), A.data_ptr(), W.data_ptr(), _dtype_of(dY), T, N, K,
+                              ctypes.byref(c0), ctypes.byref(c1), ctypes.byref(c2), _ptr(dA), _ptr(dW),
+                              ctypes.byref(o0) if o0 is not None else None,
+                              ctypes.byref(o1) if o1 is not None else None, None, None,
+                              ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "qlinear_bwd_ex")
 
 
 def srq_poll_status(ws: torch.Tensor) -> int:

@@ -17,6 +17,34 @@ srq_status_t check_qspec(const srq_qspec_t* q) {
     return SRQ_OK;
 }
 
+// Host-side checks of the output options of a product with an [M, N] result, and their device form.
+srq_status_t make_out_options(const srq_output_t* o, int64_t N, bool have_out, OutOptions* r) {
+    *r = OutOptions();
+    if (!o) return have_out ? SRQ_OK : SRQ_ERR_INVALID_ARG;
+    if (o->accumulate != 0 && o->accumulate != 1) return SRQ_ERR_INVALID_ARG;
+    if (o->accumulate && !have_out) return SRQ_ERR_INVALID_ARG;
+    r->accumulate = o->accumulate;
+    if (o->q) {
+        srq_status_t s = check_qspec(o->q);
+        if (s != SRQ_OK) return s;
+        if (o->q->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;
+        if (!o->step || !o->codes || o->ld_codes < N || ((uintptr_t)o->step % 4) != 0) return SRQ_ERR_INVALID_ARG;
+        r->requant = 1;
+        r->rq_sr = o->q->round == SRQ_SR;
+        r->rq_lim = (float)(((1 << (o->q->bits - 1)) - 1)) * 16777216.0f;
+        r->rq_step = o->step; r->rq_codes = o->codes; r->rq_ld = o->ld_codes;
+        r->rq_offset = o->q->index_offset;
+        r->rq_keys = make_philox_keys(o->q->seed, o->q->tensor_id);
+    } else if (!have_out) {
+        return SRQ_ERR_INVALID_ARG;                       // nothing would be produced
+    }
+    if (o->absmax) {
+        if (((uintptr_t)o->absmax % 4) != 0) return SRQ_ERR_INVALID_ARG;
+        r->absmax_bits = (uint32_t*)o->absmax;
+    }
+    return SRQ_OK;
+}
+
 inline bool aligned_to(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 inline int64_t pitch16(int64_t n) { return (n + 15) / 16 * 16; }
 inline size_t f32_block(int64_t n) { return align_up((size_t)n * 4); }
@@ -52,16 +80,22 @@ LayerPlan plan_layer(const Operand& a, const Operand& b) {
     return p;
 }
 
-srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float* out, const srq_debug_out_t* dbg,
-                       void* ws, size_t ws_bytes, void* cuda_stream) {
+srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float* out, const srq_output_t* oopt,
+                       const srq_debug_out_t* dbg, void* ws, size_t ws_bytes, void* cuda_stream) {
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (!a.x || !b.x || !out || !ws) return SRQ_ERR_INVALID_ARG;
+    if (!a.x || !b.x || !ws) return SRQ_ERR_INVALID_ARG;
+    OutOptions opt;
+    {
+        const srq_status_t so = make_out_options(oopt, b.out_rows(), out != nullptr, &opt);
+        if (so != SRQ_OK) return so;
+    }
     if (dt != SRQ_F32 && dt != SRQ_BF16) return SRQ_ERR_INVALID_ARG;
     if (a.rows < 0 || a.cols < 0 || b.rows < 0 || b.cols < 0) return SRQ_ERR_INVALID_ARG;
     srq_status_t s;
     if ((s = check_qspec(a.q)) != SRQ_OK) return s;
     if ((s = check_qspec(b.q)) != SRQ_OK) return s;
     if (!aligned_to(a.x, 16) || !aligned_to(b.x, 16) || !aligned_to(out, 16) || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
+    if (opt.requant && a.q->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;
     const int64_t M = a.out_rows(), Nn = b.out_rows(), Kc = a.out_cols();
     if (Kc != b.out_cols()) return SRQ_ERR_INVALID_ARG;
     if (a.q->format != b.q->format) return SRQ_ERR_INVALID_ARG;          // one product, one kind of code
@@ -89,6 +123,7 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
             return SRQ_ERR_CUDA;
     }
     if (Kc == 0) {   // empty contraction: the product is zero
+        if (!out || opt.accumulate) return SRQ_OK;
         return cudaMemset2DAsync(out, (size_t)Nn * 4, 0, (size_t)Nn * 4, (size_t)M, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
     }
 
@@ -97,7 +132,7 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
     g.M = M; g.N = Nn; g.Kc = Kc; g.kind = a.q->format == SRQ_GRID_E4M3;
     g.s_row = scales[0]; g.row_stride = a.q->scale == SRQ_PER_ROW;
     g.s_col = scales[1]; g.col_stride = b.q->scale == SRQ_PER_ROW;
-    g.out = out; g.ldo = Nn; g.acc_out = dbg ? dbg->acc : nullptr;
+    g.out = out; g.ldo = Nn; g.acc_out = dbg ? dbg->acc : nullptr; g.opt = opt;
     g.splitk_ws = base + p.off_split; g.splitk_ws_bytes = p.total - p.off_split;
     if ((s = launch_gemm_i8(g, status, st)) != SRQ_OK) return s;
 
@@ -204,9 +239,16 @@ srq_status_t copy_debug(const srq_debug_out_t* dbg, const int8_t* ca, const floa
 
 srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
                      const srq_qspec_t* qdY, const srq_qspec_t* qA, const srq_qspec_t* qW, float* dA, float* dW,
+                     const srq_output_t* o_in, const srq_output_t* o_w,
                      const srq_debug_out_t* dbg_in, const srq_debug_out_t* dbg_w, void* ws, size_t ws_bytes, void* cuda_stream) {
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (!dY || !A || !W || !dA || !dW || !ws) return SRQ_ERR_INVALID_ARG;
+    if (!dY || !A || !W || !ws) return SRQ_ERR_INVALID_ARG;
+    OutOptions opt_in, opt_w;
+    {
+        srq_status_t so = make_out_options(o_in, K, dA != nullptr, &opt_in);
+        if (so == SRQ_OK) so = make_out_options(o_w, K, dW != nullptr, &opt_w);
+        if (so != SRQ_OK) return so;
+    }
     if (dt != SRQ_F32 && dt != SRQ_BF16) return SRQ_ERR_INVALID_ARG;
     if (T < 0 || N < 0 || K < 0) return SRQ_ERR_INVALID_ARG;
     srq_status_t s;
@@ -250,12 +292,12 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
     // dA[T,K] = Q(dY)[T,N] . Q(W)^T[K,N]
     if (T > 0 && K > 0) {
         if (N == 0) {
-            if (cudaMemset2DAsync(dA, (size_t)K * 4, 0, (size_t)K * 4, (size_t)T, st) != cudaSuccess) return SRQ_ERR_CUDA;
+            if (dA && !opt_in.accumulate && cudaMemset2DAsync(dA, (size_t)K * 4, 0, (size_t)K * 4, (size_t)T, st) != cudaSuccess) return SRQ_ERR_CUDA;
         } else {
             GemmArgs g;
             g.a = cd[0]; g.lda = p.pitch_n; g.b = cd[2]; g.ldb = p.pitch_n; g.M = T; g.N = K; g.Kc = N; g.kind = kind;
             g.s_row = sc[0]; g.row_stride = qdY->scale == SRQ_PER_ROW; g.s_col = sc[2]; g.col_stride = qW->scale == SRQ_PER_ROW;
-            g.out = dA; g.ldo = K; g.acc_out = dbg_in ? dbg_in->acc : nullptr;
+            g.out = dA; g.ldo = K; g.acc_out = dbg_in ? dbg_in->acc : nullptr; g.opt = opt_in;
             g.splitk_ws = base + p.off_split[0]; g.splitk_ws_bytes = p.off_split[1] - p.off_split[0];
             if ((s = launch_gemm_i8(g, status, st)) != SRQ_OK) return s;
             if ((s = copy_debug(dbg_in, cd[0], sc[0], T, g.row_stride, cd[2], sc[2], K, g.col_stride, N, p.pitch_n, st)) != SRQ_OK) return s;
@@ -264,12 +306,12 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
     // dW[N,K] = Q(dY)^T[N,T] . Q(A)^T[K,T]
     if (N > 0 && K > 0) {
         if (T == 0) {
-            if (cudaMemset2DAsync(dW, (size_t)K * 4, 0, (size_t)K * 4, (size_t)N, st) != cudaSuccess) return SRQ_ERR_CUDA;
+            if (dW && !opt_w.accumulate && cudaMemset2DAsync(dW, (size_t)K * 4, 0, (size_t)K * 4, (size_t)N, st) != cudaSuccess) return SRQ_ERR_CUDA;
         } else {
             GemmArgs g;
             g.a = cd[1]; g.lda = p.pitch_t; g.b = cd[3]; g.ldb = p.pitch_t; g.M = N; g.N = K; g.Kc = T; g.kind = kind;
             g.s_row = sc[1]; g.row_stride = qdY->scale == SRQ_PER_ROW; g.s_col = sc[3]; g.col_stride = qA->scale == SRQ_PER_ROW;
-            g.out = dW; g.ldo = K; g.acc_out = dbg_w ? dbg_w->acc : nullptr;
+            g.out = dW; g.ldo = K; g.acc_out = dbg_w ? dbg_w->acc : nullptr; g.opt = opt_w;
             g.splitk_ws = base + p.off_split[1]; g.splitk_ws_bytes = p.total - p.off_split[1];
             if ((s = launch_gemm_i8(g, status, st)) != SRQ_OK) return s;
             if ((s = copy_debug(dbg_w, cd[1], sc[1], N, g.row_stride, cd[3], sc[3], K, g.col_stride, T, p.pitch_t, st)) != SRQ_OK) return s;
@@ -378,28 +420,67 @@ srq_status_t qlinear_fwd(const void* A, const void* W, srq_dtype_t dt, int64_t T
                          void* ws, size_t ws_bytes, void* cuda_stream) {
     if (qA && qA->format == SRQ_GRID_NONE) return run_fwd_fp_act(A, W, dt, T, N, K, qW, Y, ws, ws_bytes, cuda_stream);
     const Operand a{A, T, K, false, qA}, b{W, N, K, false, qW};
-    return run_layer(a, b, dt, Y, dbg, ws, ws_bytes, cuda_stream);
+    return run_layer(a, b, dt, Y, nullptr, dbg, ws, ws_bytes, cuda_stream);
 }
 
 srq_status_t qlinear_bwd_input(const void* dY, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
                                const srq_qspec_t* qdY, const srq_qspec_t* qW, float* dA, const srq_debug_out_t* dbg,
                                void* ws, size_t ws_bytes, void* cuda_stream) {
     const Operand a{dY, T, N, false, qdY}, b{W, N, K, true, qW};
-    return run_layer(a, b, dt, dA, dbg, ws, ws_bytes, cuda_stream);
+    return run_layer(a, b, dt, dA, nullptr, dbg, ws, ws_bytes, cuda_stream);
 }
 
 srq_status_t qlinear_bwd_weight(const void* dY, const void* A, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
                                 const srq_qspec_t* qdY, const srq_qspec_t* qA, float* dW, const srq_debug_out_t* dbg,
                                 void* ws, size_t ws_bytes, void* cuda_stream) {
     const Operand a{dY, T, N, true, qdY}, b{A, T, K, true, qA};
-    return run_layer(a, b, dt, dW, dbg, ws, ws_bytes, cuda_stream);
+    return run_layer(a, b, dt, dW, nullptr, dbg, ws, ws_bytes, cuda_stream);
 }
 
 srq_status_t qlinear_bwd(const void* dY, const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
                          const srq_qspec_t* qdY, const srq_qspec_t* qA, const srq_qspec_t* qW, float* dA, float* dW,
                          const srq_debug_out_t* dbg_input, const srq_debug_out_t* dbg_weight,
                          void* ws, size_t ws_bytes, void* cuda_stream) {
-    return run_bwd(dY, A, W, dt, T, N, K, qdY, qA, qW, dA, dW, dbg_input, dbg_weight, ws, ws_bytes, cuda_stream);
+    return run_bwd(dY, A, W, dt, T, N, K, qdY, qA, qW, dA, dW, nullptr, nullptr, dbg_input, dbg_weight, ws, ws_bytes, cuda_stream);
+}
+
+srq_status_t srq_gemm_i8_ex(const int8_t* a, int64_t lda, const int8_t* b, int64_t ldb, int64_t M, int64_t N, int64_t Kc,
+                            const float* s_row, int32_t row_stride, const float* s_col, int32_t col_stride,
+                            float* out, int64_t ldo, int32_t* acc_out, const srq_output_t* output,
+                            void* ws, size_t ws_bytes, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!a || !b || !s_row || !s_col || !ws) return SRQ_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || Kc <= 0 || lda < Kc || ldb < Kc || (out && ldo < N)) return SRQ_ERR_INVALID_ARG;
+    if ((row_stride != 0 && row_stride != 1) || (col_stride != 0 && col_stride != 1)) return SRQ_ERR_INVALID_ARG;
+    if (!aligned_to(a, 16) || !aligned_to(b, 16) || lda % 16 || ldb % 16 || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
+    if ((double)Kc * 127.0 * 127.0 >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
+    if (ws_bytes < sizeof(WsHeader)) return SRQ_ERR_WORKSPACE;
+    GemmArgs g;
+    const srq_status_t so = make_out_options(output, N, out != nullptr, &g.opt);
+    if (so != SRQ_OK) return so;
+    if (M == 0 || N == 0) return SRQ_OK;
+    uint32_t* status = &((WsHeader*)ws)->status;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    g.a = a; g.lda = lda; g.b = b; g.ldb = ldb; g.M = M; g.N = N; g.Kc = Kc; g.kind = 0;
+    g.s_row = s_row; g.row_stride = row_stride; g.s_col = s_col; g.col_stride = col_stride;
+    g.out = out; g.ldo = ldo; g.acc_out = acc_out;
+    g.splitk_ws = (char*)ws + sizeof(WsHeader); g.splitk_ws_bytes = ws_bytes - sizeof(WsHeader);
+    return launch_gemm_i8(g, status, st);
+}
+
+srq_status_t qlinear_fwd_ex(const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
+                            const srq_qspec_t* qA, const srq_qspec_t* qW, float* Y, const srq_output_t* output,
+                            const srq_debug_out_t* dbg, void* ws, size_t ws_bytes, void* cuda_stream) {
+    const Operand a{A, T, K, false, qA}, b{W, N, K, false, qW};
+    return run_layer(a, b, dt, Y, output, dbg, ws, ws_bytes, cuda_stream);
+}
+
+srq_status_t qlinear_bwd_ex(const void* dY, const void* A, const void* W, srq_dtype_t dt, int64_t T, int64_t N, int64_t K,
+                            const srq_qspec_t* qdY, const srq_qspec_t* qA, const srq_qspec_t* qW, float* dA, float* dW,
+                            const srq_output_t* output_dA, const srq_output_t* output_dW,
+                            const srq_debug_out_t* dbg_input, const srq_debug_out_t* dbg_weight,
+                            void* ws, size_t ws_bytes, void* cuda_stream) {
+    return run_bwd(dY, A, W, dt, T, N, K, qdY, qA, qW, dA, dW, output_dA, output_dW, dbg_input, dbg_weight, ws, ws_bytes, cuda_stream);
 }
 
 srq_status_t srq_poll_status(void* ws, void* cuda_stream) {

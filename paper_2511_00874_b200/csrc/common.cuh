@@ -93,6 +93,19 @@ cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, 
 // ------------------------------------------------------------------------------------------
 // int8 GEMM (gemm_i8.cu)
 // ------------------------------------------------------------------------------------------
+// What else a product does with its results (all optional).
+struct OutOptions {
+    int32_t accumulate = 0;          // out += result instead of out = result
+    int32_t requant = 0;             // also write Q(result) as int8 codes with a given step size
+    int32_t rq_sr = 0;               // stochastic rounding (else round to nearest)
+    float rq_lim = 0.0f;             // qmax * 2^24: saturation bound of the fixed-point quotient
+    const float* rq_step = nullptr;  // device [1]
+    int8_t* rq_codes = nullptr; int64_t rq_ld = 0;
+    uint64_t rq_offset = 0;          // flat index of result [0, 0] in the threshold stream
+    PhiloxKeys rq_keys = {};
+    uint32_t* absmax_bits = nullptr; // device [1]: raised to the bit pattern of max |result|
+};
+
 struct GemmArgs {
     const int8_t* a; int64_t lda; const int8_t* b; int64_t ldb;
     int64_t M, N, Kc;
@@ -100,6 +113,7 @@ struct GemmArgs {
                                                 // 2: bfloat16 operands, binary32 sums (Kc, lda, ldb in BYTES)
     const float* s_row; int32_t row_stride; const float* s_col; int32_t col_stride;
     float* out; int64_t ldo; int32_t* acc_out;
+    OutOptions opt;
     void* splitk_ws; size_t splitk_ws_bytes;   // int32 [M,N] partial sums
 };
 size_t gemm_splitk_bytes(int64_t M, int64_t N);

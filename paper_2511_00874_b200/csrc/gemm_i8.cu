@@ -282,7 +282,68 @@ struct GemmParams {
     int32_t vec_out;           // 16-byte stores to out allowed
     int32_t tma_out;           // out is written with TMA stores (map_out valid, no acc_out)
     int32_t tma_part;          // partial sums are added with TMA reductions (map_part valid)
+    int32_t write_out;         // out is wanted (it may be left out when only codes are)
+    int32_t rq_vec;            // 16-byte stores of codes allowed
+    OutOptions opt;
 };
+
+// Re-quantization of 32 consecutive results of one row (columns col0 .. col0 + 31) with the
+// caller's step size, saturating, by the quantizer's fixed-point rule; and their absmax.
+// o holds binary32 bit patterns.  Thresholds follow the flat index rq_offset + row * N + col.
+__device__ __forceinline__ void output_options(const GemmParams& P, const uint32_t (&o)[32], int64_t row, int64_t col0,
+                                               float rq_inv, uint32_t& amax) {
+    if (row >= P.M || col0 >= P.N) return;
+    if (P.opt.absmax_bits) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (col0 + i < P.N) amax = max(amax, o[i] & 0x7FFFFFFFu);
+    }
+    if (!P.opt.requant) return;
+    const uint64_t i0 = P.opt.rq_offset + (uint64_t)row * (uint64_t)P.N + (uint64_t)col0;
+    const bool aligned = (i0 & 3u) == 0;
+    const float lim = P.opt.rq_lim;
+    uint32_t words[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        uint32_t rnd[4] = {0u, 0u, 0u, 0u};
+        if (P.opt.rq_sr) {
+            if (aligned) {
+                const uint64_t jb = (i0 >> 2) + q;
+                philox_rounds((uint32_t)jb, (uint32_t)(jb >> 32), P.opt.rq_keys, rnd);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint64_t ie = i0 + 4 * q + e, jb = ie >> 2;
+                    uint32_t w[4];
+                    philox_rounds((uint32_t)jb, (uint32_t)(jb >> 32), P.opt.rq_keys, w);
+                    const uint32_t sel = (uint32_t)ie & 3u;
+                    rnd[e] = sel == 0 ? w[0] : sel == 1 ? w[1] : sel == 2 ? w[2] : w[3];
+                }
+            }
+        }
+        uint32_t sums[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float s = __fmul_rn(__fmul_rn(__uint_as_float(o[4 * q + e]), rq_inv), 16777216.0f);
+            s = fminf(fmaxf(s, -lim), lim);                                  // saturation
+            if (P.opt.rq_sr) {
+                asm("mad.hi.u32 %0, %1, 16777216, %2;" : "=r"(sums[e]) : "r"(~rnd[e]), "r"((uint32_t)__float2int_ru(s)));
+            } else {
+                sums[e] = (uint32_t)__float2int_rd(s) + 0x00800000u;
+            }
+        }
+        words[q] = __byte_perm(__byte_perm(sums[0], sums[1], 0x0073), __byte_perm(sums[2], sums[3], 0x0073), 0x5410);
+    }
+    int8_t* dst = P.opt.rq_codes + row * P.opt.rq_ld + col0;
+    if (P.rq_vec && col0 + 32 <= P.N) {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(words[0], words[1], words[2], words[3]);
+        *reinterpret_cast<uint4*>(dst + 16) = make_uint4(words[4], words[5], words[6], words[7]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (col0 + i < P.N) dst[i] = (int8_t)((words[i >> 2] >> (8 * (i & 3))) & 0xFF);
+    }
+}
 
 template <int STAGES>
 __device__ __forceinline__ void give_up(SharedTail<STAGES>* T, uint32_t* status) {
@@ -408,6 +469,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // the MMA issuer's barriers (in the leader CTA)
         const uint32_t empty_bar0 = CTAS == 1 ? smem_u32(&T->tmem_empty[0]) : map_to_cta(smem_u32(&T->tmem_empty[0]), 0);
         const uint32_t empty_bar1 = CTAS == 1 ? smem_u32(&T->tmem_empty[1]) : map_to_cta(smem_u32(&T->tmem_empty[1]), 0);
+        float rq_inv = 0.0f;                                  // reciprocal of the caller's step size
+        if (P.opt.requant) {
+            const float d = *P.opt.rq_step;
+            rq_inv = d == 0.0f ? 0.0f : __fdiv_rn(1.0f, d);
+            if (!(fabsf(rq_inv) <= 3.402823466e38f)) rq_inv = 0.0f;
+        }
+        uint32_t amax = 0u;
         uint32_t lt = 0;
         bool ok = true;
         for (int64_t u = group; u < units && ok; u += groups, ++lt) {
@@ -449,13 +517,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         v[4 * q + 2] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 2]), __fmul_rn(sr, c4.z)));
                         v[4 * q + 3] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 3]), __fmul_rn(sr, c4.w)));
                     }
+                    const int32_t col0 = (int32_t)col_base + j * 32;
+                    output_options(P, v, row, col0, rq_inv, amax);
                     if (lane == 0) bulk_wait_read();          // the previous block has left the staging buffer
                     __syncwarp();
                     stage_block(stage, lane, v);
                     fence_async_smem();
                     __syncwarp();
-                    const int32_t col0 = (int32_t)col_base + j * 32;
-                    if (lane == 0 && wrow < P.M && col0 < P.N) { tma_store_2d(&map_out, stage, col0, wrow); bulk_commit(); }
+                    if (lane == 0 && wrow < P.M && col0 < P.N) {
+                        if (P.opt.accumulate) tma_reduce_add_2d(&map_out, stage, col0, wrow);   // binary32 adds in memory
+                        else tma_store_2d(&map_out, stage, col0, wrow);
+                        bulk_commit();
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -468,29 +541,36 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     tmem_ld_wait();
                     const int64_t col0 = col_base + j * 32;
                     if (row < P.M && col0 < P.N) {
-                        float* dst = P.out + row * P.ldo + col0;
                         const float* sc = &T->s_col[buf][j * 32];
-                        if (P.vec_out && col0 + 32 <= P.N) {
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                const float4 c4 = *reinterpret_cast<const float4*>(sc + 4 * q);
-                                float4 o;
-                                o.x = __fmul_rn(acc_to_float<KIND>(v[4 * q + 0]), __fmul_rn(sr, c4.x));
-                                o.y = __fmul_rn(acc_to_float<KIND>(v[4 * q + 1]), __fmul_rn(sr, c4.y));
-                                o.z = __fmul_rn(acc_to_float<KIND>(v[4 * q + 2]), __fmul_rn(sr, c4.z));
-                                o.w = __fmul_rn(acc_to_float<KIND>(v[4 * q + 3]), __fmul_rn(sr, c4.w));
-                                __stcs(reinterpret_cast<float4*>(dst + 4 * q), o);
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (col0 + i < P.N) dst[i] = __fmul_rn(acc_to_float<KIND>(v[i]), __fmul_rn(sr, sc[i]));
-                        }
                         if (P.acc_out) {
                             int32_t* ad = P.acc_out + row * P.N + col0;
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
                                 if (col0 + i < P.N) ad[i] = (int32_t)v[i];
+                        }
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            v[i] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[i]), __fmul_rn(sr, sc[i])));
+                        output_options(P, v, row, col0, rq_inv, amax);
+                        if (P.write_out) {
+                            float* dst = P.out + row * P.ldo + col0;
+                            if (P.vec_out && col0 + 32 <= P.N) {
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) {
+                                    float4 o = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                                           __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                                    if (P.opt.accumulate) {
+                                        const float4 p = *reinterpret_cast<const float4*>(dst + 4 * q);
+                                        o.x = __fadd_rn(p.x, o.x); o.y = __fadd_rn(p.y, o.y); o.z = __fadd_rn(p.z, o.z); o.w = __fadd_rn(p.w, o.w);
+                                    }
+                                    __stcs(reinterpret_cast<float4*>(dst + 4 * q), o);
+                                }
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (col0 + i < P.N)
+                                        dst[i] = P.opt.accumulate ? __fadd_rn(dst[i], __uint_as_float(v[i])) : __uint_as_float(v[i]);
+                            }
                         }
                     }
                 }
@@ -524,6 +604,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             }
         }
+        if (P.opt.absmax_bits) {      // absmax of everything this warp produced: one guarded atomic
+            amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+            if (lane == 0 && amax > __ldcg(P.opt.absmax_bits)) atomicMax(P.opt.absmax_bits, amax);
+        }
     }
 
     if (warp >= 2 && lane == 0) bulk_wait_all();      // stores still reading the staging buffers
@@ -543,7 +627,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 __global__ void __launch_bounds__(256)
 dequant_kernel(const int32_t* __restrict__ part, int64_t M, int64_t N, const float* __restrict__ s_row, int32_t row_stride,
                const float* __restrict__ s_col, int32_t col_stride, float* __restrict__ out, int64_t ldo,
-               int32_t* __restrict__ acc_out, int vec) {
+               int32_t* __restrict__ acc_out, int vec, int accumulate) {
     const int64_t nq = (N + 3) / 4;                      // groups of four columns per row
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < M * nq; g += (int64_t)gridDim.x * blockDim.x) {
         const int64_t r = g / nq, c = (g % nq) * 4;
@@ -555,12 +639,17 @@ dequant_kernel(const int32_t* __restrict__ part, int64_t M, int64_t N, const flo
             o.y = __fmul_rn(__int2float_rn(a.y), __fmul_rn(sr, s_col[(c + 1) * col_stride]));
             o.z = __fmul_rn(__int2float_rn(a.z), __fmul_rn(sr, s_col[(c + 2) * col_stride]));
             o.w = __fmul_rn(__int2float_rn(a.w), __fmul_rn(sr, s_col[(c + 3) * col_stride]));
+            if (accumulate) {
+                const float4 p = *reinterpret_cast<const float4*>(out + r * ldo + c);
+                o.x = __fadd_rn(p.x, o.x); o.y = __fadd_rn(p.y, o.y); o.z = __fadd_rn(p.z, o.z); o.w = __fadd_rn(p.w, o.w);
+            }
             *reinterpret_cast<float4*>(out + r * ldo + c) = o;
             if (acc_out) *reinterpret_cast<int4*>(acc_out + r * N + c) = a;
         } else {
             for (int e = 0; e < 4 && c + e < N; ++e) {
                 const int32_t a = __ldcg(part + r * N + c + e);
-                out[r * ldo + c + e] = __fmul_rn(__int2float_rn(a), __fmul_rn(sr, s_col[(c + e) * col_stride]));
+                const float o = __fmul_rn(__int2float_rn(a), __fmul_rn(sr, s_col[(c + e) * col_stride]));
+                out[r * ldo + c + e] = accumulate ? __fadd_rn(out[r * ldo + c + e], o) : o;
                 if (acc_out) acc_out[r * N + c + e] = a;
             }
         }
@@ -696,7 +785,8 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.tiles_n = (int32_t)((g.N + BN - 1) / BN);
     const int64_t tiles = (int64_t)P.tiles_m * P.tiles_n;
     // binary32 accumulators do not add exactly: the E4M3 product is never split
-    P.splits = g.kind == 0 ? choose_splits(tiles, P.num_kb, groups_max) : 1;
+    // nor is a product whose results are re-quantized or whose absmax is wanted (done in the epilogue)
+    P.splits = (g.kind == 0 && !g.opt.requant && !g.opt.absmax_bits) ? choose_splits(tiles, P.num_kb, groups_max) : 1;
     P.part = nullptr;
     if (P.splits > 1) {
         const size_t part_bytes = align_up((size_t)g.M * g.N * 4);
@@ -711,11 +801,14 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.s_col = g.s_col; P.col_stride = g.col_stride;
     P.out = g.out; P.ldo = g.ldo; P.acc_out = g.acc_out;
     P.status = status;
-    P.vec_out = ((uintptr_t)g.out % 16 == 0) && (g.ldo % 4 == 0);
+    P.vec_out = g.out && ((uintptr_t)g.out % 16 == 0) && (g.ldo % 4 == 0);
 
     // results leave through TMA stores when the output (and the partial sums) meet the 16-byte rules
     CUtensorMap map_out = map_a, map_part = map_a;       // placeholders when unused
-    P.tma_out = P.vec_out && !g.acc_out && g.M < (1ll << 31) && g.N < (1ll << 31) &&
+    P.opt = g.opt;
+    P.write_out = g.out != nullptr;
+    P.rq_vec = g.opt.requant && ((uintptr_t)g.opt.rq_codes % 16 == 0) && (g.opt.rq_ld % 16 == 0);
+    P.tma_out = P.write_out && P.vec_out && !g.acc_out && g.M < (1ll << 31) && g.N < (1ll << 31) &&
                 encode_output(&map_out, g.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.M, g.N, g.ldo);
     P.tma_part = P.splits > 1 && g.N % 4 == 0 && g.M < (1ll << 31) && g.N < (1ll << 31) &&
                  encode_output(&map_part, P.part, CU_TENSOR_MAP_DATA_TYPE_INT32, g.M, g.N, g.N);
@@ -737,7 +830,7 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
         const int64_t blocks = (work + 255) / 256;
         const unsigned grid = (unsigned)(blocks < 8 * (int64_t)dev->sms ? blocks : 8 * (int64_t)dev->sms);
         dequant_kernel<<<grid, 256, 0, stream>>>(P.part, g.M, g.N, g.s_row, g.row_stride, g.s_col, g.col_stride, g.out, g.ldo,
-                                                 g.acc_out, vec);
+                                                 g.acc_out, vec, g.opt.accumulate);
         ++g_launches;
         if (cudaGetLastError() != cudaSuccess) return SRQ_ERR_CUDA;
     }
