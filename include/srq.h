@@ -90,6 +90,11 @@ typedef struct {
     uint64_t seed;         /* Philox key; one per training step */
     uint64_t tensor_id;    /* Philox counter words 2-3; one per (layer, operand, pass) */
     uint64_t index_offset; /* added to the flat index; first_row*cols for a row shard */
+    const float *absmax;   /* optional, DEVICE pointer to one float: max |x| of the operand when the
+                            * caller already knows it (srq_absmax, or an all-reduced maximum over
+                            * token shards).  The absmax pass over the operand is then skipped.  Only
+                            * with SRQ_PER_TENSOR.  The value must not be smaller than the true
+                            * maximum (codes are unspecified otherwise).  NULL: compute it. */
 } srq_qspec_t;
 
 /* Optional copies of what a layer pass fed to its product: dense code matrices in the layout
@@ -153,6 +158,12 @@ srq_status_t sr_quantize_static(const void *x, srq_dtype_t dt, int64_t rows, int
                                 int8_t *codes_rm, int64_t ld_rm, float *scale_rm,
                                 int8_t *codes_tr, int64_t ld_tr, float *scale_tr,
                                 uint32_t *device_status, void *cuda_stream);
+
+/* max |x| over x[rows, cols] (row pitch ld elements) into *absmax (device, one float), e.g. to
+ * share it between the forward and the backward quantization point of the same tensor, or to
+ * all-reduce it over token shards, through srq_qspec_t.absmax.  Needs no workspace. */
+srq_status_t srq_absmax(const void *x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+                        float *absmax, void *cuda_stream);
 
 /*
  * The product of two quantized matrices (mixed-precision matmul subsection): int8 codes

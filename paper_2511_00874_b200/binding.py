@@ -26,7 +26,7 @@ SR, RTN = 0, 1
 GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
-           "sr_quantize", "sr_quantize_static", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
+           "sr_quantize", "sr_quantize_static", "srq_absmax", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
            "srq_gemm_i8_ex", "qlinear_fwd_ex", "qlinear_bwd_ex",
            "srq_poll_status", "srq_status_string", "srq_launch_count"]
 
@@ -40,7 +40,8 @@ class SrqError(RuntimeError):
 class _QSpec(ctypes.Structure):
     _fields_ = [("bits", ctypes.c_int32), ("scale", ctypes.c_int32), ("round", ctypes.c_int32),
                 ("format", ctypes.c_int32), ("seed", ctypes.c_uint64),
-                ("tensor_id", ctypes.c_uint64), ("index_offset", ctypes.c_uint64)]
+                ("tensor_id", ctypes.c_uint64), ("index_offset", ctypes.c_uint64),
+                ("absmax", ctypes.c_void_p)]
 
 
 class _DebugOut(ctypes.Structure):
@@ -65,10 +66,11 @@ class QSpec:
     tensor_id: int = 0
     index_offset: int = 0
     format: int = GRID_INT
+    absmax: Optional[torch.Tensor] = None      # device float tensor of one element: known max |x| (per tensor)
 
     def c(self) -> _QSpec:
         return _QSpec(self.bits, self.scale, self.round, self.format, self.seed, self.tensor_id,
-                      self.index_offset)
+                      self.index_offset, None if self.absmax is None else self.absmax.data_ptr())
 
 
 _lib: Optional[ctypes.CDLL] = None
@@ -94,6 +96,8 @@ def lib() -> ctypes.CDLL:
     L.srq_workspace_bytes.restype = sz
     L.sr_quantize.argtypes = [vp, ctypes.c_int, i64, i64, i64, qp, vp, i64, vp, vp, i64, vp, vp, sz, vp]
     L.sr_quantize.restype = ctypes.c_int
+    L.srq_absmax.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, vp]
+    L.srq_absmax.restype = ctypes.c_int
     L.sr_quantize_static.argtypes = [vp, ctypes.c_int, i64, i64, i64, qp, vp, i64, vp, vp, i64, vp, vp, vp]
     L.sr_quantize_static.restype = ctypes.c_int
     L.srq_gemm_i8.argtypes = [vp, i64, vp, i64, i64, i64, i64, vp, i32, vp, i32, vp, i64, vp, vp, sz, vp]
@@ -189,6 +193,13 @@ def sr_quantize(x: torch.Tensor, q: QSpec, codes_rm: Optional[torch.Tensor] = No
                            _ptr(codes_tr), codes_tr.stride(0) if codes_tr is not None else 0,
                            _ptr(scale_tr), ws.data_ptr(), ws.numel(), _stream())
     _check(st, "sr_quantize")
+
+
+def srq_absmax(x: torch.Tensor, absmax: torch.Tensor) -> None:
+    """max |x| into the one-element float32 CUDA tensor ``absmax``."""
+    _dev2d(x, "x")
+    st = lib().srq_absmax(x.data_ptr(), _dtype_of(x), x.shape[0], x.shape[1], x.stride(0), absmax.data_ptr(), _stream())
+    _check(st, "srq_absmax")
 
 
 def sr_quantize_static(x: torch.Tensor, q: QSpec, codes_rm: Optional[torch.Tensor] = None,

@@ -86,6 +86,9 @@ struct QuantArgs {
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& scratch, uint32_t* status,
                             cudaStream_t stream);
 
+// max |x| of the whole matrix into *absmax (device float, overwritten).
+cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax, cudaStream_t stream);
+
 // int8 codes as bfloat16 integers (pitches in elements); *one receives 1.0f.
 cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, int64_t ld, void* out_bf16, int64_t ld_out,
                                float* one, cudaStream_t stream);

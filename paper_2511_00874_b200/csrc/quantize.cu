@@ -615,6 +615,15 @@ cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, 
     return cudaGetLastError();
 }
 
+cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax, cudaStream_t stream) {
+    cudaError_t e = cudaMemsetAsync(absmax, 0, sizeof(float), stream);
+    if (e != cudaSuccess || rows == 0 || cols == 0) return e;
+    if (dt == SRQ_F32) launch_amax<float>(x, rows, cols, ld, (uint32_t*)absmax, false, nullptr, false, stream);
+    else launch_amax<__nv_bfloat16>(x, rows, cols, ld, (uint32_t*)absmax, false, nullptr, false, stream);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream) {
     const bool want_rm = a.codes_rm != nullptr, want_tr = a.codes_tr != nullptr;
     const bool per_row = a.q.scale == SRQ_PER_ROW;
@@ -632,11 +641,13 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     float* inv_rm = s.inv_rm;
     float* inv_tr = per_row ? s.inv_tr : s.inv_rm;
 
-    cudaError_t e = cudaMemsetAsync(s.amax_rm, 0, (size_t)((char*)s.inv_rm - (char*)s.amax_rm), stream);
-    if (e != cudaSuccess) return e;
-
     const bool vec_in = ((uintptr_t)a.x % (4 * esize) == 0) && (a.ld % 4 == 0);
-    {
+    const bool given = a.q.absmax != nullptr && !per_row;   // a known absmax is only taken per tensor
+    if (given) {
+        amax_rm = amax_tr = (uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
+    } else {
+        cudaError_t e = cudaMemsetAsync(s.amax_rm, 0, (size_t)((char*)s.inv_rm - (char*)s.amax_rm), stream);
+        if (e != cudaSuccess) return e;
         const bool want_rows = per_row && want_rm, want_cols = per_row && want_tr;
         if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, stream);
         else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, stream);

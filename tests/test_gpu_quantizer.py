@@ -154,3 +154,32 @@ def test_unbiasedness_of_1e4_draws_on_the_gpu():
         srq.sr_quantize(x, srq.QSpec(8, 0, 0, seed, 3), c, s, ws=ws)
         ref = oracle.sr_quantize(xs, oracle.QSpec(8, 0, 0, seed, 3))[0]
         assert np.array_equal(c.cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_absmax_entry_point_and_a_known_absmax(dtype):
+    """srq_absmax equals the plain maximum; a quantization point that carries it skips its own
+    absmax pass and gives the same codes and step size (also a larger, all-reduced-like maximum
+    works: then the oracle is given a tensor whose maximum is that value)."""
+    x = synth.with_outliers((300, 388), seed=8, dtype=dtype, device="cuda")
+    m = torch.full((1,), -1.0, device="cuda")
+    srq.srq_absmax(x, m)
+    assert m.item() == x.float().abs().max().item()
+    srq.srq_absmax(x[:, 8:209], m)                       # strided view (16-byte aligned start), ragged width
+    assert m.item() == x[:, 8:209].float().abs().max().item()
+    srq.srq_absmax(x, m)
+    for rnd in (srq.SR, srq.RTN):
+        a = _run_gpu(x, srq.QSpec(8, srq.PER_TENSOR, rnd, 3, 4))
+        b = _run_gpu(x, srq.QSpec(8, srq.PER_TENSOR, rnd, 3, 4, absmax=m))
+        for g, r in zip(a, b):
+            assert np.array_equal(g, r)
+    # a maximum larger than this tensor's own (as after a maximum over several shards)
+    big = torch.tensor([m.item() * 1.7], device="cuda")
+    got = _run_gpu(x, srq.QSpec(6, srq.PER_TENSOR, srq.SR, 3, 4, absmax=big))
+    xs = torch.cat([x.float().cpu(), torch.tensor([[big.item()] + [0.0] * 387])], 0).numpy()   # same maximum for the oracle
+    ref = oracle.sr_quantize(xs, oracle.QSpec(6, 0, 0, 3, 4), True, True)
+    assert np.array_equal(got[0], ref[0][:300]) and np.array_equal(got[1], ref[1])
+    assert np.array_equal(got[2], ref[2][:, :300])
+    with pytest.raises(srq.SrqError):                    # only with one step size per tensor
+        srq.sr_quantize(x, srq.QSpec(8, srq.PER_ROW, absmax=m), torch.empty((300, 388), dtype=torch.int8, device="cuda"),
+                        torch.empty(300, device="cuda"))
