@@ -271,17 +271,17 @@ __device__ __forceinline__ float acc_to_float(uint32_t v) {
 struct GemmParams {
     int64_t M, N;
     int32_t num_kb;            // 128-byte blocks along the contraction
-    int32_t splits;            // parts the contraction is cut into (1 = none)
+    int32_t splits;            // parts the contraction of the LAST tiles is cut into (1 = none)
+    int32_t full_tiles;        // tiles [0, full_tiles) are not split; the rest are, their sums going to `part`
     int32_t tiles_m, tiles_n;  // tiles of (128 * CTAS) x 256
     const float* s_row; int32_t row_stride;
     const float* s_col; int32_t col_stride;
     float* out; int64_t ldo;
     int32_t* acc_out;          // optional raw sums [M, N]
-    int32_t* part;             // split contraction: zeroed int32 [M, N]
+    int32_t* part;             // split tiles: zeroed int32 [(tiles - full_tiles) * 128 * CTAS, 256], tile after tile
     uint32_t* status;
     int32_t vec_out;           // 16-byte stores to out allowed
     int32_t tma_out;           // out is written with TMA stores (map_out valid, no acc_out)
-    int32_t tma_part;          // partial sums are added with TMA reductions (map_part valid)
     int32_t write_out;         // out is wanted (it may be left out when only codes are)
     int32_t rq_vec;            // 16-byte stores of codes allowed
     OutOptions opt;
@@ -382,8 +382,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t tmem_base = T->tmem_base;
 
     const int64_t groups = gridDim.x / CTAS, group = blockIdx.x / CTAS;   // a group = the CTAs of one tile
-    const int64_t units = (int64_t)P.tiles_m * P.tiles_n * P.splits;
+    // work units: the first full_tiles tiles whole, then every remaining tile in `splits` parts
+    const int64_t tiles_all = (int64_t)P.tiles_m * P.tiles_n;
+    const int64_t units = P.full_tiles + (tiles_all - P.full_tiles) * P.splits;
     const int32_t kb_per_split = (P.num_kb + P.splits - 1) / P.splits;
+    auto decode = [&](int64_t u, int64_t& tile, int32_t& kb0, int32_t& kb1) {
+        if (u < P.full_tiles) { tile = u; kb0 = 0; kb1 = P.num_kb; return; }
+        const int64_t v = u - P.full_tiles;
+        tile = P.full_tiles + v / P.splits;
+        kb0 = (int32_t)(v % P.splits) * kb_per_split;
+        kb1 = min(kb0 + kb_per_split, P.num_kb);
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -393,11 +402,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t it = 0;
             bool ok = true;
             for (int64_t u = group; u < units && ok; u += groups) {
-                const int32_t split = (int32_t)(u % P.splits);
-                const int64_t tile = u / P.splits;
+                int64_t tile; int32_t kb0, kb1;
+                decode(u, tile, kb0, kb1);
                 const int32_t tn = (int32_t)(tile % P.tiles_n), tm = (int32_t)(tile / P.tiles_n);
-                const int32_t kb0 = split * kb_per_split;
-                const int32_t kb1 = min(kb0 + kb_per_split, P.num_kb);
                 const int32_t row_a = (tm * CTAS + (int32_t)rank) * BM;
                 const int32_t row_b = tn * BN + (int32_t)rank * C::B_ROWS;
                 for (int32_t kb = kb0; kb < kb1; ++kb, ++it) {
@@ -433,9 +440,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t it = 0, lt = 0;
             bool ok = true;
             for (int64_t u = group; u < units && ok; u += groups, ++lt) {
-                const int32_t split = (int32_t)(u % P.splits);
-                const int32_t kb0 = split * kb_per_split;
-                const int32_t kb1 = min(kb0 + kb_per_split, P.num_kb);
+                int64_t tile; int32_t kb0, kb1;
+                decode(u, tile, kb0, kb1);
                 const uint32_t buf = lt & 1u, use = lt >> 1;
                 if (!mbar_wait(&T->tmem_empty[buf], (use & 1u) ^ 1u, &T->abort_flag)) { give_up(T, P.status); ok = false; break; }
                 tc_fence_after();
@@ -479,7 +485,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t lt = 0;
         bool ok = true;
         for (int64_t u = group; u < units && ok; u += groups, ++lt) {
-            const int64_t tile = u / P.splits;
+            int64_t tile; int32_t kb0_unused, kb1_unused;
+            decode(u, tile, kb0_unused, kb1_unused);
+            const bool whole = u < P.full_tiles;              // this unit holds the complete sums of its tile
             const int32_t tn = (int32_t)(tile % P.tiles_n), tm = (int32_t)(tile / P.tiles_n);
             const uint32_t buf = lt & 1u, use = lt >> 1;
             const int64_t row0 = ((int64_t)tm * CTAS + rank) * BM;      // first row of this CTA's half
@@ -501,7 +509,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
             const uint32_t stage = smem_u32(out_stage + (warp - 2) * OUT_STAGE_BYTES);
             const int32_t wrow = (int32_t)(row0 + quarter * 32);           // first row of this warp's blocks
-            if (P.splits == 1 && P.tma_out) {
+            if (whole && P.tma_out) {
                 // registers -> swizzled shared-memory block -> one TMA store per 32 x 32 block
 #pragma unroll 1
                 for (int j = 0; j < BN / 32; ++j) {
@@ -533,7 +541,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
-            } else if (P.splits == 1) {
+            } else if (whole) {
 #pragma unroll 1
                 for (int j = 0; j < BN / 32; ++j) {
                     uint32_t v[32];
@@ -578,26 +586,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             } else {
-                // exact partial sums: integer adds commute, so any arrival order gives the same total
+                // exact partial sums: integer adds commute, so any arrival order gives the same total.
+                // `part` holds the split tiles one after another, 128 * CTAS rows of 256 sums each.
+                const int32_t prow = (int32_t)((tile - P.full_tiles) * (BM * CTAS) + rank * BM + quarter * 32);
 #pragma unroll 1
                 for (int j = 0; j < BN / 32; ++j) {
                     uint32_t v[32];
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
-                    const int64_t col0 = col_base + j * 32;
-                    if (P.tma_part) {
-                        if (lane == 0) bulk_wait_read();
-                        __syncwarp();
-                        stage_block(stage, lane, v);
-                        fence_async_smem();
-                        __syncwarp();
-                        if (lane == 0 && wrow < P.M && col0 < P.N) { tma_reduce_add_2d(&map_part, stage, (int32_t)col0, wrow); bulk_commit(); }
-                    } else if (row < P.M && col0 < P.N) {
-                        int32_t* pd = P.part + row * P.N + col0;
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (col0 + i < P.N) atomicAdd(pd + i, (int32_t)v[i]);
-                    }
+                    if (lane == 0) bulk_wait_read();
+                    __syncwarp();
+                    stage_block(stage, lane, v);
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) { tma_reduce_add_2d(&map_part, stage, j * 32, prow); bulk_commit(); }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -623,36 +625,41 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
-// Second step of a split contraction: out = float(sum) * (s_row * s_col) over the finished sums.
+// Second step of a split contraction: out = float(sum) * (s_row * s_col) over the finished sums of the
+// split tiles.  `part` holds them tile after tile ([tile_rows, 256] each); tile t of it is output tile
+// first_tile + t in row-major tile order.  One thread per four consecutive columns.
 __global__ void __launch_bounds__(256)
-dequant_kernel(const int32_t* __restrict__ part, int64_t M, int64_t N, const float* __restrict__ s_row, int32_t row_stride,
+dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_tile, int32_t tiles_n, int32_t tile_rows,
+               int64_t M, int64_t N, const float* __restrict__ s_row, int32_t row_stride,
                const float* __restrict__ s_col, int32_t col_stride, float* __restrict__ out, int64_t ldo,
                int32_t* __restrict__ acc_out, int vec, int accumulate) {
-    const int64_t nq = (N + 3) / 4;                      // groups of four columns per row
-    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < M * nq; g += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = g / nq, c = (g % nq) * 4;
+    const int64_t per_tile = (int64_t)tile_rows * (BN / 4);
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_tiles * per_tile; g += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t t = g / per_tile, in_tile = g % per_tile;
+        const int64_t tile = first_tile + t;
+        const int64_t r = (tile / tiles_n) * tile_rows + in_tile / (BN / 4);
+        const int64_t c = (tile % tiles_n) * BN + (in_tile % (BN / 4)) * 4;
+        if (r >= M || c >= N) continue;
+        const int4 a = __ldcg(reinterpret_cast<const int4*>(part + g * 4));
+        const int32_t av[4] = {a.x, a.y, a.z, a.w};
         const float sr = s_row[r * row_stride];
-        if (vec) {
-            const int4 a = __ldcg(reinterpret_cast<const int4*>(part + r * N + c));
-            float4 o;
-            o.x = __fmul_rn(__int2float_rn(a.x), __fmul_rn(sr, s_col[(c + 0) * col_stride]));
-            o.y = __fmul_rn(__int2float_rn(a.y), __fmul_rn(sr, s_col[(c + 1) * col_stride]));
-            o.z = __fmul_rn(__int2float_rn(a.z), __fmul_rn(sr, s_col[(c + 2) * col_stride]));
-            o.w = __fmul_rn(__int2float_rn(a.w), __fmul_rn(sr, s_col[(c + 3) * col_stride]));
+        float o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            o[e] = (c + e < N) ? __fmul_rn(__int2float_rn(av[e]), __fmul_rn(sr, s_col[(c + e) * col_stride])) : 0.0f;
+        float* dst = out + r * ldo + c;
+        if (vec && c + 4 <= N) {
+            float4 w = make_float4(o[0], o[1], o[2], o[3]);
             if (accumulate) {
-                const float4 p = *reinterpret_cast<const float4*>(out + r * ldo + c);
-                o.x = __fadd_rn(p.x, o.x); o.y = __fadd_rn(p.y, o.y); o.z = __fadd_rn(p.z, o.z); o.w = __fadd_rn(p.w, o.w);
+                const float4 p = *reinterpret_cast<const float4*>(dst);
+                w.x = __fadd_rn(p.x, w.x); w.y = __fadd_rn(p.y, w.y); w.z = __fadd_rn(p.z, w.z); w.w = __fadd_rn(p.w, w.w);
             }
-            *reinterpret_cast<float4*>(out + r * ldo + c) = o;
-            if (acc_out) *reinterpret_cast<int4*>(acc_out + r * N + c) = a;
+            *reinterpret_cast<float4*>(dst) = w;
         } else {
-            for (int e = 0; e < 4 && c + e < N; ++e) {
-                const int32_t a = __ldcg(part + r * N + c + e);
-                const float o = __fmul_rn(__int2float_rn(a), __fmul_rn(sr, s_col[(c + e) * col_stride]));
-                out[r * ldo + c + e] = accumulate ? __fadd_rn(out[r * ldo + c + e], o) : o;
-                if (acc_out) acc_out[r * N + c + e] = a;
-            }
+            for (int e = 0; e < 4 && c + e < N; ++e) dst[e] = accumulate ? __fadd_rn(dst[e], o[e]) : o[e];
         }
+        if (acc_out)
+            for (int e = 0; e < 4 && c + e < N; ++e) acc_out[r * N + c + e] = av[e];
     }
 }
 
@@ -733,26 +740,30 @@ static bool device_info(DeviceInfo** out) {
     return true;
 }
 
-// Parts the contraction is cut into when there are too few tiles to fill the machine (`groups`
-// tiles run at a time).
-static int choose_splits(int64_t tiles, int32_t num_kb, int groups) {
-    if (num_kb < 16) return 1;
-    int s = 1;
-    if (tiles * 2 <= groups) {
-        s = (int)(groups / tiles);
-    }
-    const int max_by_k = num_kb / 8;                        // keep at least 8 k-blocks per part
-    if (s > max_by_k) s = max_by_k;
-    if (s < 1) s = 1;
+// Which tiles are split, and into how many parts.  `groups` tiles run at a time.  Too few tiles to fill
+// the machine: all of them are split.  Several rounds of tiles with a last, partly empty round: only
+// the tiles of that round are split, so that it takes a fraction of a round.  Each part keeps at least
+// 8 k-blocks.
+static void plan_splits(int64_t tiles, int32_t num_kb, int groups, int32_t* full_tiles, int32_t* splits) {
+    *full_tiles = (int32_t)tiles; *splits = 1;
+    if (num_kb < 16 || tiles > 8 * (int64_t)groups) return;
+    const int64_t full = tiles / groups * groups, rem = tiles - full;
+    if (rem == 0) return;
+    int s = (int)(groups / rem);
+    if (s > num_kb / 8) s = num_kb / 8;
+    if (s < 2) return;
     const int per = (num_kb + s - 1) / s;                   // no part may be empty
-    return (num_kb + per - 1) / per;
+    s = (num_kb + per - 1) / per;
+    if (s < 2) return;
+    *full_tiles = (int32_t)full; *splits = s;
 }
 
-// What launch_gemm_i8 may use: an int32 matrix of partial sums, for outputs small enough to be split.
+// What launch_gemm_i8 may use: int32 partial sums of the split tiles (fewer than one round of tiles,
+// i.e. at most 160 blocks of 128 x 256 on any device this runs on).
 size_t gemm_splitk_bytes(int64_t M, int64_t N) {
-    const int64_t tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
-    if (tiles > 8 * 160) return 0;   // never split (bound is generous with respect to the SM count)
-    return align_up((size_t)M * N * 4);
+    int64_t blocks = 2 * ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
+    if (blocks > 160) blocks = 160;
+    return align_up((size_t)blocks * BM * BN * 4);
 }
 
 template <int CTAS, int KIND>
@@ -784,14 +795,16 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.tiles_m = (int32_t)((g.M + BM * ctas - 1) / (BM * ctas));
     P.tiles_n = (int32_t)((g.N + BN - 1) / BN);
     const int64_t tiles = (int64_t)P.tiles_m * P.tiles_n;
-    // binary32 accumulators do not add exactly: the E4M3 product is never split
-    // nor is a product whose results are re-quantized or whose absmax is wanted (done in the epilogue)
-    P.splits = (g.kind == 0 && !g.opt.requant && !g.opt.absmax_bits) ? choose_splits(tiles, P.num_kb, groups_max) : 1;
+    // binary32 accumulators do not add exactly: the E4M3 and bf16 products are never split; nor is a
+    // product whose results are re-quantized or whose absmax is wanted (done in the epilogue)
+    P.full_tiles = (int32_t)tiles; P.splits = 1;
+    if (g.kind == 0 && !g.opt.requant && !g.opt.absmax_bits) plan_splits(tiles, P.num_kb, groups_max, &P.full_tiles, &P.splits);
     P.part = nullptr;
+    const int64_t split_tiles = tiles - P.full_tiles;
+    const size_t part_bytes = (size_t)split_tiles * BM * ctas * BN * 4;
     if (P.splits > 1) {
-        const size_t part_bytes = align_up((size_t)g.M * g.N * 4);
-        if (g.splitk_ws == nullptr || g.splitk_ws_bytes < part_bytes) {
-            P.splits = 1;   // no room: run unsplit (same result)
+        if (g.splitk_ws == nullptr || g.splitk_ws_bytes < part_bytes || tiles * BM * ctas >= (1ll << 31)) {
+            P.full_tiles = (int32_t)tiles; P.splits = 1;   // no room: run unsplit (same result)
         } else {
             P.part = (int32_t*)g.splitk_ws;
             if (cudaMemsetAsync(g.splitk_ws, 0, part_bytes, stream) != cudaSuccess) return SRQ_ERR_CUDA;
@@ -810,10 +823,10 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.rq_vec = g.opt.requant && ((uintptr_t)g.opt.rq_codes % 16 == 0) && (g.opt.rq_ld % 16 == 0);
     P.tma_out = P.write_out && P.vec_out && !g.acc_out && g.M < (1ll << 31) && g.N < (1ll << 31) &&
                 encode_output(&map_out, g.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.M, g.N, g.ldo);
-    P.tma_part = P.splits > 1 && g.N % 4 == 0 && g.M < (1ll << 31) && g.N < (1ll << 31) &&
-                 encode_output(&map_part, P.part, CU_TENSOR_MAP_DATA_TYPE_INT32, g.M, g.N, g.N);
+    if (P.splits > 1 && !encode_output(&map_part, P.part, CU_TENSOR_MAP_DATA_TYPE_INT32, split_tiles * BM * ctas, BN, BN))
+        return SRQ_ERR_CUDA;
 
-    const int64_t units = tiles * P.splits;
+    const int64_t units = P.full_tiles + split_tiles * P.splits;
     const unsigned groups = (unsigned)(units < groups_max ? units : groups_max);
     cudaError_t e;
     if (g.kind == 0) e = ctas == 2 ? launch_kernel<2, 0>(groups, map_a, map_b, map_out, map_part, P, stream)
@@ -825,12 +838,13 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     ++g_launches;
     if (e != cudaSuccess) return SRQ_ERR_CUDA;
     if (P.splits > 1) {
-        const int vec = g.N % 4 == 0 && g.ldo % 4 == 0 && (uintptr_t)g.out % 16 == 0 && (!g.acc_out || (uintptr_t)g.acc_out % 16 == 0);
-        const int64_t work = g.M * ((g.N + 3) / 4);
+        const int vec = g.ldo % 4 == 0 && (uintptr_t)g.out % 16 == 0;
+        const int64_t work = split_tiles * BM * ctas * (BN / 4);
         const int64_t blocks = (work + 255) / 256;
         const unsigned grid = (unsigned)(blocks < 8 * (int64_t)dev->sms ? blocks : 8 * (int64_t)dev->sms);
-        dequant_kernel<<<grid, 256, 0, stream>>>(P.part, g.M, g.N, g.s_row, g.row_stride, g.s_col, g.col_stride, g.out, g.ldo,
-                                                 g.acc_out, vec, g.opt.accumulate);
+        dequant_kernel<<<grid, 256, 0, stream>>>(P.part, split_tiles, P.full_tiles, P.tiles_n, BM * ctas, g.M, g.N, g.s_row,
+                                                 g.row_stride, g.s_col, g.col_stride, g.out, g.ldo, g.acc_out, vec,
+                                                 g.opt.accumulate);
         ++g_launches;
         if (cudaGetLastError() != cudaSuccess) return SRQ_ERR_CUDA;
     }
