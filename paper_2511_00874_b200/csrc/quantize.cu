@@ -345,6 +345,7 @@ struct QuantParams {
     const float* inv_tr;          // [1] or [cols]
     int vec_in;                   // 4-element vector loads allowed
     int vec_rm, vec_tr;           // 4-byte code stores allowed
+    int vec_tr16;                 // 16-byte stores of the transposed layout allowed
 };
 
 // Row-wise read of the transposed tile and its stores: one warp per tile column, lane = row quad.
@@ -384,7 +385,11 @@ __device__ __forceinline__ void widen(const uint2& q, float v[4]) {
 // current one is processed, which keeps two quads of loads in flight per thread.
 // FULL: the 128 x 128 tile lies inside the matrix and its Philox block indices do not carry into the
 // upper counter word, so rows need no bounds checks and the counter is one 32-bit multiply-add.
-template <typename T, int MODE, int LAYOUT, bool PER_ROW, bool FULL>
+// TR16 (full tiles whose transposed layout allows 16-byte stores): a warp takes 16 consecutive rows
+// instead of every eighth row quad, so that a thread ends up with 16 consecutive codes of each of
+// its four columns, writes them to the shared tile as one 16-byte chunk and the tile leaves in
+// 16-byte stores (a quarter of the instructions of the 4-byte path).
+template <typename T, int MODE, int LAYOUT, bool PER_ROW, bool FULL, bool TR16>
 __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const QuantParams& P, uint32_t* tileT,
                                               int64_t r0, int64_t c0) {
     using Raw = typename Raw4<T>::type;
@@ -413,10 +418,11 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
 
     Raw cur[4], nxt[4];
     float inv_cur[4], inv_nxt[4];
+    uint32_t tw[TR16 ? 4 : 1][4];                       // TR16: codes of 16 rows x 4 columns, one word per row quad
     auto load_quad = [&](int it, Raw raw[4], float inv_r[4]) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const uint32_t tr = (uint32_t)(warp + 8 * it) * 4 + i;
+            const uint32_t tr = (uint32_t)(TR16 ? warp * 4 + it : warp + 8 * it) * 4 + i;
             if (FULL || (col_ok && r0 + tr < P.rows)) {
                 raw[i] = __ldcs(reinterpret_cast<const Raw*>(xt + tr * ld));
                 if constexpr (PER_ROW && WANT_RM) inv_r[i] = P.inv_rm[r0 + tr];
@@ -431,7 +437,7 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
         if (it + 1 < 4) load_quad(it + 1, nxt, inv_nxt);
-        const int rq = warp + 8 * it;
+        const int rq = TR16 ? warp * 4 + it : warp + 8 * it;
         uint32_t wr[4], wt[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -460,13 +466,35 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
         if constexpr (WANT_TR) {
             uint32_t o[4];
             transpose4x4(wt, o);
+            if constexpr (TR16) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) tileT[(lane * 4 + e) * 32 + (rq ^ lane)] = o[e];
+                for (int e = 0; e < 4; ++e) tw[e][it] = o[e];
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) tileT[(lane * 4 + e) * 32 + (rq ^ lane)] = o[e];
+            }
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) { cur[i] = nxt[i]; inv_cur[i] = inv_nxt[i]; }
     }
-    if constexpr (WANT_TR) {
+    if constexpr (WANT_TR && TR16) {
+        // column col of the tile is a 128-byte row of tileT; rows 16 w .. 16 w + 15 (warp w) are its 16-byte
+        // chunk w, stored at chunk position w ^ ((col >> 2) & 7) so that a warp's stores spread over all banks
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            *reinterpret_cast<uint4*>(tileT + (lane * 4 + e) * 32 + ((warp ^ (lane & 7)) << 2)) =
+                make_uint4(tw[e][0], tw[e][1], tw[e][2], tw[e][3]);
+        __syncthreads();
+        // a warp stores 16 columns, four per instruction: 8 lanes x 16 bytes = the 128 rows of one column
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int col = warp * 16 + k * 4 + (lane >> 3);
+            const int chunk = lane & 7;
+            const uint4 v = *reinterpret_cast<const uint4*>(tileT + col * 32 + (chunk << 2));
+            const int rows16 = chunk ^ ((col >> 2) & 7);           // which 16 rows this chunk holds
+            *reinterpret_cast<uint4*>(P.codes_tr + (c0 + col) * P.ld_tr + r0 + rows16 * 16) = v;
+        }
+    } else if constexpr (WANT_TR) {
         __syncthreads();
         store_transposed_tile(tileT, P, r0, c0, warp, lane);
     }
@@ -483,8 +511,11 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
     const uint64_t j_first = (P.index_offset + (uint64_t)r0 * (uint64_t)P.cols + (uint64_t)c0) >> 2;
     const uint64_t j_span = (uint64_t)(Q_TILE - 1) * ((uint64_t)P.cols >> 2) + (Q_TILE / 4 - 1);
     const bool full = r0 + Q_TILE <= P.rows && c0 + Q_TILE <= P.cols && (j_first & 0xFFFFFFFFull) + j_span <= 0xFFFFFFFFull;
-    if (full) quantize_tile<T, MODE, LAYOUT, PER_ROW, true>(x, P, tileT, r0, c0);
-    else quantize_tile<T, MODE, LAYOUT, PER_ROW, false>(x, P, tileT, r0, c0);
+    if constexpr ((LAYOUT & 2) != 0) {
+        if (full && P.vec_tr16) { quantize_tile<T, MODE, LAYOUT, PER_ROW, true, true>(x, P, tileT, r0, c0); return; }
+    }
+    if (full) quantize_tile<T, MODE, LAYOUT, PER_ROW, true, false>(x, P, tileT, r0, c0);
+    else quantize_tile<T, MODE, LAYOUT, PER_ROW, false, false>(x, P, tileT, r0, c0);
 }
 
 // General path: any extent, pitch, alignment and index offset; one Philox block per element
@@ -678,6 +709,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         P.vec_in = vec_in;
         P.vec_rm = want_rm && ((uintptr_t)a.codes_rm % 4 == 0) && (a.ld_rm % 4 == 0);
         P.vec_tr = want_tr && ((uintptr_t)a.codes_tr % 4 == 0) && (a.ld_tr % 4 == 0);
+        P.vec_tr16 = want_tr && ((uintptr_t)a.codes_tr % 16 == 0) && (a.ld_tr % 16 == 0);
         const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) &&
                           (!want_tr || (P.vec_tr && rows % 4 == 0));
         const unsigned grid = (unsigned)(((cols + Q_TILE - 1) / Q_TILE) * ((rows + Q_TILE - 1) / Q_TILE));
