@@ -142,7 +142,7 @@ srq_status_t sr_quantize(const void *x, srq_dtype_t dt, int64_t rows, int64_t co
  * framework whose memory pool is already fully assigned, in a plug-in that is handed only its
  * input and output tensors, or in a latency-critical loop that must not hit the allocator's
  * implicit synchronisation.  The call itself allocates nothing, on the host or the device.
- *   - Limit: 256 + 2 * (pad64(rows) + pad64(cols)) * 4 bytes must fit in 1 MiB, pad64 rounding
+ *   - Limit: 512 + 2 * (pad64(rows) + pad64(cols)) * 4 bytes must fit in 1 MiB, pad64 rounding
  *     up to a multiple of 64 (about rows + cols <= 131000); larger inputs return
  *     SRQ_ERR_WORKSPACE and enqueue nothing.
  *   - The first call on each device looks up the array's device address (with that device

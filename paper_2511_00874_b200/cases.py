@@ -114,13 +114,22 @@ def case_layer(a):
     dW = torch.empty((a.N, a.K), device="cuda")
     ws = B.new_workspace(B.srq_workspace_bytes(a.T, a.N, a.K))
     fn = _layer_fn(A, W, dY, q, Y, dA, dW, ws)
+    if getattr(a, "graph", False):
+        # the calls only enqueue work on the stream, so a caller can record them once in a CUDA graph and
+        # replay it: for small layers this removes most of the per-launch cost
+        fn()                                     # first call outside the capture (one-time device set-up)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        fn = g.replay
     small = (A.numel() + dY.numel()) * A.element_size() < 2 * L2_BYTES
     med, best = _time(fn, a.iters, a.warmup, flush=small)
     assert B.srq_poll_status(ws) == 0
     ops = 6.0 * a.T * a.N * a.K
     return {"op": "layer fwd+bwd", "T": a.T, "N": a.N, "K": a.K, "dtype": a.dtype, "bits_fwd": a.bits_fwd,
-            "bits_bwd": a.bits_bwd, "scale": a.scale, "round": a.round, "grid": getattr(a, "grid", "int"), "ms": med, "ms_best": best,
-            "TOPS": ops / med / 1e9}
+            "bits_bwd": a.bits_bwd, "scale": a.scale, "round": a.round, "grid": getattr(a, "grid", "int"), "graph": bool(getattr(a, "graph", False)),
+            "ms": med, "ms_best": best, "TOPS": ops / med / 1e9}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -247,6 +256,7 @@ def main(argv=None):
             p.add_argument("--K", type=int, default=4096)
             p.add_argument("--bits-fwd", dest="bits_fwd", type=int, default=8)
             p.add_argument("--bits-bwd", dest="bits_bwd", type=int, default=8)
+            p.add_argument("--graph", action="store_true", help="record the step in a CUDA graph and time its replay")
         if name == "sweep":
             p.add_argument("--config", type=int, required=True, choices=[2, 3, 4, 5])
         if name not in ("gemm", "sweep"):

@@ -107,7 +107,8 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
 
     char* base = (char*)ws;
     uint32_t* status = &((WsHeader*)ws)->status;
-    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    // one clear for the status word and the scratch of both operands
+    if (cudaMemsetAsync(ws, 0, p.off_scale[0], st) != cudaSuccess) return SRQ_ERR_CUDA;
 
     const Operand* ops[2] = {&a, &b};
     int8_t* codes[2];
@@ -120,7 +121,7 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
         qa.x = o.x; qa.dt = dt; qa.rows = o.rows; qa.cols = o.cols; qa.ld = o.cols; qa.q = *o.q;
         qa.codes_rm = o.transposed ? nullptr : codes[i]; qa.ld_rm = p.pitch; qa.scale_rm = o.transposed ? nullptr : scales[i];
         qa.codes_tr = o.transposed ? codes[i] : nullptr; qa.ld_tr = p.pitch; qa.scale_tr = o.transposed ? scales[i] : nullptr;
-        if (Kc > 0 && launch_quantize(qa, carve_quant_scratch(base + p.off_scratch[i], o.rows, o.cols), status, st) != cudaSuccess)
+        if (Kc > 0 && launch_quantize(qa, carve_quant_scratch(base + p.off_scratch[i], o.rows, o.cols), status, st, true) != cudaSuccess)
             return SRQ_ERR_CUDA;
     }
     if (Kc == 0) {   // empty contraction: the product is zero
@@ -188,13 +189,13 @@ srq_status_t run_fwd_fp_act(const void* A, const void* W, srq_dtype_t dt, int64_
     if (K == 0) return cudaMemset2DAsync(Y, (size_t)N * 4, 0, (size_t)N * 4, (size_t)T, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
     char* base = (char*)ws;
     uint32_t* status = &((WsHeader*)ws)->status;
-    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, p.off_scale, st) != cudaSuccess) return SRQ_ERR_CUDA;      // status word and scratch
     int8_t* c8 = (int8_t*)(base + p.off_codes8);
     float* scale = (float*)(base + p.off_scale);
     float* one = (float*)(base + p.off_one);
     QuantArgs q; q.x = W; q.dt = dt; q.rows = N; q.cols = K; q.ld = K; q.q = *qW;
     q.codes_rm = c8; q.ld_rm = p.pitch8; q.scale_rm = scale; q.codes_tr = nullptr; q.ld_tr = 0; q.scale_tr = nullptr;
-    if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch, N, K), status, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch, N, K), status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
     if (launch_widen_codes(c8, N, K, p.pitch8, base + p.off_codes16, p.pitch16, one, st) != cudaSuccess) return SRQ_ERR_CUDA;
     GemmArgs g;
     g.a = (const int8_t*)A; g.lda = 2 * K; g.b = (const int8_t*)(base + p.off_codes16); g.ldb = 2 * p.pitch16;
@@ -267,7 +268,7 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
 
     char* base = (char*)ws;
     uint32_t* status = &((WsHeader*)ws)->status;
-    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, p.off_scale[0], st) != cudaSuccess) return SRQ_ERR_CUDA;   // status word and all scratch
     float* sc[4]; int8_t* cd[4];
     for (int i = 0; i < 4; ++i) { sc[i] = (float*)(base + p.off_scale[i]); cd[i] = (int8_t*)(base + p.off_codes[i]); }
 
@@ -275,19 +276,19 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
         QuantArgs q; q.x = dY; q.dt = dt; q.rows = T; q.cols = N; q.ld = N; q.q = *qdY;
         q.codes_rm = cd[0]; q.ld_rm = p.pitch_n; q.scale_rm = sc[0];
         q.codes_tr = cd[1]; q.ld_tr = p.pitch_t; q.scale_tr = sc[1];
-        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[0], T, N), status, st) != cudaSuccess) return SRQ_ERR_CUDA;
+        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[0], T, N), status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
     }
     if (N > 0 && K > 0) {      // W -> [K,N]
         QuantArgs q; q.x = W; q.dt = dt; q.rows = N; q.cols = K; q.ld = K; q.q = *qW;
         q.codes_rm = nullptr; q.ld_rm = 0; q.scale_rm = nullptr;
         q.codes_tr = cd[2]; q.ld_tr = p.pitch_n; q.scale_tr = sc[2];
-        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[1], N, K), status, st) != cudaSuccess) return SRQ_ERR_CUDA;
+        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[1], N, K), status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
     }
     if (T > 0 && K > 0) {      // A -> [K,T]
         QuantArgs q; q.x = A; q.dt = dt; q.rows = T; q.cols = K; q.ld = K; q.q = *qA;
         q.codes_rm = nullptr; q.ld_rm = 0; q.scale_rm = nullptr;
         q.codes_tr = cd[3]; q.ld_tr = p.pitch_t; q.scale_tr = sc[3];
-        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[2], T, K), status, st) != cudaSuccess) return SRQ_ERR_CUDA;
+        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[2], T, K), status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
     }
 
     // dA[T,K] = Q(dY)[T,N] . Q(W)^T[K,N]
@@ -366,13 +367,13 @@ srq_status_t sr_quantize(const void* x, srq_dtype_t dt, int64_t rows, int64_t co
     if (ws_bytes < srq_quantize_workspace_bytes(rows, cols)) return SRQ_ERR_WORKSPACE;
     if (rows == 0 || cols == 0) return SRQ_OK;
     uint32_t* status = &((WsHeader*)ws)->status;
-    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, srq_quantize_workspace_bytes(rows, cols), st) != cudaSuccess) return SRQ_ERR_CUDA;
     QuantArgs a;
     a.x = x; a.dt = dt; a.rows = rows; a.cols = cols; a.ld = ld; a.q = *q;
     a.codes_rm = codes_rm; a.ld_rm = ld_rm; a.scale_rm = scale_rm;
     a.codes_tr = codes_tr; a.ld_tr = ld_tr; a.scale_tr = scale_tr;
     const QuantScratch sc = carve_quant_scratch((char*)ws + sizeof(WsHeader), rows, cols);
-    return launch_quantize(a, sc, status, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+    return launch_quantize(a, sc, status, st, true) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
 }
 
 srq_status_t srq_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax, void* cuda_stream) {

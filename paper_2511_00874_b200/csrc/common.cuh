@@ -66,6 +66,7 @@ inline PhiloxKeys make_philox_keys(uint64_t seed, uint64_t tensor_id) {
 // Scratch carved from a workspace for one sr_quantize: absmax words and reciprocal steps for
 // the row-major layout (1 or rows) and the transposed layout (1 or cols).
 struct QuantScratch {
+    uint32_t* counter;   // CTAs of the absmax launch that have finished, zeroed before use
     uint32_t* amax_rm;   // fp32 bit patterns, zeroed before use
     uint32_t* amax_tr;
     float* inv_rm;
@@ -81,10 +82,10 @@ struct QuantArgs {
     int8_t* codes_rm; int64_t ld_rm; float* scale_rm;
     int8_t* codes_tr; int64_t ld_tr; float* scale_tr;
 };
-// Enqueues: clear scratch, absmax, step sizes, quantize.  `scratch` must be exclusively this
-// call's until the kernels finish.
+// Enqueues: clear scratch (unless the caller has zeroed the whole scratch block already), absmax with
+// step sizes, quantize.  `scratch` must be exclusively this call's until the kernels finish.
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& scratch, uint32_t* status,
-                            cudaStream_t stream);
+                            cudaStream_t stream, bool scratch_zeroed = false);
 
 // max |x| of the whole matrix into *absmax (device float, overwritten).
 cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax, cudaStream_t stream);

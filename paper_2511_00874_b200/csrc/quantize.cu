@@ -31,13 +31,14 @@ unsigned long long g_launches = 0;
 static inline size_t f32_block(int64_t n) { return align_up((size_t)n * 4); }
 
 size_t quant_scratch_bytes(int64_t rows, int64_t cols) {
-    return 2 * (f32_block(rows) + f32_block(cols));
+    return kAlign + 2 * (f32_block(rows) + f32_block(cols));
 }
 
 QuantScratch carve_quant_scratch(void* base, int64_t rows, int64_t cols) {
-    // amax blocks first and contiguous, so that one memset clears both
+    // counter and amax blocks first and contiguous, so that one memset clears them
     char* p = (char*)base;
     QuantScratch s;
+    s.counter = (uint32_t*)p; p += kAlign;
     s.amax_rm = (uint32_t*)p; p += f32_block(rows);
     s.amax_tr = (uint32_t*)p; p += f32_block(cols);
     s.inv_rm = (float*)p; p += f32_block(rows);
@@ -77,6 +78,28 @@ __device__ __forceinline__ uint32_t abs_bits(float v) { return __float_as_uint(v
 // ------------------------------------------------------------------------------------------
 // absmax
 // ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void scale_from_bits(uint32_t bits, float qmax, float* delta, float* inv,
+                                                uint32_t* status) {
+    if (bits >= 0x7F800000u) record_status(status, SRQ_ERR_NONFINITE);
+    const float m = __uint_as_float(bits);
+    // toward zero, so that |x * r| <= qmax for the whole group; a reciprocal that overflows when
+    // rounded to nearest marks a group too small to scale, which is treated as all zeros
+    float r = 0.0f;
+    if (m != 0.0f && fabsf(__fdiv_rn(qmax, m)) <= 3.402823466e38f) r = __fdiv_rz(qmax, m);
+    *inv = r;
+    *delta = (r == 0.0f) ? 0.0f : __fdiv_rn(m, qmax);
+}
+
+// What the last CTA of an absmax launch does once every CTA has contributed: the step sizes of all
+// groups (saves a launch; `counter` must be zero when the launch starts).  counter == nullptr: nothing.
+struct ScaleStep {
+    uint32_t* counter;
+    int64_t n_rm; float* inv_rm; float* delta_rm;
+    int64_t n_tr; float* inv_tr; float* delta_tr;
+    float qmax;
+    uint32_t* status;
+};
+
 constexpr int AMAX_THREADS = 256;
 constexpr int AMAX_TILE_R = 64;    // 8 warps x 8 rows
 constexpr int AMAX_GROUPS = 2;     // 16-byte groups per lane and row
@@ -105,7 +128,7 @@ __device__ __forceinline__ uint32_t abs_max16(const uint4& q, __nv_bfloat16) {
 template <typename T, bool ROWS, bool COLS>
 __global__ void __launch_bounds__(AMAX_THREADS, COLS ? 3 : 4)
 amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok,
-            uint32_t* __restrict__ amax_rm, uint32_t* __restrict__ amax_tr) {
+            uint32_t* __restrict__ amax_rm, uint32_t* __restrict__ amax_tr, const ScaleStep S) {
     constexpr int EPL = 16 / (int)sizeof(T);                   // elements per 16-byte group
     constexpr int TILE_C = 32 * AMAX_GROUPS * EPL;
     __shared__ uint32_t col_max[COLS ? TILE_C : 1];
@@ -192,36 +215,45 @@ amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, boo
             if (c < cols && col_max[i]) atomicMax(&amax_tr[c], col_max[i]);
         }
     }
+    if (S.counter == nullptr) return;
+    // the CTA that arrives last sees every maximum and turns them into step sizes
+    __shared__ uint32_t is_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(S.counter, 1u) == gridDim.x - 1 ? 1u : 0u;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int64_t i = threadIdx.x; i < S.n_rm; i += AMAX_THREADS) {
+        float d, r;
+        scale_from_bits(__ldcg(&amax_rm[i]), S.qmax, &d, &r, S.status);
+        S.inv_rm[i] = r;
+        if (S.delta_rm) S.delta_rm[i] = d;
+    }
+    for (int64_t i = threadIdx.x; i < S.n_tr; i += AMAX_THREADS) {
+        float d, r;
+        scale_from_bits(__ldcg(&amax_tr[i]), S.qmax, &d, &r, S.status);
+        S.inv_tr[i] = r;
+        if (S.delta_tr) S.delta_tr[i] = d;
+    }
 }
 
 template <typename T>
 static void launch_amax(const void* x, int64_t rows, int64_t cols, int64_t ld, uint32_t* amax_rm, bool want_rows,
-                        uint32_t* amax_tr, bool want_cols, cudaStream_t st) {
+                        uint32_t* amax_tr, bool want_cols, const ScaleStep& S, cudaStream_t st) {
     const T* p = (const T*)x;
     constexpr int tile_c = 32 * AMAX_GROUPS * (16 / (int)sizeof(T));
     const unsigned grid = (unsigned)(((cols + tile_c - 1) / tile_c) * ((rows + AMAX_TILE_R - 1) / AMAX_TILE_R));
     const bool vec_ok = ((uintptr_t)x % 16 == 0) && ((ld * (int64_t)sizeof(T)) % 16 == 0);
-    if (want_rows && want_cols) amax_kernel<T, true, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
-    else if (want_rows) amax_kernel<T, true, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
-    else if (want_cols) amax_kernel<T, false, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
-    else amax_kernel<T, false, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr);
+    if (want_rows && want_cols) amax_kernel<T, true, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
+    else if (want_rows) amax_kernel<T, true, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
+    else if (want_cols) amax_kernel<T, false, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
+    else amax_kernel<T, false, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
 }
 
 // ------------------------------------------------------------------------------------------
 // step sizes
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ void scale_from_bits(uint32_t bits, float qmax, float* delta, float* inv,
-                                                uint32_t* status) {
-    if (bits >= 0x7F800000u) record_status(status, SRQ_ERR_NONFINITE);
-    const float m = __uint_as_float(bits);
-    // toward zero, so that |x * r| <= qmax for the whole group; a reciprocal that overflows when
-    // rounded to nearest marks a group too small to scale, which is treated as all zeros
-    float r = 0.0f;
-    if (m != 0.0f && fabsf(__fdiv_rn(qmax, m)) <= 3.402823466e38f) r = __fdiv_rz(qmax, m);
-    *inv = r;
-    *delta = (r == 0.0f) ? 0.0f : __fdiv_rn(m, qmax);
-}
-
 // The rm and tr arrays may be the same memory (per tensor, one group serves both layouts).
 __global__ void scales_kernel(const uint32_t* amax_rm, int64_t n_rm, float* inv_rm, float* delta_rm,
                               const uint32_t* amax_tr, int64_t n_tr, float* inv_tr, float* delta_tr,
@@ -649,13 +681,14 @@ cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, 
 cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax, cudaStream_t stream) {
     cudaError_t e = cudaMemsetAsync(absmax, 0, sizeof(float), stream);
     if (e != cudaSuccess || rows == 0 || cols == 0) return e;
-    if (dt == SRQ_F32) launch_amax<float>(x, rows, cols, ld, (uint32_t*)absmax, false, nullptr, false, stream);
-    else launch_amax<__nv_bfloat16>(x, rows, cols, ld, (uint32_t*)absmax, false, nullptr, false, stream);
+    const ScaleStep none = {};
+    if (dt == SRQ_F32) launch_amax<float>(x, rows, cols, ld, (uint32_t*)absmax, false, nullptr, false, none, stream);
+    else launch_amax<__nv_bfloat16>(x, rows, cols, ld, (uint32_t*)absmax, false, nullptr, false, none, stream);
     ++g_launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream) {
+cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream, bool scratch_zeroed) {
     const bool want_rm = a.codes_rm != nullptr, want_tr = a.codes_tr != nullptr;
     const bool per_row = a.q.scale == SRQ_PER_ROW;
     const int64_t rows = a.rows, cols = a.cols;
@@ -674,25 +707,28 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
 
     const bool vec_in = ((uintptr_t)a.x % (4 * esize) == 0) && (a.ld % 4 == 0);
     const bool given = a.q.absmax != nullptr && !per_row;   // a known absmax is only taken per tensor
+    // per tensor: one group feeds both layouts' scale outputs
+    const int64_t n0 = per_row ? n_rm : 1;
+    const int64_t n1 = per_row ? n_tr : ((want_tr && a.scale_tr) ? 1 : 0);
     if (given) {
         amax_rm = amax_tr = (uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
-    } else {
-        cudaError_t e = cudaMemsetAsync(s.amax_rm, 0, (size_t)((char*)s.inv_rm - (char*)s.amax_rm), stream);
-        if (e != cudaSuccess) return e;
-        const bool want_rows = per_row && want_rm, want_cols = per_row && want_tr;
-        if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, stream);
-        else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, stream);
-        ++g_launches;
-    }
-    {
-        // per tensor: one group feeds both layouts' scale outputs
-        const int64_t n0 = per_row ? n_rm : 1;
-        const int64_t n1 = per_row ? n_tr : ((want_tr && a.scale_tr) ? 1 : 0);
         const int64_t n = n0 > n1 ? n0 : n1;
         const int threads = 256;
         scales_kernel<<<(unsigned)((n + threads - 1) / threads), threads, 0, stream>>>(
             amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
             amax_tr, n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status);
+        ++g_launches;
+    } else {
+        if (!scratch_zeroed) {
+            cudaError_t e = cudaMemsetAsync(s.counter, 0, (size_t)((char*)s.inv_rm - (char*)s.counter), stream);
+            if (e != cudaSuccess) return e;
+        }
+        // absmax of every group; the last CTA to finish turns them into step sizes
+        const ScaleStep S = {s.counter, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
+                             n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status};
+        const bool want_rows = per_row && want_rm, want_cols = per_row && want_tr;
+        if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, S, stream);
+        else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, S, stream);
         ++g_launches;
     }
     {
