@@ -194,17 +194,24 @@ def run_ours(args):
     dW = torch.empty((N, K), device=dev)
     ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K), dev)
 
-    amax_a = torch.zeros(1, device=dev)               # max |A|, found once per step, used by both of A's quantization points
+    # max |A| and max |dY|: found once per step, max-reduced over the token shards when there are several
+    # (so that every rank uses the step sizes of the whole batch), and handed to the quantization points
+    amax_a = torch.zeros(1, device=dev)
+    amax_dy = torch.zeros(1, device=dev)
 
     def specs(step):
         off_a, off_y = rank * T * K, rank * T * N       # thresholds follow the global flat index
         return (srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 0, off_a, absmax=amax_a), srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 1),
                 srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 2, off_a, absmax=amax_a), srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 3),
-                srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 4, off_y))
+                srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 4, off_y, absmax=amax_dy))
 
     def step(i, a=A, w=W, dy=dY, y=Y, da=dA, dw=dW):
         qa_f, qw_f, qa_b, qw_b, qdy = specs(i)
         srq.srq_absmax(a, amax_a)
+        srq.srq_absmax(dy, amax_dy)
+        if world > 1:
+            dist.all_reduce(amax_a, op=dist.ReduceOp.MAX)
+            dist.all_reduce(amax_dy, op=dist.ReduceOp.MAX)
         srq.qlinear_fwd(a, w, qa_f, qw_f, y, None, ws)
         srq.qlinear_bwd(dy, a, w, qdy, qa_b, qw_b, da, dw, None, None, ws)      # Alg. 2: both backward products
         if world > 1:
@@ -276,9 +283,9 @@ def run_ours(args):
               "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
               "vs_baseline": None, "dtype": "int8", "data": "synthetic",
               "config": {"workload": WORKLOAD, "tokens_per_gpu": T, "l2": "inputs (1 GiB each) are larger than L2",
-                         "absmax": "max |A| is computed once per step (srq_absmax) and shared by A's forward and backward "
-                                   "quantization points; every other operand finds its own",
-                         "multi_gpu": "token shards, one NCCL all-reduce of dW per step" if world > 1 else "single GPU"},
+                         "absmax": "max |A| and max |dY| are computed once per step (srq_absmax; max-reduced over ranks when "
+                                   "N > 1) and handed to their quantization points; max |A| serves both of A's points",
+                         "multi_gpu": "token shards, two scalar all-reduce(max) and one all-reduce(sum) of dW per step" if world > 1 else "single GPU"},
               "gpu_launches": int(launches)}
 
     # ---- end to end through the public API with host buffers (every rank, max over ranks).
