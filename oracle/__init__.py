@@ -19,7 +19,7 @@ _SRC = os.path.join(_HERE, "srq_oracle.c")
 _LIB = os.path.join(_HERE, "libsrq_oracle.so")
 
 PER_TENSOR, PER_ROW = 0, 1
-SR, RTN = 0, 1
+SR, RTN, SR8 = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.orc_philox4x32_10.restype = None
         L.orc_threshold_u24.argtypes = [ctypes.c_uint64] * 3
         L.orc_threshold_u24.restype = ctypes.c_uint32
+        L.orc_threshold_sr8.argtypes = [ctypes.c_uint64] * 3
+        L.orc_threshold_sr8.restype = ctypes.c_uint32
         L.orc_scale_from_absmax.argtypes = [ctypes.c_float, ctypes.c_int,
                                             ctypes.POINTER(ctypes.c_float),
                                             ctypes.POINTER(ctypes.c_float)]
@@ -141,6 +143,11 @@ def philox4x32_10(ctr, key):
 
 def threshold_u24(seed: int, tensor_id: int, i: int) -> int:
     return int(lib().orc_threshold_u24(seed, tensor_id, i))
+
+
+def threshold_sr8(seed: int, tensor_id: int, i: int) -> int:
+    """Threshold of element i in the 8-random-bit mode, on the 2^-24 lattice: (2 b + 1) 2^15."""
+    return int(lib().orc_threshold_sr8(seed, tensor_id, i))
 
 
 def scale_from_absmax(m: float, bits: int):

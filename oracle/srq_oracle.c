@@ -45,6 +45,7 @@
 #define ORC_PER_ROW 1
 #define ORC_SR 0
 #define ORC_RTN 1
+#define ORC_SR8 2   /* stochastic rounding with 8 random bits per element */
 
 /* ---------------------------------------------------------------------- */
 /* Thresholds eps (Def. 3): counter-based Philox4x32-10                     */
@@ -91,6 +92,38 @@ uint32_t orc_threshold_u24(uint64_t seed, uint64_t tensor_id, uint64_t i)
     uint32_t out[4];
     orc_philox4x32_10(ctr, key, out);
     return out[i & 3] >> 8;
+}
+
+/*
+ * Thresholds with 8 random bits per element.  The paper's hardware section
+ * argues that a rounding unit needs only a few pseudo-random bits (its FPGA
+ * estimate uses a 6-bit LFSR); this variant takes eps = (b + 1/2) / 256 with b
+ * one byte of the Philox stream, so that one 128-bit block serves 16 elements:
+ * block j = i >> 4, word (i >> 2) & 3 of it, byte i & 3 of that word (least
+ * significant byte first).  Returned on the 2^-24 lattice of orc_threshold_u24,
+ * (2 b + 1) 2^15, so that the same comparison rule applies.  The half offset
+ * centres the 256 thresholds: P(round up) is then the fraction rounded to the
+ * nearest multiple of 1/256 (ties down), within 2^-9 of it and without a
+ * systematic sign.
+ */
+uint32_t orc_threshold_sr8(uint64_t seed, uint64_t tensor_id, uint64_t i)
+{
+    uint64_t j = i >> 4;
+    uint32_t ctr[4] = { (uint32_t)j, (uint32_t)(j >> 32),
+                        (uint32_t)tensor_id, (uint32_t)(tensor_id >> 32) };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    uint32_t b = (out[(i >> 2) & 3] >> (8 * (i & 3))) & 0xFFu;
+    return (2u * b + 1u) << 15;
+}
+
+/* Threshold of element i on the 2^-24 lattice for the given rounding mode (0 for RTN). */
+static uint32_t orc_threshold(int round_mode, uint64_t seed, uint64_t tensor_id, uint64_t i)
+{
+    if (round_mode == ORC_SR) return orc_threshold_u24(seed, tensor_id, i);
+    if (round_mode == ORC_SR8) return orc_threshold_sr8(seed, tensor_id, i);
+    return 0u;
 }
 
 /* ---------------------------------------------------------------------- */
@@ -152,7 +185,7 @@ int orc_quantize_scalar(float x, float inv, int bits, int round_mode, uint32_t u
     double td = (double)t;
     double f = floor(td);
     int up;
-    if (round_mode == ORC_SR)
+    if (round_mode == ORC_SR || round_mode == ORC_SR8)
         up = ((double)u24 + f * 0x1p24) < td * 0x1p24;
     else
         up = (f * 0x1p24 + 0x1p23) <= td * 0x1p24;
@@ -261,7 +294,7 @@ int orc_sr_quantize(const float *x, int64_t rows, int64_t cols, int64_t ld,
             }
             for (int64_t c = 0; c < cols; ++c) {
                 uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
-                uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, i) : 0u;
+                uint32_t u24 = orc_threshold(round_mode, seed, tensor_id, i);
                 codes_rm[r * cols + c] =
                     (int8_t)orc_quantize_scalar(x[r * ld + c], inv, bits, round_mode, u24);
             }
@@ -287,7 +320,7 @@ int orc_sr_quantize(const float *x, int64_t rows, int64_t cols, int64_t ld,
             }
             for (int64_t r = 0; r < rows; ++r) {
                 uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
-                uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, i) : 0u;
+                uint32_t u24 = orc_threshold(round_mode, seed, tensor_id, i);
                 codes_tr[c * rows + r] =
                     (int8_t)orc_quantize_scalar(x[r * ld + c], inv, bits, round_mode, u24);
             }
@@ -481,7 +514,7 @@ uint8_t orc_quantize_e4m3_scalar(float x, float inv, int round_mode, uint32_t u2
     double u = ldexp(td, 3 - e);                 /* t / D, exact */
     double f = floor(u);
     int up;
-    if (round_mode == ORC_SR)
+    if (round_mode == ORC_SR || round_mode == ORC_SR8)
         up = ((double)u24 + f * 0x1p24) < u * 0x1p24;
     else
         up = (f * 0x1p24 + 0x1p23) <= u * 0x1p24;
@@ -526,7 +559,7 @@ int orc_sr_quantize_e4m3(const float *x, int64_t rows, int64_t cols, int64_t ld,
             else if (r == 0) scale_rm[0] = delta;
             for (int64_t c = 0; c < cols; ++c) {
                 uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
-                uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, i) : 0u;
+                uint32_t u24 = orc_threshold(round_mode, seed, tensor_id, i);
                 codes_rm[r * cols + c] = orc_quantize_e4m3_scalar(x[r * ld + c], inv, round_mode, u24);
             }
         }
@@ -542,7 +575,7 @@ int orc_sr_quantize_e4m3(const float *x, int64_t rows, int64_t cols, int64_t ld,
             else if (c == 0) scale_tr[0] = delta;
             for (int64_t r = 0; r < rows; ++r) {
                 uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
-                uint32_t u24 = (round_mode == ORC_SR) ? orc_threshold_u24(seed, tensor_id, i) : 0u;
+                uint32_t u24 = orc_threshold(round_mode, seed, tensor_id, i);
                 codes_tr[c * rows + r] = orc_quantize_e4m3_scalar(x[r * ld + c], inv, round_mode, u24);
             }
         }

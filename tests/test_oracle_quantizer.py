@@ -277,3 +277,41 @@ def test_quotient_of_the_extreme_element_never_passes_qmax():
             assert oracle.quantize_scalar(float(m), float(inv), bits, RTN) == q
             assert oracle.quantize_scalar(-float(m), float(inv), bits, RTN) == -q
     assert below
+
+
+def test_eight_bit_thresholds_bytes_of_the_philox_stream_and_centred_probabilities():
+    """SR with 8 random bits per element: the threshold of element i is byte i & 3 of word (i >> 2) & 3 of
+    Philox block i >> 4 (independent numpy Philox), placed at (b + 1/2) / 256; P(up) is then the fraction
+    rounded to the nearest multiple of 1/256, and the rounding stays unbiased on average."""
+    from _independent import philox_np
+    seed, tid, off = 2 ** 40 + 5, 2 ** 33 + 7, 2 ** 36 + 3
+    idx = np.arange(off, off + 200, dtype=np.uint64)
+    j = idx >> np.uint64(4)
+    words = philox_np(j & np.uint64(0xFFFFFFFF), j >> np.uint64(32), np.full_like(j, tid & 0xFFFFFFFF),
+                      np.full_like(j, tid >> 32), seed & 0xFFFFFFFF, seed >> 32)
+    stacked = np.stack(words, axis=0)
+    w = np.take_along_axis(stacked, ((idx >> np.uint64(2)) & np.uint64(3)).astype(np.int64)[None, :], axis=0)[0]
+    b = (w >> (np.uint64(8) * (idx & np.uint64(3)))) & np.uint64(0xFF)
+    want = (2 * b.astype(np.int64) + 1) << 15
+    got = np.array([oracle.threshold_sr8(seed, tid, int(i)) for i in idx])
+    assert np.array_equal(got, want)
+    # exact probability: thresholds (2b+1) 2^15 for b = 0..255, up iff threshold < frac 2^24
+    for p in (0.0, 1 / 512, 1 / 256, 0.3, 0.5, 0.7, 1 - 1 / 512, 1 - 2.0 ** -20):
+        ups = sum(oracle.quantize_scalar(2.0 + p, 1.0, 8, oracle.SR8, (2 * bb + 1) << 15) == 3 for bb in range(256))
+        assert ups == math.floor(256 * p + 0.5) or (256 * p + 0.5 == math.floor(256 * p + 0.5) and ups == 256 * p - 0.5)
+    # matrix form against the restatement, and unbiasedness over seeds
+    rng = np.random.default_rng(13)
+    x = rng.normal(0, 1, (1, 2048)).astype(np.float32)
+    d, inv = scale_ref(np.abs(x).max(), 8)
+    u = np.array([oracle.threshold_sr8(3, 9, i) for i in range(2048)]).reshape(1, 2048)
+    c, s, _, _ = oracle.sr_quantize(x, QSpec(8, PER_TENSOR, oracle.SR8, 3, 9))
+    assert np.array_equal(c, quantize_matrix_ref(x, inv, 8, True, u)) and s[0] == d
+    acc = np.zeros((1, 2048))
+    draws = 3000
+    for seed in range(draws):
+        acc += oracle.sr_quantize(x, QSpec(8, PER_TENSOR, oracle.SR8, seed, 9))[0]
+    t = x.astype(np.float64) * float(inv)
+    p = t - np.floor(t)
+    err = acc / draws - t
+    assert np.all(np.abs(err) <= 5 * np.sqrt(p * (1 - p) / draws) + 1 / 512 + 3.0 / draws)      # per element: within 2^-9 of unbiased
+    assert abs(err.mean()) < 3e-3                                                                  # and no systematic sign
