@@ -74,7 +74,11 @@ typedef enum {
 
 typedef enum { SRQ_F32 = 0, SRQ_BF16 = 1 } srq_dtype_t;
 typedef enum { SRQ_PER_TENSOR = 0, SRQ_PER_ROW = 1 } srq_scale_t;
-typedef enum { SRQ_SR = 0, SRQ_RTN = 1 } srq_round_t;
+/* SRQ_SR8: stochastic rounding with 8 random bits per element instead of 24 (the paper's hardware
+ * section argues that a few pseudo-random bits per rounding suffice): eps = (b + 1/2) / 256 with b
+ * byte (i & 3) of word ((i >> 2) & 3) of Philox block i >> 4, so that one block serves 16 elements.
+ * P(round up) is the fraction rounded to the nearest 1/256.  Integer grid only. */
+typedef enum { SRQ_SR = 0, SRQ_RTN = 1, SRQ_SR8 = 2 } srq_round_t;
 /* Grid of a quantization point: integers times the step size (bits 2..8), or the E4M3 8-bit
  * floating-point values times the step size (1 sign, 4 exponent, 3 mantissa bits, bias 7, no
  * infinities, largest value 448; `bits` is ignored). */

@@ -22,7 +22,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_ACC_OVERFLOW, ERR_CUDA,
     ERR_TIMEOUT = range(8)
 F32, BF16 = 0, 1
 PER_TENSOR, PER_ROW = 0, 1
-SR, RTN = 0, 1
+SR, RTN, SR8 = 0, 1, 2
 GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",

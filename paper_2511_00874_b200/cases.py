@@ -49,7 +49,7 @@ def case_quantize(a):
     dt = torch.float32 if a.dtype == "f32" else torch.bfloat16
     x = synth.with_outliers((a.rows, a.cols), a.seed, dt, "cuda")
     per_row = a.scale == "row"
-    q = B.QSpec(a.bits, B.PER_ROW if per_row else B.PER_TENSOR, B.SR if a.round == "sr" else B.RTN, a.seed, 1,
+    q = B.QSpec(a.bits, B.PER_ROW if per_row else B.PER_TENSOR, {"sr": B.SR, "rtn": B.RTN, "sr8": B.SR8}[a.round], a.seed, 1,
                 0, B.GRID_E4M3 if getattr(a, "grid", "int") == "e4m3" else B.GRID_INT)
     rm, tr = a.layouts in ("rm", "both"), a.layouts in ("tr", "both")
     crm = torch.empty((a.rows, a.cols), dtype=torch.int8, device="cuda") if rm else None
@@ -107,7 +107,7 @@ def case_layer(a):
     dt = torch.float32 if a.dtype == "f32" else torch.bfloat16
     A, W, dY = synth.layer_inputs(a.T, a.N, a.K, a.seed, dt, "cuda", std_dy=1e-3)
     sc = B.PER_ROW if a.scale == "row" else B.PER_TENSOR
-    rd = B.SR if a.round == "sr" else B.RTN
+    rd = {"sr": B.SR, "rtn": B.RTN, "sr8": B.SR8}[a.round]
     q = _layer_specs(a.bits_fwd, a.bits_bwd, sc, rd, a.seed, getattr(a, "grid", "int"))
     Y = torch.empty((a.T, a.N), device="cuda")
     dA = torch.empty((a.T, a.K), device="cuda")
@@ -262,7 +262,7 @@ def main(argv=None):
         if name not in ("gemm", "sweep"):
             p.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
             p.add_argument("--scale", default="tensor", choices=["tensor", "row"])
-            p.add_argument("--round", default="sr", choices=["sr", "rtn"])
+            p.add_argument("--round", default="sr", choices=["sr", "rtn", "sr8"])
     a = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("a CUDA device is required (there is no CPU fallback)")

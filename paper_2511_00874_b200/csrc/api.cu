@@ -13,7 +13,8 @@ srq_status_t check_qspec(const srq_qspec_t* q) {
     if (q->format != SRQ_GRID_INT && q->format != SRQ_GRID_E4M3) return SRQ_ERR_INVALID_ARG;
     if (q->format == SRQ_GRID_INT && (q->bits < 2 || q->bits > 8)) return SRQ_ERR_UNSUPPORTED;
     if (q->scale != SRQ_PER_TENSOR && q->scale != SRQ_PER_ROW) return SRQ_ERR_INVALID_ARG;
-    if (q->round != SRQ_SR && q->round != SRQ_RTN) return SRQ_ERR_INVALID_ARG;
+    if (q->round != SRQ_SR && q->round != SRQ_RTN && q->round != SRQ_SR8) return SRQ_ERR_INVALID_ARG;
+    if (q->round == SRQ_SR8 && q->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;
     if (q->absmax && (q->scale != SRQ_PER_TENSOR || ((uintptr_t)q->absmax % 4) != 0)) return SRQ_ERR_INVALID_ARG;
     return SRQ_OK;
 }
@@ -28,7 +29,7 @@ srq_status_t make_out_options(const srq_output_t* o, int64_t N, bool have_out, O
     if (o->q) {
         srq_status_t s = check_qspec(o->q);
         if (s != SRQ_OK) return s;
-        if (o->q->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;
+        if (o->q->format != SRQ_GRID_INT || o->q->round == SRQ_SR8) return SRQ_ERR_UNSUPPORTED;
         if (!o->step || !o->codes || o->ld_codes < N || ((uintptr_t)o->step % 4) != 0) return SRQ_ERR_INVALID_ARG;
         r->requant = 1;
         r->rq_sr = o->q->round == SRQ_SR;

@@ -288,8 +288,10 @@ __global__ void scales_kernel(const uint32_t* amax_rm, int64_t n_rm, float* inv_
 //        (floor(S) + 2^23) >> 24.
 // |t| <= qmax for every element of a group (the reciprocal step is rounded toward zero), so
 // |C| <= qmax 2^24, the sum stays inside int32 and the code inside [-qmax, qmax] without a clamp.
-// MODE: bit 0 = stochastic rounding (else round to nearest), bit 1 = E4M3 grid (else integer grid).
-constexpr int MODE_SR = 1, MODE_E4M3 = 2;
+// MODE: bit 0 = stochastic rounding (else round to nearest), bit 1 = E4M3 grid (else integer grid),
+// bit 2 = stochastic rounding with 8 random bits per element (integer grid only; the thresholds are
+// then handed to the same arithmetic as words (b << 24) | 2^23, whose top 24 bits are (2 b + 1) 2^15).
+constexpr int MODE_SR = 1, MODE_E4M3 = 2, MODE_SR8 = 4;
 
 // Integer grid: returns the 32-bit sum whose top byte is the code (two's complement).
 template <int MODE>
@@ -327,11 +329,20 @@ __device__ __forceinline__ uint32_t quantize_e4m3(float x, float inv, uint32_t w
     return ((uint32_t)q & 0x80u) | ((E << 3) + (uint32_t)abs(q) - 968u);
 }
 
+// 8-random-bit mode: the threshold words of four consecutive elements from the stream word that holds
+// their four bytes.
+__device__ __forceinline__ void sr8_words(uint32_t w, uint32_t rnd[4]) {
+    rnd[0] = __byte_perm(w, 0x00800000u, 0x0644); rnd[1] = __byte_perm(w, 0x00800000u, 0x1644);
+    rnd[2] = __byte_perm(w, 0x00800000u, 0x2644); rnd[3] = __byte_perm(w, 0x00800000u, 0x3644);
+}
+
 // Four codes packed into one word, first element in the low byte.
 template <int MODE>
 __device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3,
                                               const uint32_t rnd[4]) {
-    if constexpr ((MODE & MODE_E4M3) != 0) {
+    if constexpr ((MODE & MODE_SR8) != 0) {
+        return quantize4<MODE_SR>(v, i0, i1, i2, i3, rnd);
+    } else if constexpr ((MODE & MODE_E4M3) != 0) {
         const uint32_t c0 = quantize_e4m3<MODE>(v[0], i0, rnd[0]), c1 = quantize_e4m3<MODE>(v[1], i1, rnd[1]);
         const uint32_t c2 = quantize_e4m3<MODE>(v[2], i2, rnd[2]), c3 = quantize_e4m3<MODE>(v[3], i3, rnd[3]);
         return __byte_perm(__byte_perm(c0, c1, 0x0040), __byte_perm(c2, c3, 0x0040), 0x5410);
@@ -349,7 +360,8 @@ __device__ __forceinline__ uint32_t quantize4_rt(int mode, const float v[4], flo
         case 0: return quantize4<0>(v, i0, i1, i2, i3, rnd);
         case 1: return quantize4<1>(v, i0, i1, i2, i3, rnd);
         case 2: return quantize4<2>(v, i0, i1, i2, i3, rnd);
-        default: return quantize4<3>(v, i0, i1, i2, i3, rnd);
+        case 3: return quantize4<3>(v, i0, i1, i2, i3, rnd);
+        default: return quantize4<MODE_SR>(v, i0, i1, i2, i3, rnd);      // MODE_SR8: thresholds already in word form
     }
 }
 
@@ -427,7 +439,7 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
     using Raw = typename Raw4<T>::type;
     constexpr bool WANT_RM = (LAYOUT & 1) != 0, WANT_TR = (LAYOUT & 2) != 0;
     constexpr bool TWO_STEPS = WANT_TR && PER_ROW;     // transposed layout has its own step sizes
-    constexpr bool SRM = (MODE & MODE_SR) != 0;
+    constexpr bool SRM = (MODE & MODE_SR) != 0, SR8 = (MODE & MODE_SR8) != 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t c = c0 + lane * 4;
     const bool col_ok = FULL || c < P.cols;             // cols % 4 == 0: a group is all in or all out
@@ -471,12 +483,34 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
         if (it + 1 < 4) load_quad(it + 1, nxt, inv_nxt);
         const int rq = TR16 ? warp * 4 + it : warp + 8 * it;
         uint32_t wr[4], wt[4];
+        uint32_t sw[4] = {0u, 0u, 0u, 0u};     // 8-bit mode: stream word of this thread's 4 elements, per row
+        if constexpr (SR8) {
+            // one Philox block covers 16 consecutive elements = the 4-element groups of 4 neighbouring
+            // lanes.  Lane 4 g + j computes the block of row j of the quad; a 4 x 4 transpose over the four
+            // lanes then gives each lane word j of the blocks of rows 0 .. 3.
+            const int j4 = lane & 3;
+            const uint64_t i16 = P.index_offset + (uint64_t)(r0 + rq * 4 + j4) * (uint64_t)P.cols + (uint64_t)(c0 + (lane >> 2) * 16);
+            philox_rounds((uint32_t)(i16 >> 4), (uint32_t)(i16 >> 36), P.keys, sw);
+            {
+                const bool hi = (j4 & 2) != 0;
+                const uint32_t r0w = __shfl_xor_sync(0xFFFFFFFFu, hi ? sw[0] : sw[2], 2);
+                const uint32_t r1w = __shfl_xor_sync(0xFFFFFFFFu, hi ? sw[1] : sw[3], 2);
+                if (hi) { sw[0] = r0w; sw[1] = r1w; } else { sw[2] = r0w; sw[3] = r1w; }
+            }
+            {
+                const bool odd = (j4 & 1) != 0;
+                const uint32_t r0w = __shfl_xor_sync(0xFFFFFFFFu, odd ? sw[0] : sw[1], 1);
+                const uint32_t r1w = __shfl_xor_sync(0xFFFFFFFFu, odd ? sw[2] : sw[3], 1);
+                if (odd) { sw[0] = r0w; sw[2] = r1w; } else { sw[1] = r0w; sw[3] = r1w; }
+            }
+        }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const uint32_t tr = (uint32_t)rq * 4 + i;
             float v[4];
             widen(cur[i], v);
             uint32_t rnd[4] = {0u, 0u, 0u, 0u};
+            if constexpr (SR8) sr8_words(sw[i], rnd);
             if constexpr (SRM) {
                 if constexpr (FULL) {
                     philox_rounds(jb_lo + tr * j_row, jb_hi, P.keys, rnd);
@@ -587,15 +621,17 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
                 float v[4];
                 load4(x + r * P.ld, c, P.cols, P.vec_in != 0, v);
                 uint32_t rnd[4] = {0u, 0u, 0u, 0u};
-                if (sr) {
+                if (sr || (P.mode & MODE_SR8)) {
+                    const bool sr8 = (P.mode & MODE_SR8) != 0;        // 16 elements per block, one byte each
                     const uint64_t i0 = P.index_offset + (uint64_t)r * (uint64_t)P.cols + (uint64_t)c;
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const uint64_t ie = i0 + e, jb = ie >> 2;
+                        const uint64_t ie = i0 + e, jb = sr8 ? ie >> 4 : ie >> 2;
                         uint32_t o[4];
                         philox_rounds((uint32_t)jb, (uint32_t)(jb >> 32), P.keys, o);
-                        const uint32_t s = (uint32_t)ie & 3u;
-                        rnd[e] = s == 0 ? o[0] : s == 1 ? o[1] : s == 2 ? o[2] : o[3];
+                        const uint32_t s = sr8 ? (uint32_t)(ie >> 2) & 3u : (uint32_t)ie & 3u;
+                        const uint32_t w = s == 0 ? o[0] : s == 1 ? o[1] : s == 2 ? o[2] : o[3];
+                        rnd[e] = sr8 ? ((((w >> (8 * ((uint32_t)ie & 3u))) & 0xFFu) << 24) | 0x00800000u) : w;
                     }
                 }
                 const float inv_r = P.per_row ? P.inv_rm[want_rm ? r : 0] : inv_tensor;
@@ -649,7 +685,8 @@ static void launch_fast_mode(int mode, int layout, bool per_row, const void* x, 
         case 0: launch_fast_layout<T, 0>(layout, per_row, x, P, grid, st); break;
         case 1: launch_fast_layout<T, 1>(layout, per_row, x, P, grid, st); break;
         case 2: launch_fast_layout<T, 2>(layout, per_row, x, P, grid, st); break;
-        default: launch_fast_layout<T, 3>(layout, per_row, x, P, grid, st); break;
+        case 3: launch_fast_layout<T, 3>(layout, per_row, x, P, grid, st); break;
+        default: launch_fast_layout<T, MODE_SR8>(layout, per_row, x, P, grid, st); break;
     }
 }
 static void launch_fast(srq_dtype_t dt, int mode, int layout, bool per_row, const void* x, const QuantParams& P, unsigned grid,
@@ -737,7 +774,8 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         P.index_offset = a.q.index_offset;
         P.keys = make_philox_keys(a.q.seed, a.q.tensor_id);
         P.sr = a.q.round == SRQ_SR;
-        P.mode = (P.sr ? MODE_SR : 0) | (e4m3 ? MODE_E4M3 : 0);
+        const bool sr8 = a.q.round == SRQ_SR8;
+        P.mode = sr8 ? MODE_SR8 : ((P.sr ? MODE_SR : 0) | (e4m3 ? MODE_E4M3 : 0));
         P.per_row = per_row;
         P.codes_rm = a.codes_rm; P.ld_rm = a.ld_rm;
         P.codes_tr = a.codes_tr; P.ld_tr = a.ld_tr;
@@ -746,7 +784,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         P.vec_rm = want_rm && ((uintptr_t)a.codes_rm % 4 == 0) && (a.ld_rm % 4 == 0);
         P.vec_tr = want_tr && ((uintptr_t)a.codes_tr % 4 == 0) && (a.ld_tr % 4 == 0);
         P.vec_tr16 = want_tr && ((uintptr_t)a.codes_tr % 16 == 0) && (a.ld_tr % 16 == 0);
-        const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) &&
+        const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && (!sr8 || (cols % 16 == 0 && a.q.index_offset % 16 == 0)) && a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) &&
                           (!want_tr || (P.vec_tr && rows % 4 == 0));
         const unsigned grid = (unsigned)(((cols + Q_TILE - 1) / Q_TILE) * ((rows + Q_TILE - 1) / Q_TILE));
         if (fast) launch_fast(a.dt, P.mode, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);

@@ -174,3 +174,9 @@ def test_overflowing_contraction_is_refused():
     assert e.value.status == 4
     srq.qlinear_bwd_weight(dY, A, srq.QSpec(4), srq.QSpec(8), dW)       # 7 * 127 * T fits
     assert torch.count_nonzero(dW).item() == 0
+
+
+def test_layer_with_eight_random_bits_per_element():
+    T, N, K = 264, 400, 336
+    A, W, dY = synth.layer_inputs(T, N, K, seed=6, device="cuda", std_dy=1e-3)
+    all_passes(A, W, dY, layer_specs(srq.PER_TENSOR, srq.SR8, seed=4, bits_fwd=8, bits_bwd=4))

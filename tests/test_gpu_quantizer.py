@@ -183,3 +183,21 @@ def test_absmax_entry_point_and_a_known_absmax(dtype):
     with pytest.raises(srq.SrqError):                    # only with one step size per tensor
         srq.sr_quantize(x, srq.QSpec(8, srq.PER_ROW, absmax=m), torch.empty((300, 388), dtype=torch.int8, device="cuda"),
                         torch.empty(300, device="cuda"))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("scale", [srq.PER_TENSOR, srq.PER_ROW])
+def test_eight_random_bits_per_element(dtype, scale):
+    """SRQ_SR8 against the oracle: aligned tiles (one Philox block per 16 elements, shared by four lanes),
+    ragged shapes and index offsets that break the 16-element alignment (element-wise path)."""
+    x = synth.with_outliers((300, 400), seed=12, dtype=dtype, device="cuda")
+    _check(x, 8, scale, srq.SR8, seed=7, tid=3, off=0)
+    _check(x, 4, scale, srq.SR8, seed=7, tid=3, off=2 ** 36 + 32)
+    _check(x, 8, scale, srq.SR8, seed=1, tid=2, off=8)                 # offset not a multiple of 16
+    _check(x[:, :388].contiguous(), 6, scale, srq.SR8, seed=2)          # width not a multiple of 16
+    y = synth.normal((131, 259), 1.0, seed=5, dtype=dtype, device="cuda")
+    _check(y, 8, scale, srq.SR8, seed=3, off=5)
+    _check(x, 8, scale, srq.SR8, want_rm=False, want_tr=True)
+    with pytest.raises(srq.SrqError):                                    # integer grid only
+        srq.sr_quantize(x, srq.QSpec(8, scale, srq.SR8, format=srq.GRID_E4M3),
+                        torch.empty((300, 400), dtype=torch.int8, device="cuda"), torch.empty(300, device="cuda"))
