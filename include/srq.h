@@ -302,6 +302,12 @@ srq_status_t qlinear_bwd_ex(const void *dY, const void *A, const void *W, srq_dt
  * was last cleared (every entry point clears it when it starts). */
 srq_status_t srq_poll_status(void *ws, void *cuda_stream);
 
+/* Self-test of the failure path of the product kernel: enqueues a one-thread kernel that waits, for
+ * at most limit_us microseconds (1 .. 1000000), on a barrier that nothing signals.  The wait gives
+ * up in the same way the bounded waits of the product kernel do: the status word of ws receives
+ * SRQ_ERR_TIMEOUT (read it with srq_poll_status), the kernel returns and the context stays usable. */
+srq_status_t srq_selftest_bounded_wait(void *ws, size_t ws_bytes, uint32_t limit_us, void *cuda_stream);
+
 /* Static, human-readable name of a status. */
 const char *srq_status_string(srq_status_t s);
 

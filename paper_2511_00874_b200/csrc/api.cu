@@ -493,6 +493,14 @@ srq_status_t qlinear_bwd_ex(const void* dY, const void* A, const void* W, srq_dt
     return run_bwd(dY, A, W, dt, T, N, K, qdY, qA, qW, dA, dW, output_dA, output_dW, dbg_input, dbg_weight, ws, ws_bytes, cuda_stream);
 }
 
+srq_status_t srq_selftest_bounded_wait(void* ws, size_t ws_bytes, uint32_t limit_us, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!ws || !aligned_to(ws, 256) || limit_us == 0 || limit_us > 1000000u) return SRQ_ERR_INVALID_ARG;
+    if (ws_bytes < sizeof(WsHeader)) return SRQ_ERR_WORKSPACE;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    return launch_bounded_wait_probe(&((WsHeader*)ws)->status, (uint64_t)limit_us * 1000ull, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+}
+
 srq_status_t srq_poll_status(void* ws, void* cuda_stream) {
     if (!ws) return SRQ_ERR_INVALID_ARG;
     uint32_t v = 0;

@@ -93,14 +93,15 @@ __device__ __forceinline__ uint64_t global_ns() {
     return t;
 }
 // Bounded wait: false if the limit passed or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint64_t limit_ns = WAIT_LIMIT_NS) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
     for (uint32_t spin = 0;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 63u) == 63u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+            if (global_ns() - t0 > limit_ns) return false;
         }
     }
 }
@@ -661,6 +662,25 @@ dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_
         if (acc_out)
             for (int e = 0; e < 4 && c + e < N; ++e) acc_out[r * N + c + e] = av[e];
     }
+}
+
+// Self-test of the bounded wait: one thread waits on a barrier that nothing ever arrives on, with a
+// short limit; the wait gives up, the status word receives SRQ_ERR_TIMEOUT and the kernel returns.
+__global__ void bounded_wait_probe_kernel(uint32_t* status, uint64_t limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ volatile uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait(&bar, 0u, &abort_flag, limit_ns)) record_status(status, SRQ_ERR_TIMEOUT);
+    }
+}
+
+cudaError_t launch_bounded_wait_probe(uint32_t* status, uint64_t limit_ns, cudaStream_t stream) {
+    bounded_wait_probe_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
+    ++g_launches;
+    return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------

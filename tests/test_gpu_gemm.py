@@ -125,3 +125,19 @@ def test_output_pitch_and_ragged_edges_on_the_block_store_path(M, N, Kc, pad):
     guard = full.clone()
     guard[1:M + 1, (4 if pad else 0):(4 if pad else 0) + N] = 7.5
     assert bool((guard == 7.5).all()), "a store went outside the output"
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
+    """Failure detection without a fault: a wait on a barrier that nothing signals gives up after its
+    limit, the status word says so, and the next call on the same context works."""
+    import time
+    ws = srq.new_workspace(srq.srq_gemm_workspace_bytes(128, 256))
+    t0 = time.perf_counter()
+    srq.srq_selftest_bounded_wait(ws, limit_us=2000)
+    assert srq.srq_poll_status(ws) == 7
+    assert time.perf_counter() - t0 < 1.0
+    assert srq.status_string(7) == "bounded wait in a kernel ran out"
+    a, b = _codes(128, 256, 1), _codes(256, 256, 2)
+    one = torch.ones(1, device="cuda")
+    out, acc = _run(a, b, one, one)
+    assert np.array_equal(acc, oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy()))
