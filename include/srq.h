@@ -302,6 +302,12 @@ srq_status_t qlinear_bwd_ex(const void *dY, const void *A, const void *W, srq_dt
  * was last cleared (every entry point clears it when it starts). */
 srq_status_t srq_poll_status(void *ws, void *cuda_stream);
 
+/* Host-side planning rule of the product kernel, exposed so that it can be checked without a device:
+ * with `tiles` output tiles, `k_blocks` 128-byte blocks along the contraction and `groups` tiles
+ * running at a time, tiles [0, *full_tiles) are computed whole and each remaining tile in *splits
+ * parts (*splits == 1: nothing is split).  Invalid arguments give 0, 0. */
+void srq_plan_splits(int64_t tiles, int32_t k_blocks, int32_t groups, int32_t *full_tiles, int32_t *splits);
+
 /* Self-test of the failure path of the product kernel: enqueues a one-thread kernel that waits, for
  * at most limit_us microseconds (1 .. 1000000), on a barrier that nothing signals.  The wait gives
  * up in the same way the bounded waits of the product kernel do: the status word of ws receives

@@ -28,7 +28,7 @@ GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
            "sr_quantize", "sr_quantize_static", "srq_absmax", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
            "srq_gemm_i8_ex", "qlinear_fwd_ex", "qlinear_bwd_ex",
-           "srq_poll_status", "srq_status_string", "srq_launch_count", "srq_selftest_bounded_wait"]
+           "srq_poll_status", "srq_status_string", "srq_launch_count", "srq_selftest_bounded_wait", "srq_plan_splits"]
 
 
 class SrqError(RuntimeError):
@@ -119,6 +119,8 @@ def lib() -> ctypes.CDLL:
     L.qlinear_bwd_ex.restype = ctypes.c_int
     L.srq_selftest_bounded_wait.argtypes = [vp, sz, ctypes.c_uint32, vp]
     L.srq_selftest_bounded_wait.restype = ctypes.c_int
+    L.srq_plan_splits.argtypes = [i64, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    L.srq_plan_splits.restype = None
     L.srq_poll_status.argtypes = [vp, vp]
     L.srq_poll_status.restype = ctypes.c_int
     L.srq_status_string.argtypes = [ctypes.c_int]
@@ -426,6 +428,13 @@ def qlinear_bwd_ex(dY: torch.Tensor, A: torch.Tensor, W: torch.Tensor, qdY: QSpe
                               ctypes.byref(o1) if o1 is not None else None, None, None,
                               ws.data_ptr(), ws.numel(), _stream())
     _check(st, "qlinear_bwd_ex")
+
+
+def srq_plan_splits(tiles: int, k_blocks: int, groups: int):
+    """(full_tiles, splits) the product kernel would use (host-side rule, no device needed)."""
+    f, s = ctypes.c_int32(), ctypes.c_int32()
+    lib().srq_plan_splits(tiles, k_blocks, groups, ctypes.byref(f), ctypes.byref(s))
+    return f.value, s.value
 
 
 def srq_selftest_bounded_wait(ws: torch.Tensor, limit_us: int = 1000) -> None:

@@ -493,6 +493,13 @@ srq_status_t qlinear_bwd_ex(const void* dY, const void* A, const void* W, srq_dt
     return run_bwd(dY, A, W, dt, T, N, K, qdY, qA, qW, dA, dW, output_dA, output_dW, dbg_input, dbg_weight, ws, ws_bytes, cuda_stream);
 }
 
+void srq_plan_splits(int64_t tiles, int32_t k_blocks, int32_t groups, int32_t* full_tiles, int32_t* splits) {
+    if (!full_tiles || !splits) return;
+    *full_tiles = 0; *splits = 0;
+    if (tiles <= 0 || k_blocks <= 0 || groups <= 0 || tiles > 2147483647ll) return;
+    gemm_plan_splits(tiles, k_blocks, groups, full_tiles, splits);
+}
+
 srq_status_t srq_selftest_bounded_wait(void* ws, size_t ws_bytes, uint32_t limit_us, void* cuda_stream) {
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (!ws || !aligned_to(ws, 256) || limit_us == 0 || limit_us > 1000000u) return SRQ_ERR_INVALID_ARG;

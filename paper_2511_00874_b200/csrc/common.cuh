@@ -121,6 +121,8 @@ struct GemmArgs {
     void* splitk_ws; size_t splitk_ws_bytes;   // int32 [M,N] partial sums
 };
 size_t gemm_splitk_bytes(int64_t M, int64_t N);
+// Host-side planning of the split contraction (exposed for tests).
+void gemm_plan_splits(int64_t tiles, int32_t num_kb, int groups, int32_t* full_tiles, int32_t* splits);
 // One thread waits (at most limit_ns) on a barrier nobody signals and records SRQ_ERR_TIMEOUT.
 cudaError_t launch_bounded_wait_probe(uint32_t* status, uint64_t limit_ns, cudaStream_t stream);
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream);

@@ -778,6 +778,10 @@ static void plan_splits(int64_t tiles, int32_t num_kb, int groups, int32_t* full
     *full_tiles = (int32_t)full; *splits = s;
 }
 
+void gemm_plan_splits(int64_t tiles, int32_t num_kb, int groups, int32_t* full_tiles, int32_t* splits) {
+    plan_splits(tiles, num_kb, groups, full_tiles, splits);
+}
+
 // What launch_gemm_i8 may use: int32 partial sums of the split tiles (fewer than one round of tiles,
 // i.e. at most 160 blocks of 128 x 256 on any device this runs on).
 size_t gemm_splitk_bytes(int64_t M, int64_t N) {

@@ -100,3 +100,24 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "libsrq.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         binding.lib()
+
+
+def test_split_planning_rule(L):
+    """Host logic of the product: which tiles are split along the contraction and into how many parts."""
+    plan = binding.srq_plan_splits
+    for groups in (74, 148, 1, 7):
+        for tiles in list(range(1, 40)) + [73, 74, 75, 148, 176, 222, 256, 512, 600, 4096]:
+            for kb in (1, 8, 15, 16, 17, 32, 64, 512):
+                full, s = plan(tiles, kb, groups)
+                assert 0 <= full <= tiles and s >= 1
+                if s == 1:
+                    assert full == tiles                      # nothing split
+                    continue
+                assert full % groups == 0 and full < tiles      # whole rounds first, the rest is split
+                per = -(-kb // s)
+                assert per >= 8 and (s - 1) * per < kb          # every part has at least 8 k-blocks, none is empty
+                assert (tiles - full) * s <= groups or s == kb // 8   # the split units fit into one round
+    assert plan(256, 512, 74) == (222, 2)                   # dW of the benchmark layer: last 34 tiles in two parts
+    assert plan(9, 512, 74) == (0, 8)                       # 768 x 768 output: every tile in eight parts
+    assert plan(4096, 32, 74) == (4096, 1)                  # many rounds: not worth splitting
+    assert plan(0, 1, 1) == (0, 0) and plan(5, 0, 3) == (0, 0)
