@@ -264,11 +264,16 @@ srq_status_t qlinear_bwd(const void *dY, const void *A, const void *W, srq_dtype
  *               codes given, the fp32 output pointer of the call may be NULL.
  *   absmax      device [1], holding a non-negative number (usually 0) on entry: raised to
  *               max |result|, from which the caller derives the step size of its next step.
+ *   out_bf16    1: the output pointer of the call addresses bfloat16 numbers (pass it cast to
+ *               float *; its pitch counts bfloat16 elements): each binary32 result is rounded to
+ *               the nearest bfloat16, ties to even, as it is stored, which halves the bytes the
+ *               product writes.  Codes and absmax still come from the binary32 result.  Not with
+ *               accumulate (SRQ_ERR_UNSUPPORTED): running sums stay in binary32.
  * Products with q or absmax set are never split along the contraction.
  */
 typedef struct {
     int32_t accumulate;
-    int32_t reserved;
+    int32_t out_bf16;
     const srq_qspec_t *q;
     const float *step;
     int8_t *codes;

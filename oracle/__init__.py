@@ -111,6 +111,8 @@ def lib() -> ctypes.CDLL:
         L.orc_requantize.restype = None
         L.orc_accumulate.argtypes = [vp, vp, i64]
         L.orc_accumulate.restype = None
+        L.orc_to_bf16.argtypes = [vp, i64, vp]
+        L.orc_to_bf16.restype = None
         L.orc_num_threads.argtypes = []
         L.orc_num_threads.restype = ctypes.c_int
     return _lib
@@ -378,3 +380,11 @@ def accumulate(dst, src) -> np.ndarray:
     assert d.shape == s.shape
     lib().orc_accumulate(_ptr(d), _ptr(s), d.size)
     return d
+
+
+def to_bf16(x) -> np.ndarray:
+    """Bit patterns (uint16) of the bfloat16 numbers nearest to the binary32 values, ties to even."""
+    v = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.zeros(v.shape, dtype=np.uint16)
+    lib().orc_to_bf16(_ptr(v), v.size, _ptr(out))
+    return out

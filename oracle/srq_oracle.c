@@ -649,3 +649,21 @@ void orc_accumulate(float *dst, const float *src, int64_t n)
 {
     for (int64_t i = 0; i < n; ++i) dst[i] = dst[i] + src[i];
 }
+
+/*
+ * A product stored as bfloat16 (the optional narrow output of the dequantizing step): the
+ * bfloat16 number nearest to the binary32 value, ties to the one whose last kept bit is even.
+ * bfloat16 is the upper half of the binary32 pattern, so the two neighbours are the pattern with
+ * its low 16 bits cleared and that plus one unit of the 17th bit; the discarded half decides.
+ * Finite inputs only (a value beyond the largest bfloat16 goes to infinity, as the format says).
+ */
+void orc_to_bf16(const float *x, int64_t n, uint16_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        uint32_t b;
+        memcpy(&b, &x[i], 4);
+        uint32_t keep = b >> 16, rest = b & 0xFFFFu;
+        if (rest > 0x8000u || (rest == 0x8000u && (keep & 1u))) keep += 1u;
+        out[i] = (uint16_t)keep;
+    }
+}

@@ -51,7 +51,7 @@ class _DebugOut(ctypes.Structure):
 
 
 class _Output(ctypes.Structure):
-    _fields_ = [("accumulate", ctypes.c_int32), ("reserved", ctypes.c_int32), ("q", ctypes.POINTER(_QSpec)),
+    _fields_ = [("accumulate", ctypes.c_int32), ("out_bf16", ctypes.c_int32), ("q", ctypes.POINTER(_QSpec)),
                 ("step", ctypes.c_void_p), ("codes", ctypes.c_void_p), ("ld_codes", ctypes.c_int64),
                 ("absmax", ctypes.c_void_p)]
 
@@ -358,23 +358,30 @@ def qlinear_bwd(dY: torch.Tensor, A: torch.Tensor, W: torch.Tensor, qdY: QSpec, 
 @dataclass
 class Output:
     """Output options of a product (srq_output_t): accumulate into out, codes of Q(result) with a
-    caller-supplied step (q, step, codes), absmax of the result."""
+    caller-supplied step (q, step, codes), absmax of the result.  A bfloat16 output tensor passed
+    to one of the *_ex calls sets the struct's out_bf16 member."""
     accumulate: bool = False
     q: Optional[QSpec] = None
     step: Optional[torch.Tensor] = None
     codes: Optional[torch.Tensor] = None
     absmax: Optional[torch.Tensor] = None
 
-    def c(self):
+    def c(self, out_bf16: bool = False):
         cq = self.q.c() if self.q is not None else None
-        o = _Output(int(self.accumulate), 0, ctypes.pointer(cq) if cq is not None else None, _ptr(self.step),
+        o = _Output(int(self.accumulate), int(out_bf16), ctypes.pointer(cq) if cq is not None else None, _ptr(self.step),
                     _ptr(self.codes), self.codes.stride(0) if self.codes is not None else 0, _ptr(self.absmax))
         o._keep = cq                      # the struct points into cq
         return o
 
 
-def _opt(o: Optional[Output]):
-    return None if o is None else o.c()
+def _opt(o: Optional[Output], out: Optional[torch.Tensor] = None):
+    """The C struct of the options; a bfloat16 output tensor selects out_bf16 by itself."""
+    bf16 = out is not None and out.dtype == torch.bfloat16
+    if out is not None and not bf16 and out.dtype != torch.float32:
+        raise TypeError("the output of a product is float32 or bfloat16")
+    if o is None:
+        return Output().c(True) if bf16 else None
+    return o.c(bf16)
 
 
 def srq_gemm_i8_ex(a: torch.Tensor, b: torch.Tensor, s_row: torch.Tensor, s_col: torch.Tensor,
@@ -387,7 +394,7 @@ def srq_gemm_i8_ex(a: torch.Tensor, b: torch.Tensor, s_row: torch.Tensor, s_col:
     N = b.shape[0]
     if ws is None:
         ws = new_workspace(srq_gemm_workspace_bytes(M, N), a.device)
-    co = _opt(output)
+    co = _opt(output, out)
     st = lib().srq_gemm_i8_ex(a.data_ptr(), a.stride(0), b.data_ptr(), b.stride(0), M, N, Kc,
                               s_row.data_ptr(), int(s_row.numel() != 1), s_col.data_ptr(), int(s_col.numel() != 1),
                               _ptr(out), out.stride(0) if out is not None else 0, _ptr(acc_out),
@@ -405,7 +412,7 @@ def qlinear_fwd_ex(A: torch.Tensor, W: torch.Tensor, qA: QSpec, qW: QSpec, Y: Op
         ws = new_workspace(srq_workspace_bytes(T, N, K), A.device)
     c0, c1 = qA.c(), qW.c()
     cd = dbg.c() if dbg is not None else None
-    co = _opt(output)
+    co = _opt(output, Y)
     st = lib().qlinear_fwd_ex(A.data_ptr(), W.data_ptr(), _dtype_of(A), T, N, K, ctypes.byref(c0), ctypes.byref(c1),
                               _ptr(Y), ctypes.byref(co) if co is not None else None,
                               ctypes.byref(cd) if cd is not None else None, ws.data_ptr(), ws.numel(), _stream())
@@ -421,7 +428,7 @@ def qlinear_bwd_ex(dY: torch.Tensor, A: torch.Tensor, W: torch.Tensor, qdY: QSpe
     if ws is None:
         ws = new_workspace(srq_workspace_bytes(T, N, K), dY.device)
     c0, c1, c2 = qdY.c(), qA.c(), qW.c()
-    o0, o1 = _opt(output_dA), _opt(output_dW)
+    o0, o1 = _opt(output_dA, dA), _opt(output_dW, dW)
     st = lib().qlinear_bwd_ex(dY.data_ptr(), A.data_ptr(), W.data_ptr(), _dtype_of(dY), T, N, K,
                               ctypes.byref(c0), ctypes.byref(c1), ctypes.byref(c2), _ptr(dA), _ptr(dW),
                               ctypes.byref(o0) if o0 is not None else None,

@@ -73,13 +73,16 @@ def case_gemm(a):
     A = torch.randint(-127, 128, (a.M, a.K), generator=g, dtype=torch.int8, device="cuda")
     Bm = torch.randint(-127, 128, (a.N, a.K), generator=g, dtype=torch.int8, device="cuda")
     one = torch.ones(1, device="cuda")
-    out = torch.empty((a.M, a.N), device="cuda")
+    out_bf16 = getattr(a, "out", "f32") == "bf16"
+    out = torch.empty((a.M, a.N), dtype=torch.bfloat16 if out_bf16 else torch.float32, device="cuda")
     ws = B.new_workspace(B.srq_gemm_workspace_bytes(a.M, a.N))
     if getattr(a, "grid", "int") == "e4m3":
         A, Bm = A.view(torch.uint8), Bm.view(torch.uint8)
         A[(A & 0x7F) == 0x7F] = 0x38          # no NaN codes
         Bm[(Bm & 0x7F) == 0x7F] = 0x38
         fn = lambda: B.srq_gemm_e4m3(A, Bm, one, one, out, None, ws)
+    elif out_bf16:
+        fn = lambda: B.srq_gemm_i8_ex(A, Bm, one, one, out, None, None, ws)
     else:
         fn = lambda: B.srq_gemm_i8(A, Bm, one, one, out, None, ws)
     small = (a.M + a.N) * a.K + 4 * a.M * a.N < 2 * L2_BYTES
@@ -87,7 +90,7 @@ def case_gemm(a):
     assert B.srq_poll_status(ws) == 0
     ops = 2.0 * a.M * a.N * a.K
     return {"op": "srq_gemm_e4m3" if getattr(a, "grid", "int") == "e4m3" else "srq_gemm_i8", "M": a.M, "N": a.N, "K": a.K, "ms": med, "ms_best": best, "TOPS": ops / med / 1e9,
-            "out_GBps": 4.0 * a.M * a.N / med / 1e6}
+            "out": "bf16" if out_bf16 else "f32", "out_GBps": out.element_size() * a.M * a.N / med / 1e6}
 
 
 def _layer_fn(A, W, dY, q, Y, dA, dW, ws):
@@ -250,6 +253,7 @@ def main(argv=None):
             p.add_argument("--M", type=int, default=8192)
             p.add_argument("--N", type=int, default=4096)
             p.add_argument("--K", type=int, default=4096)
+            p.add_argument("--out", default="f32", choices=["f32", "bf16"], help="type the product is stored in (int grid only)")
         if name == "layer":
             p.add_argument("--T", type=int, default=16384)
             p.add_argument("--N", type=int, default=4096)

@@ -25,7 +25,10 @@ srq_status_t make_out_options(const srq_output_t* o, int64_t N, bool have_out, O
     if (!o) return have_out ? SRQ_OK : SRQ_ERR_INVALID_ARG;
     if (o->accumulate != 0 && o->accumulate != 1) return SRQ_ERR_INVALID_ARG;
     if (o->accumulate && !have_out) return SRQ_ERR_INVALID_ARG;
+    if (o->out_bf16 != 0 && o->out_bf16 != 1) return SRQ_ERR_INVALID_ARG;
+    if (o->out_bf16 && o->accumulate) return SRQ_ERR_UNSUPPORTED;   // sums are kept in binary32
     r->accumulate = o->accumulate;
+    r->out_bf16 = o->out_bf16;
     if (o->q) {
         srq_status_t s = check_qspec(o->q);
         if (s != SRQ_OK) return s;
@@ -127,7 +130,8 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
     }
     if (Kc == 0) {   // empty contraction: the product is zero
         if (!out || opt.accumulate) return SRQ_OK;
-        return cudaMemset2DAsync(out, (size_t)Nn * 4, 0, (size_t)Nn * 4, (size_t)M, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+        const size_t eb = opt.out_bf16 ? 2 : 4;
+        return cudaMemset2DAsync(out, (size_t)Nn * eb, 0, (size_t)Nn * eb, (size_t)M, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
     }
 
     GemmArgs g;
@@ -295,7 +299,7 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
     // dA[T,K] = Q(dY)[T,N] . Q(W)^T[K,N]
     if (T > 0 && K > 0) {
         if (N == 0) {
-            if (dA && !opt_in.accumulate && cudaMemset2DAsync(dA, (size_t)K * 4, 0, (size_t)K * 4, (size_t)T, st) != cudaSuccess) return SRQ_ERR_CUDA;
+            if (dA && !opt_in.accumulate && cudaMemset2DAsync(dA, (size_t)K * (opt_in.out_bf16 ? 2 : 4), 0, (size_t)K * (opt_in.out_bf16 ? 2 : 4), (size_t)T, st) != cudaSuccess) return SRQ_ERR_CUDA;
         } else {
             GemmArgs g;
             g.a = cd[0]; g.lda = p.pitch_n; g.b = cd[2]; g.ldb = p.pitch_n; g.M = T; g.N = K; g.Kc = N; g.kind = kind;
@@ -309,7 +313,7 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
     // dW[N,K] = Q(dY)^T[N,T] . Q(A)^T[K,T]
     if (N > 0 && K > 0) {
         if (T == 0) {
-            if (dW && !opt_w.accumulate && cudaMemset2DAsync(dW, (size_t)K * 4, 0, (size_t)K * 4, (size_t)N, st) != cudaSuccess) return SRQ_ERR_CUDA;
+            if (dW && !opt_w.accumulate && cudaMemset2DAsync(dW, (size_t)K * (opt_w.out_bf16 ? 2 : 4), 0, (size_t)K * (opt_w.out_bf16 ? 2 : 4), (size_t)N, st) != cudaSuccess) return SRQ_ERR_CUDA;
         } else {
             GemmArgs g;
             g.a = cd[1]; g.lda = p.pitch_t; g.b = cd[3]; g.ldb = p.pitch_t; g.M = N; g.N = K; g.Kc = T; g.kind = kind;
@@ -468,6 +472,7 @@ srq_status_t srq_gemm_i8_ex(const int8_t* a, int64_t lda, const int8_t* b, int64
     GemmArgs g;
     const srq_status_t so = make_out_options(output, N, out != nullptr, &g.opt);
     if (so != SRQ_OK) return so;
+    if (!aligned_to(out, g.opt.out_bf16 ? 2 : 4)) return SRQ_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return SRQ_OK;
     uint32_t* status = &((WsHeader*)ws)->status;
     if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;

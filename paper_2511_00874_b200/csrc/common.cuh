@@ -100,6 +100,7 @@ cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, 
 // What else a product does with its results (all optional).
 struct OutOptions {
     int32_t accumulate = 0;          // out += result instead of out = result
+    int32_t out_bf16 = 0;            // out holds bfloat16 [M, ldo]: each result rounded to nearest even
     int32_t requant = 0;             // also write Q(result) as int8 codes with a given step size
     int32_t rq_sr = 0;               // stochastic rounding (else round to nearest)
     float rq_lim = 0.0f;             // qmax * 2^24: saturation bound of the fixed-point quotient

@@ -27,6 +27,7 @@
 // Every wait is bounded by a wall-clock limit; on expiry the CTA records SRQ_ERR_TIMEOUT,
 // stops issuing work, waits (bounded) for what it has in flight, frees its TMEM and returns.
 #include <cuda.h>
+#include <cuda_bf16.h>
 
 #include <mutex>
 
@@ -165,6 +166,12 @@ __device__ __forceinline__ void stage_block(uint32_t stage, int lane, const uint
     for (int q = 0; q < 8; ++q)
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (uint32_t)((q ^ (lane & 7)) << 4)),
                      "r"(w[4 * q]), "r"(w[4 * q + 1]), "r"(w[4 * q + 2]), "r"(w[4 * q + 3]) : "memory");
+}
+
+// Two binary32 numbers rounded to nearest even bfloat16, the first in the low half.
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -510,7 +517,37 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
             const uint32_t stage = smem_u32(out_stage + (warp - 2) * OUT_STAGE_BYTES);
             const int32_t wrow = (int32_t)(row0 + quarter * 32);           // first row of this warp's blocks
-            if (whole && P.tma_out) {
+            if (whole && P.tma_out && P.opt.out_bf16) {
+                // two 32-column blocks at a time: 64 bfloat16 results per row fill the 128-byte rows
+                // of the staging block, stored as one 32 x 64 box
+#pragma unroll 1
+                for (int j = 0; j < BN / 64; ++j) {
+                    uint32_t w[32];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + j * 64 + h * 32, v);
+                        tmem_ld_wait();
+                        const float* sc = &T->s_col[buf][j * 64 + h * 32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            v[i] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[i]), __fmul_rn(sr, sc[i])));
+                        output_options(P, v, row, (int32_t)col_base + j * 64 + h * 32, rq_inv, amax);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) w[h * 16 + i] = pack_bf16(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                    }
+                    const int32_t col0 = (int32_t)col_base + j * 64;
+                    if (lane == 0) bulk_wait_read();
+                    __syncwarp();
+                    stage_block(stage, lane, w);
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && wrow < P.M && col0 < P.N) { tma_store_2d(&map_out, stage, col0, wrow); bulk_commit(); }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
+            } else if (whole && P.tma_out) {
                 // registers -> swizzled shared-memory block -> one TMA store per 32 x 32 block
 #pragma unroll 1
                 for (int j = 0; j < BN / 32; ++j) {
@@ -561,7 +598,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int i = 0; i < 32; ++i)
                             v[i] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[i]), __fmul_rn(sr, sc[i])));
                         output_options(P, v, row, col0, rq_inv, amax);
-                        if (P.write_out) {
+                        if (P.write_out && P.opt.out_bf16) {
+                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(P.out) + row * P.ldo + col0;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (col0 + i < P.N) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                        } else if (P.write_out) {
                             float* dst = P.out + row * P.ldo + col0;
                             if (P.vec_out && col0 + 32 <= P.N) {
 #pragma unroll
@@ -633,7 +675,7 @@ __global__ void __launch_bounds__(256)
 dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_tile, int32_t tiles_n, int32_t tile_rows,
                int64_t M, int64_t N, const float* __restrict__ s_row, int32_t row_stride,
                const float* __restrict__ s_col, int32_t col_stride, float* __restrict__ out, int64_t ldo,
-               int32_t* __restrict__ acc_out, int vec, int accumulate) {
+               int32_t* __restrict__ acc_out, int vec, int accumulate, int out_bf16) {
     const int64_t per_tile = (int64_t)tile_rows * (BN / 4);
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_tiles * per_tile; g += (int64_t)gridDim.x * blockDim.x) {
         const int64_t t = g / per_tile, in_tile = g % per_tile;
@@ -648,6 +690,17 @@ dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_
 #pragma unroll
         for (int e = 0; e < 4; ++e)
             o[e] = (c + e < N) ? __fmul_rn(__int2float_rn(av[e]), __fmul_rn(sr, s_col[(c + e) * col_stride])) : 0.0f;
+        if (out_bf16) {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(out) + r * ldo + c;
+            if (vec && c + 4 <= N) {
+                *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3]));
+            } else {
+                for (int e = 0; e < 4 && c + e < N; ++e) dst[e] = __float2bfloat16_rn(o[e]);
+            }
+            if (acc_out)
+                for (int e = 0; e < 4 && c + e < N; ++e) acc_out[r * N + c + e] = av[e];
+            continue;
+        }
         float* dst = out + r * ldo + c;
         if (vec && c + 4 <= N) {
             float4 w = make_float4(o[0], o[1], o[2], o[3]);
@@ -715,13 +768,15 @@ static bool encode_operand(CUtensorMap* map, const int8_t* base, int64_t rows, i
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// [rows, cols] matrix of 32-bit elements with row pitch ld elements, boxes of 32 x 32, 128-byte swizzle.
+// [rows, cols] matrix of 32-bit (or bfloat16) elements with row pitch ld elements, boxes of 32 rows x
+// 128 bytes, 128-byte swizzle.
 static bool encode_output(CUtensorMap* map, void* base, CUtensorMapDataType dt, int64_t rows, int64_t cols, int64_t ld) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
+    const unsigned esize = dt == CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 ? 2 : 4;     // rows of a box are 128 bytes
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
-    cuuint32_t box[2] = {32, 32};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * esize};
+    cuuint32_t box[2] = {128 / esize, 32};
     cuuint32_t estr[2] = {1, 1};
     return enc(map, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -838,15 +893,18 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.s_col = g.s_col; P.col_stride = g.col_stride;
     P.out = g.out; P.ldo = g.ldo; P.acc_out = g.acc_out;
     P.status = status;
-    P.vec_out = g.out && ((uintptr_t)g.out % 16 == 0) && (g.ldo % 4 == 0);
+    const int out_vec_elems = g.opt.out_bf16 ? 8 : 4;      // elements per 16 bytes of output
+    P.vec_out = g.out && ((uintptr_t)g.out % 16 == 0) && (g.ldo % out_vec_elems == 0);
 
     // results leave through TMA stores when the output (and the partial sums) meet the 16-byte rules
     CUtensorMap map_out = map_a, map_part = map_a;       // placeholders when unused
     P.opt = g.opt;
     P.write_out = g.out != nullptr;
     P.rq_vec = g.opt.requant && ((uintptr_t)g.opt.rq_codes % 16 == 0) && (g.opt.rq_ld % 16 == 0);
-    P.tma_out = P.write_out && P.vec_out && !g.acc_out && g.M < (1ll << 31) && g.N < (1ll << 31) &&
-                encode_output(&map_out, g.out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.M, g.N, g.ldo);
+    // (a row must also END on a 16-byte boundary: a store that reaches over the edge of the tensor map
+    // was seen to write the whole last 16-byte piece of the row, into the columns of a wider buffer)
+    P.tma_out = P.write_out && P.vec_out && g.N % out_vec_elems == 0 && !g.acc_out && g.M < (1ll << 31) && g.N < (1ll << 31) &&
+                encode_output(&map_out, g.out, g.opt.out_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.M, g.N, g.ldo);
     if (P.splits > 1 && !encode_output(&map_part, P.part, CU_TENSOR_MAP_DATA_TYPE_INT32, split_tiles * BM * ctas, BN, BN))
         return SRQ_ERR_CUDA;
 
@@ -862,13 +920,13 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     ++g_launches;
     if (e != cudaSuccess) return SRQ_ERR_CUDA;
     if (P.splits > 1) {
-        const int vec = g.ldo % 4 == 0 && (uintptr_t)g.out % 16 == 0;
+        const int vec = g.ldo % 4 == 0 && (uintptr_t)g.out % 16 == 0;     // 16-byte (binary32) or 8-byte (bfloat16) stores
         const int64_t work = split_tiles * BM * ctas * (BN / 4);
         const int64_t blocks = (work + 255) / 256;
         const unsigned grid = (unsigned)(blocks < 8 * (int64_t)dev->sms ? blocks : 8 * (int64_t)dev->sms);
         dequant_kernel<<<grid, 256, 0, stream>>>(P.part, split_tiles, P.full_tiles, P.tiles_n, BM * ctas, g.M, g.N, g.s_row,
                                                  g.row_stride, g.s_col, g.col_stride, g.out, g.ldo, g.acc_out, vec,
-                                                 g.opt.accumulate);
+                                                 g.opt.accumulate, g.opt.out_bf16);
         ++g_launches;
         if (cudaGetLastError() != cudaSuccess) return SRQ_ERR_CUDA;
     }

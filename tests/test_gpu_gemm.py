@@ -108,7 +108,7 @@ def test_many_tiles_per_cta_and_freivalds():
     assert np.array_equal(out2, out)
 
 
-@pytest.mark.parametrize("M,N,Kc,pad", [(300, 260, 256, 0), (257, 36, 130, 4), (4096, 96, 512, 0), (520, 1000, 384, 24), (130, 70, 64, 1)])
+@pytest.mark.parametrize("M,N,Kc,pad", [(300, 260, 256, 0), (257, 36, 130, 4), (4096, 96, 512, 0), (520, 1000, 384, 24), (130, 70, 64, 1), (140, 258, 64, 2), (300, 521, 128, 3)])
 def test_output_pitch_and_ragged_edges_on_the_block_store_path(M, N, Kc, pad):
     """No raw sums requested: every result goes through shared memory and a clipped block store.
     The output has a row pitch larger than N and guard values around it that must survive."""

@@ -114,3 +114,81 @@ def test_option_errors_are_found_on_the_host():
     with pytest.raises(srq.SrqError):           # accumulate without an output
         srq.srq_gemm_i8_ex(a, b, one, one, None, srq.Output(accumulate=True, q=srq.QSpec(8), step=one,
                                                             codes=torch.empty((64, 64), dtype=torch.int8, device="cuda")))
+
+
+def _bits(t):
+    return t.view(torch.uint16).cpu().numpy()
+
+
+@pytest.mark.parametrize("M,N,Kc", [(300, 520, 256), (129, 257, 130), (64, 256, 4096), (512, 256, 8192), (1, 1, 1), (520, 96, 384)])
+@pytest.mark.parametrize("raw_sums", [False, True])
+def test_bfloat16_output_is_the_rounded_binary32_result(M, N, Kc, raw_sums):
+    """Whole blocks (TMA stores of 32 x 64 boxes), the element-wise path (raw sums requested), the
+    split contraction's finishing pass and ragged edges: every stored bfloat16 is the oracle's
+    rounding of the oracle's binary32 result, and the pad columns of the buffer stay untouched."""
+    a, b = _codes(M, Kc, 1), _codes(N, Kc, 2)
+    s_row = (torch.rand(M) * 0.02 + 1e-3).cuda()
+    s_col = (torch.rand(N) * 0.02 + 1e-3).cuda()
+    acc_ref = oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy())
+    ref = oracle.to_bf16(oracle.dequant(acc_ref, s_row.cpu().numpy(), s_col.cpu().numpy()))
+    pad = 8 - N % 8 if N % 8 else 0
+    full = torch.full((M, N + pad), 7.0, dtype=torch.bfloat16, device="cuda")
+    out = full[:, :N]
+    acc = torch.empty((M, N), dtype=torch.int32, device="cuda") if raw_sums else None
+    ws = srq.new_workspace(srq.srq_gemm_workspace_bytes(M, N))
+    srq.srq_gemm_i8_ex(a, b, s_row, s_col, out, None, acc, ws)
+    assert srq.srq_poll_status(ws) == 0
+    assert np.array_equal(_bits(out.contiguous()), ref)
+    if pad:
+        assert bool((full[:, N:] == 7.0).all())
+    if raw_sums:
+        assert np.array_equal(acc.cpu().numpy(), acc_ref)
+
+
+def test_bfloat16_output_on_an_unaligned_buffer():
+    M, N, Kc = 70, 45, 64
+    a, b = _codes(M, Kc, 3), _codes(N, Kc, 4)
+    s = torch.tensor([0.01], device="cuda")
+    ref = oracle.to_bf16(oracle.dequant(oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy()), np.float32([0.01]), np.float32([0.01])))
+    flat = torch.zeros(M * N + 1, dtype=torch.bfloat16, device="cuda")
+    out = flat[1:].view(M, N)                      # 2-byte aligned only, odd pitch
+    srq.srq_gemm_i8_ex(a, b, s, s, out)
+    assert np.array_equal(_bits(out.contiguous()), ref)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_layer_passes_with_bfloat16_outputs_and_fused_codes(dtype):
+    """Forward and backward with bfloat16 Y, dA, dW; the codes and the absmax requested next to a
+    bfloat16 output still come from the binary32 result."""
+    T, N, K = 264, 392, 328
+    A, W, dY = synth.layer_inputs(T, N, K, seed=4, dtype=dtype, device="cuda", std_dy=1e-3)
+    f = lambda t: t.float().cpu().numpy()
+    qs = [srq.QSpec(8, srq.PER_ROW, srq.SR, 9, i) for i in range(5)]
+    oq = [oracle.QSpec(8, oracle.PER_ROW, oracle.SR, 9, i) for i in range(5)]
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
+    r_f = oracle.qlinear_fwd(f(A), f(W), oq[0], oq[1])
+    step = torch.tensor([float(np.abs(r_f.out).max()) / 127.0], device="cuda")
+    qn = srq.QSpec(8, srq.PER_TENSOR, srq.SR, 9, 20)
+    codes = torch.empty((T, 400), dtype=torch.int8, device="cuda")[:, :N]
+    m = torch.zeros(1, device="cuda")
+    Y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    srq.qlinear_fwd_ex(A, W, qs[0], qs[1], Y, srq.Output(q=qn, step=step, codes=codes, absmax=m), None, ws)
+    assert srq.srq_poll_status(ws) == 0
+    assert np.array_equal(_bits(Y), oracle.to_bf16(r_f.out))
+    rc, rm = oracle.requantize(r_f.out, float(step.item()), oracle.QSpec(8, 0, oracle.SR, 9, 20))
+    assert np.array_equal(codes.cpu().numpy(), rc) and m.item() == rm
+    dA = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+    srq.qlinear_bwd_ex(dY, A, W, qs[4], qs[2], qs[3], dA, dW, None, None, ws)
+    assert srq.srq_poll_status(ws) == 0
+    assert np.array_equal(_bits(dA), oracle.to_bf16(oracle.qlinear_bwd_input(f(dY), f(W), oq[4], oq[3]).out))
+    assert np.array_equal(_bits(dW), oracle.to_bf16(oracle.qlinear_bwd_weight(f(dY), f(A), oq[4], oq[2]).out))
+
+
+def test_bfloat16_output_cannot_accumulate():
+    a, b = _codes(64, 64, 1), _codes(64, 64, 2)
+    s = torch.tensor([0.01], device="cuda")
+    out = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(srq.SrqError) as e:
+        srq.srq_gemm_i8_ex(a, b, s, s, out, srq.Output(accumulate=True))
+    assert e.value.status == 2
