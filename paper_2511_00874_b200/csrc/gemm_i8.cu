@@ -55,7 +55,6 @@ struct SharedTail {                                    // after the stage ring
     uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain;
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
-    uint32_t epi_abort;
     alignas(16) float s_col[2][BN];   // read as float4
 };
 constexpr int OUT_STAGE_BYTES = 32 * 32 * 4;           // one 32 x 32 block of 32-bit results per epilogue warp
@@ -492,27 +491,56 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t amax = 0u;
         uint32_t lt = 0;
         bool ok = true;
-        for (int64_t u = group; u < units && ok; u += groups, ++lt) {
-            int64_t tile; int32_t kb0_unused, kb1_unused;
+        // Where a unit's tile lies (one division per unit; 32-bit when the tile index allows).
+        auto locate = [&](int64_t u, int64_t& tile, int32_t& tn, int32_t& tm) {
+            int32_t kb0_unused, kb1_unused;
             decode(u, tile, kb0_unused, kb1_unused);
+            if (tile < (1ll << 32)) {
+                tm = (int32_t)((uint32_t)tile / (uint32_t)P.tiles_n);
+                tn = (int32_t)((uint32_t)tile - (uint32_t)tm * (uint32_t)P.tiles_n);
+            } else {
+                tm = (int32_t)(tile / P.tiles_n);
+                tn = (int32_t)(tile % P.tiles_n);
+            }
+        };
+        // Step sizes of a unit's tile: this thread's row and two of the 256 columns (etid, etid + 128).
+        // They are fetched one unit ahead, so that their latency falls into the previous tile's work.
+        float sc_next[2] = {0.0f, 0.0f}, sr_next = 0.0f;
+        int64_t tile_next = 0; int32_t tn_next = 0, tm_next = 0;
+        auto fetch_steps = [&](int64_t u) {
+            locate(u, tile_next, tn_next, tm_next);
+            const int64_t col_base = (int64_t)tn_next * BN;
+            const int64_t row = ((int64_t)tm_next * CTAS + rank) * BM + quarter * 32 + lane;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int64_t c = col_base + etid + 128 * h;
+                sc_next[h] = (c < P.N) ? __ldg(P.s_col + c * P.col_stride) : 0.0f;
+            }
+            sr_next = (row < P.M) ? __ldg(P.s_row + row * P.row_stride) : 0.0f;
+        };
+        if (group < units) fetch_steps(group);
+        for (int64_t u = group; u < units && ok; u += groups, ++lt) {
+            const int64_t tile = tile_next;
+            const int32_t tn = tn_next, tm = tm_next;
             const bool whole = u < P.full_tiles;              // this unit holds the complete sums of its tile
-            const int32_t tn = (int32_t)(tile % P.tiles_n), tm = (int32_t)(tile / P.tiles_n);
             const uint32_t buf = lt & 1u, use = lt >> 1;
             const int64_t row0 = ((int64_t)tm * CTAS + rank) * BM;      // first row of this CTA's half
             const int64_t row = row0 + quarter * 32 + lane;
             const int64_t col_base = (int64_t)tn * BN;
-            // stage this tile's column step sizes (other buffer may still be read by slower warps)
-            for (int i = etid; i < BN; i += 128) {
-                const int64_t c = col_base + i;
-                T->s_col[buf][i] = (c < P.N) ? P.s_col[c * P.col_stride] : 0.0f;
-            }
-            const float sr = (row < P.M) ? P.s_row[row * P.row_stride] : 0.0f;
-            if (!mbar_wait(&T->tmem_full[buf], use & 1u, &T->abort_flag)) give_up(T, P.status);
-            // the four warps must leave together (they share named barrier 1): agree on one flag
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (etid == 0) T->epi_abort = T->abort_flag;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (T->epi_abort) { ok = false; break; }
+            // stage this tile's column step sizes (the other buffer may still be read by slower warps;
+            // this one was last read two tiles ago, which every warp has left)
+            T->s_col[buf][etid] = sc_next[0];
+            T->s_col[buf][etid + 128] = sc_next[1];
+            const float sr = sr_next;
+            if (u + groups < units) fetch_steps(u + groups);
+            bool mine = mbar_wait(&T->tmem_full[buf], use & 1u, &T->abort_flag);
+            if (!mine) give_up(T, P.status);
+            // the four warps must leave together (they share named barrier 1): one barrier makes the
+            // staged step sizes visible and tells every thread whether any of them gave up
+            uint32_t any_gave_up;
+            asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.or.pred p, 1, 128, q;\nselp.u32 %0, 1, 0, p;\n}"
+                         : "=r"(any_gave_up) : "r"((uint32_t)(!mine || T->abort_flag != 0u)) : "memory");
+            if (any_gave_up) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
             const uint32_t stage = smem_u32(out_stage + (warp - 2) * OUT_STAGE_BYTES);
