@@ -113,26 +113,33 @@ def oracle_layer_seconds(T, N, K, seed=0):
 
 
 def pick_oracle_sample(target_s):
-    """Token count of the slice the oracle can do in about target_s seconds on this host."""
-    # two probes separate the part that does not grow with the tokens (quantizing W) from the rest
-    t1 = oracle_layer_seconds(64, N_FULL, K_FULL)
-    t2 = oracle_layer_seconds(256, N_FULL, K_FULL)
+    """(tokens, output features) of the slice of the layer the oracle can do in about target_s
+    seconds on this host: as many tokens as fit; output features are cut only when even 256 tokens
+    with the whole W (whose quantization does not shrink with the tokens) take longer."""
+    Ns = N_FULL
+    while True:
+        # two probes separate the part that does not grow with the tokens (quantizing W) from the rest
+        t1 = oracle_layer_seconds(64, Ns, K_FULL)
+        t2 = oracle_layer_seconds(256, Ns, K_FULL)
+        if t2 <= target_s or Ns <= 256:
+            break
+        Ns //= 2
     per_token = max((t2 - t1) / 192.0, 1e-9)
     fixed = max(t1 - 64 * per_token, 0.0)
     Ts = 256
     while Ts * 2 <= T_FULL and fixed + per_token * Ts * 2 <= target_s:
         Ts *= 2
-    return Ts
+    return Ts, Ns
 
 
 def cpu_baseline(target_s=15.0):
     import oracle
-    Ts = pick_oracle_sample(target_s)
-    sec = oracle_layer_seconds(Ts, N_FULL, K_FULL)
-    return {"value": layer_ops(Ts, N_FULL, K_FULL) / sec / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
+    Ts, Ns = pick_oracle_sample(target_s)
+    sec = oracle_layer_seconds(Ts, Ns, K_FULL)
+    return {"value": layer_ops(Ts, Ns, K_FULL) / sec / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
             "kind": "oracle", "seconds": sec,
-            "sample": f"same layer (4096->4096, fp32, 8-bit per-tensor SR), first {Ts} of 65536 tokens, "
-                      f"fwd + bwd_input + bwd_weight, ops counted as 6*T*N*K"}
+            "sample": f"same layer (4096->{Ns} of 4096 output features, fp32, 8-bit per-tensor SR), first {Ts} of "
+                      f"65536 tokens, fwd + bwd_input + bwd_weight, ops counted as 6*T*N*K"}
 
 
 def run_reference(args):
@@ -141,22 +148,22 @@ def run_reference(args):
         return
     import oracle
     oracle.build()
-    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
-    Ts = pick_oracle_sample(per_step)
+    per_step = max(0.5, min(20.0, 150.0 / max(1, args.steps + args.warmup)))   # the whole run stays within minutes
+    Ts, Ns = pick_oracle_sample(per_step)
     for _ in range(args.warmup):
-        oracle_layer_seconds(Ts, N_FULL, K_FULL)
+        oracle_layer_seconds(Ts, Ns, K_FULL)
     t0 = time.perf_counter()
     for s in range(args.steps):
-        oracle_layer_seconds(Ts, N_FULL, K_FULL, seed=s)
+        oracle_layer_seconds(Ts, Ns, K_FULL, seed=s)
     sec = (time.perf_counter() - t0) / max(1, args.steps)
-    val = layer_ops(Ts, N_FULL, K_FULL) / sec / 1e12
+    val = layer_ops(Ts, Ns, K_FULL) / sec / 1e12
     sample = (f"CPU oracle on {oracle.num_threads()} host threads; each step = fwd + bwd of the first {Ts} of "
-              f"65536 tokens of the same layer (input generation included)")
+              f"65536 tokens and the first {Ns} of 4096 output features of the same layer (input generation included)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample_tokens": Ts},
+        "config": {"workload": WORKLOAD, "sample_tokens": Ts, "sample_out_features": Ns},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
