@@ -48,6 +48,35 @@ def test_product_and_dequant_match_the_oracle(M, N, Kc, per_row):
     assert np.array_equal(out2, ref_out)
 
 
+def test_longest_contraction_with_extreme_codes_fills_int32_without_overflow():
+    """Kc = 133136 is the longest 16-aligned contraction the int32 rule admits at 8 bits
+    (133136 * 127^2 = 2147350544 < 2^31).  With every code at +-127 each sum is +-that number, on
+    the unsplit path (raw sums requested) and on the split path, whose partial sums are added in
+    memory: no intermediate may wrap."""
+    Kc, M, N = 133136, 130, 260
+    top = Kc * 127 * 127
+    assert top < 2 ** 31 <= (Kc + 16) * 127 * 127
+    sign_a = torch.where(torch.arange(M) % 3 == 0, -1, 1).to(torch.int8)
+    sign_b = torch.where(torch.arange(N) % 5 == 0, -1, 1).to(torch.int8)
+    a = (sign_a[:, None] * torch.full((M, Kc), 127, dtype=torch.int8)).cuda()
+    b = (sign_b[:, None] * torch.full((N, Kc), 127, dtype=torch.int8)).cuda()
+    want = (sign_a[:, None].int() * sign_b[None, :].int()).numpy().astype(np.int64) * top
+    s_row = torch.full((M,), 2.0 ** -20, device="cuda")
+    s_col = torch.full((1,), 3.0, device="cuda")
+    ref_out = oracle.dequant(want.astype(np.int32), s_row.cpu().numpy(), s_col.cpu().numpy())
+    for want_acc in (True, False):
+        out, acc = _run(a, b, s_row, s_col, want_acc=want_acc)
+        if want_acc:
+            assert np.array_equal(acc.astype(np.int64), want)
+        assert np.array_equal(out, ref_out)
+    # one more 16-byte step of the contraction is refused before anything is launched
+    a2 = torch.zeros((M, Kc + 16), dtype=torch.int8, device="cuda")
+    b2 = torch.zeros((N, Kc + 16), dtype=torch.int8, device="cuda")
+    with pytest.raises(srq.SrqError) as e:
+        srq.srq_gemm_i8(a2, b2, s_row, s_col, torch.empty((M, N), device="cuda"))
+    assert e.value.status == 4
+
+
 def test_special_code_matrices():
     # all ones: every sum equals the contraction length; identity: returns the other operand
     Kc = 400
