@@ -584,6 +584,134 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
     else quantize_tile<T, MODE, LAYOUT, PER_ROW, false, false>(x, P, tileT, r0, c0);
 }
 
+// Per-row step sizes, row-major codes only: absmax and quantizer in ONE pass over the input.  A CTA
+// takes whole rows; each thread holds its 4-element groups of the row in registers (G per thread,
+// groups tid, tid + 256, ...), the row maximum is reduced over the CTA (two barriers per row), the
+// step size is derived exactly as in the two-pass path, and the codes are formed from the registers,
+// so that the input is read once (e + 1 bytes per element instead of 2 e + 1).  The next row's loads
+// are issued before the current row is processed.  Same conditions as the fast path (groups of four
+// line up with the flat index), same arithmetic, same codes.
+__device__ __forceinline__ uint32_t abs_max4(const float4& q) {
+    return max(max(__float_as_uint(q.x) & 0x7FFFFFFFu, __float_as_uint(q.y) & 0x7FFFFFFFu),
+               max(__float_as_uint(q.z) & 0x7FFFFFFFu, __float_as_uint(q.w) & 0x7FFFFFFFu));
+}
+__device__ __forceinline__ uint32_t abs_max4(const uint2& q) {      // four bfloat16: packed 16-bit maxima, widened
+    const uint32_t m = __vmaxu2(q.x & 0x7FFF7FFFu, q.y & 0x7FFF7FFFu);
+    return max(m << 16, m & 0xFFFF0000u);
+}
+
+constexpr int ROWQ_MAX_G = 8;          // rows of up to 256 * 8 * 4 = 8192 elements
+
+template <typename T, int MODE, int G>
+__global__ void __launch_bounds__(Q_THREADS)
+quantize_rows_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P, float* __restrict__ delta_out,
+                     float qmax, uint32_t* status) {
+    using Raw = typename Raw4<T>::type;
+    constexpr bool SRM = (MODE & MODE_SR) != 0;
+    __shared__ uint32_t warp_max[2][Q_THREADS / 32];
+    __shared__ float row_inv[2];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t ngroups = (uint32_t)(P.cols >> 2);
+    Raw cur[G], nxt[G];
+    auto load_row = [&](int64_t r, Raw raw[G]) {
+        const Raw* src = reinterpret_cast<const Raw*>(x + r * P.ld);
+#pragma unroll
+        for (int k = 0; k < G; ++k) {
+            const uint32_t g = (uint32_t)tid + (uint32_t)(k * Q_THREADS);
+            raw[k] = g < ngroups ? __ldcs(src + g) : Raw{};
+        }
+    };
+    int64_t r = blockIdx.x;
+    if (r < P.rows) load_row(r, cur);
+    for (uint32_t it = 0; r < P.rows; r += gridDim.x, ++it) {
+        if (r + gridDim.x < P.rows) load_row(r + gridDim.x, nxt);
+        uint32_t m = 0u;
+#pragma unroll
+        for (int k = 0; k < G; ++k) m = max(m, abs_max4(cur[k]));
+        m = __reduce_max_sync(0xFFFFFFFFu, m);
+        if (lane == 0) warp_max[it & 1][warp] = m;
+        __syncthreads();
+        // one warp turns the row maximum into the step size (three divisions, done once per row instead
+        // of once per warp); both shared slots alternate between rows, and the two barriers of the
+        // following row separate every write from the last read of the same slot
+        if (warp == 0) {
+            uint32_t bits = lane < Q_THREADS / 32 ? warp_max[it & 1][lane] : 0u;
+            bits = __reduce_max_sync(0xFFFFFFFFu, bits);
+            if (lane == 0) {
+                float delta, r_inv;
+                scale_from_bits(bits, qmax, &delta, &r_inv, status);
+                row_inv[it & 1] = r_inv;
+                if (delta_out) delta_out[r] = delta;
+            }
+        }
+        __syncthreads();
+        const float inv = row_inv[it & 1];
+        const uint64_t jb = (P.index_offset + (uint64_t)r * (uint64_t)P.cols) >> 2;     // block of the row's first group
+        uint32_t* out = reinterpret_cast<uint32_t*>(P.codes_rm + r * P.ld_rm);
+        // all G groups are computed without branches (groups past the row hold zeros), so that their
+        // Philox chains interleave; only the stores are predicated
+        uint32_t w[G];
+#pragma unroll
+        for (int k = 0; k < G; ++k) {
+            const uint32_t g = (uint32_t)tid + (uint32_t)(k * Q_THREADS);
+            float v[4];
+            widen(cur[k], v);
+            uint32_t rnd[4] = {0u, 0u, 0u, 0u};
+            if constexpr (SRM) {
+                const uint32_t lo = (uint32_t)jb + g;
+                philox_rounds(lo, (uint32_t)(jb >> 32) + (lo < g ? 1u : 0u), P.keys, rnd);
+            }
+            w[k] = quantize4<MODE>(v, inv, inv, inv, inv, rnd);
+        }
+#pragma unroll
+        for (int k = 0; k < G; ++k) {
+            const uint32_t g = (uint32_t)tid + (uint32_t)(k * Q_THREADS);
+            if (g < ngroups) out[g] = w[k];
+        }
+#pragma unroll
+        for (int k = 0; k < G; ++k) cur[k] = nxt[k];
+    }
+}
+
+// One wave of CTAs: as many as are resident at once (asked once per kernel), at most one per row.
+template <typename T, int MODE, int G>
+static void launch_rows_one(const T* p, const QuantParams& P, float* delta_out, float qmax, uint32_t* status,
+                            int sms, cudaStream_t st) {
+    static int per_sm = 0;
+    if (per_sm == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_rows_kernel<T, MODE, G>, Q_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+        per_sm = n;
+    }
+    const int64_t resident = (int64_t)sms * per_sm;
+    const unsigned grid = (unsigned)(P.rows < resident ? P.rows : resident);
+    quantize_rows_kernel<T, MODE, G><<<grid, Q_THREADS, 0, st>>>(p, P, delta_out, qmax, status);
+}
+
+template <typename T, int MODE>
+static void launch_rows_g(int g, const void* x, const QuantParams& P, float* delta_out, float qmax, uint32_t* status,
+                          int sms, cudaStream_t st) {
+    const T* p = (const T*)x;
+    if (g <= 1) launch_rows_one<T, MODE, 1>(p, P, delta_out, qmax, status, sms, st);
+    else if (g <= 2) launch_rows_one<T, MODE, 2>(p, P, delta_out, qmax, status, sms, st);
+    else if (g <= 4) launch_rows_one<T, MODE, 4>(p, P, delta_out, qmax, status, sms, st);
+    else launch_rows_one<T, MODE, 8>(p, P, delta_out, qmax, status, sms, st);
+}
+
+static void launch_rows(srq_dtype_t dt, int mode, const void* x, const QuantParams& P, float* delta_out, float qmax,
+                        uint32_t* status, int sms, cudaStream_t st) {
+    const int g = (int)(((P.cols >> 2) + Q_THREADS - 1) / Q_THREADS);
+#define SRQ_ROWS(T)                                                                          \
+    switch (mode) {                                                                          \
+        case 0: launch_rows_g<T, 0>(g, x, P, delta_out, qmax, status, sms, st);  break;      \
+        case 1: launch_rows_g<T, 1>(g, x, P, delta_out, qmax, status, sms, st);  break;      \
+        case 2: launch_rows_g<T, 2>(g, x, P, delta_out, qmax, status, sms, st);  break;      \
+        default: launch_rows_g<T, 3>(g, x, P, delta_out, qmax, status, sms, st);  break;     \
+    }
+    if (dt == SRQ_F32) { SRQ_ROWS(float) } else { SRQ_ROWS(__nv_bfloat16) }
+#undef SRQ_ROWS
+}
+
 // General path: any extent, pitch, alignment and index offset; one Philox block per element
 // when the groups of four do not line up with the flat index.  Same results as the fast path.
 template <typename T>
@@ -725,6 +853,18 @@ cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t c
     return cudaGetLastError();
 }
 
+// SM count of the current device (asked once per device).
+static int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        cached[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+    }
+    return cached[dev];
+}
+
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream, bool scratch_zeroed) {
     const bool want_rm = a.codes_rm != nullptr, want_tr = a.codes_tr != nullptr;
     const bool per_row = a.q.scale == SRQ_PER_ROW;
@@ -747,6 +887,32 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     // per tensor: one group feeds both layouts' scale outputs
     const int64_t n0 = per_row ? n_rm : 1;
     const int64_t n1 = per_row ? n_tr : ((want_tr && a.scale_tr) ? 1 : 0);
+
+    QuantParams P;
+    P.rows = rows; P.cols = cols; P.ld = a.ld;
+    P.index_offset = a.q.index_offset;
+    P.keys = make_philox_keys(a.q.seed, a.q.tensor_id);
+    P.sr = a.q.round == SRQ_SR;
+    const bool sr8 = a.q.round == SRQ_SR8;
+    P.mode = sr8 ? MODE_SR8 : ((P.sr ? MODE_SR : 0) | (e4m3 ? MODE_E4M3 : 0));
+    P.per_row = per_row;
+    P.codes_rm = a.codes_rm; P.ld_rm = a.ld_rm;
+    P.codes_tr = a.codes_tr; P.ld_tr = a.ld_tr;
+    P.inv_rm = inv_rm; P.inv_tr = inv_tr;
+    P.vec_in = vec_in;
+    P.vec_rm = want_rm && ((uintptr_t)a.codes_rm % 4 == 0) && (a.ld_rm % 4 == 0);
+    P.vec_tr = want_tr && ((uintptr_t)a.codes_tr % 4 == 0) && (a.ld_tr % 4 == 0);
+    P.vec_tr16 = want_tr && ((uintptr_t)a.codes_tr % 16 == 0) && (a.ld_tr % 16 == 0);
+    const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && (!sr8 || (cols % 16 == 0 && a.q.index_offset % 16 == 0)) && a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) &&
+                      (!want_tr || (P.vec_tr && rows % 4 == 0));
+
+    // per-row steps and row-major codes only: one pass (rows of 512 .. 8192 elements)
+    if (per_row && want_rm && !want_tr && fast && !sr8 && cols >= 512 && cols <= (int64_t)ROWQ_MAX_G * Q_THREADS * 4) {
+        launch_rows(a.dt, P.mode, a.x, P, a.scale_rm, qmax, status, sm_count(), stream);
+        ++g_launches;
+        return cudaGetLastError();
+    }
+
     if (given) {
         amax_rm = amax_tr = (uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
         const int64_t n = n0 > n1 ? n0 : n1;
@@ -760,32 +926,25 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
             cudaError_t e = cudaMemsetAsync(s.counter, 0, (size_t)((char*)s.inv_rm - (char*)s.counter), stream);
             if (e != cudaSuccess) return e;
         }
-        // absmax of every group; the last CTA to finish turns them into step sizes
-        const ScaleStep S = {s.counter, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
+        // absmax of every group; the last CTA to finish turns them into step sizes when there are few
+        // (one CTA would take long over many thousands of groups: those get a launch of their own)
+        const bool few = n0 + n1 <= 2048;
+        const ScaleStep S = {few ? s.counter : nullptr, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
                              n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status};
         const bool want_rows = per_row && want_rm, want_cols = per_row && want_tr;
         if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, S, stream);
         else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, S, stream);
         ++g_launches;
+        if (!few) {
+            const int64_t n = n0 > n1 ? n0 : n1;
+            const int threads = 256;
+            scales_kernel<<<(unsigned)((n + threads - 1) / threads), threads, 0, stream>>>(
+                amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
+                amax_tr, n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status);
+            ++g_launches;
+        }
     }
     {
-        QuantParams P;
-        P.rows = rows; P.cols = cols; P.ld = a.ld;
-        P.index_offset = a.q.index_offset;
-        P.keys = make_philox_keys(a.q.seed, a.q.tensor_id);
-        P.sr = a.q.round == SRQ_SR;
-        const bool sr8 = a.q.round == SRQ_SR8;
-        P.mode = sr8 ? MODE_SR8 : ((P.sr ? MODE_SR : 0) | (e4m3 ? MODE_E4M3 : 0));
-        P.per_row = per_row;
-        P.codes_rm = a.codes_rm; P.ld_rm = a.ld_rm;
-        P.codes_tr = a.codes_tr; P.ld_tr = a.ld_tr;
-        P.inv_rm = inv_rm; P.inv_tr = inv_tr;
-        P.vec_in = vec_in;
-        P.vec_rm = want_rm && ((uintptr_t)a.codes_rm % 4 == 0) && (a.ld_rm % 4 == 0);
-        P.vec_tr = want_tr && ((uintptr_t)a.codes_tr % 4 == 0) && (a.ld_tr % 4 == 0);
-        P.vec_tr16 = want_tr && ((uintptr_t)a.codes_tr % 16 == 0) && (a.ld_tr % 16 == 0);
-        const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && (!sr8 || (cols % 16 == 0 && a.q.index_offset % 16 == 0)) && a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) &&
-                          (!want_tr || (P.vec_tr && rows % 4 == 0));
         const unsigned grid = (unsigned)(((cols + Q_TILE - 1) / Q_TILE) * ((rows + Q_TILE - 1) / Q_TILE));
         if (fast) launch_fast(a.dt, P.mode, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);
         else if (a.dt == SRQ_F32) quantize_kernel<float><<<grid, Q_THREADS, 0, stream>>>((const float*)a.x, P);

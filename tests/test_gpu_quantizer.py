@@ -201,3 +201,23 @@ def test_eight_random_bits_per_element(dtype, scale):
     with pytest.raises(srq.SrqError):                                    # integer grid only
         srq.sr_quantize(x, srq.QSpec(8, scale, srq.SR8, format=srq.GRID_E4M3),
                         torch.empty((300, 400), dtype=torch.int8, device="cuda"), torch.empty(300, device="cuda"))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("shape,off", [((70, 512), 0), ((33, 4096), 4), ((5, 8192), 2 ** 34), ((130, 2052), 8),
+                                       ((2000, 516), 0), ((3, 8196), 0)])
+def test_one_pass_per_row_path_matches_the_oracle(dtype, shape, off):
+    """Per-row steps with row-major codes only: rows of 512 .. 8192 elements take the kernel that
+    reads the input once (row maximum and codes from the same registers); more rows than resident
+    CTAs, partly filled groups per thread, a zero row, a row too small to scale, padded code
+    pitch.  The 8196-column case is past its limit and takes the two-pass path: same codes."""
+    x = synth.with_outliers(shape, seed=shape[1], dtype=dtype, device="cuda")
+    x[0] = 0
+    x[shape[0] - 1] = 1e-39 if dtype == torch.float32 else 0.0
+    for bits, rnd in ((8, srq.SR), (4, srq.SR), (6, srq.RTN)):
+        _check(x, bits, srq.PER_ROW, rnd, seed=11, tid=2 ** 33 + 5, off=off, want_rm=True, want_tr=False, pad_rm=12)
+    # the same rows through the two-pass kernels (both layouts requested) give the same row-major codes
+    q = srq.QSpec(8, srq.PER_ROW, srq.SR, 11, 3, off)
+    one = _run_gpu(x, q, True, False)
+    two = _run_gpu(x, q, True, True)
+    assert np.array_equal(one[0], two[0]) and np.array_equal(one[1], two[1])
