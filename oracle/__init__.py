@@ -104,6 +104,15 @@ def lib() -> ctypes.CDLL:
         L.orc_sr_quantize_e4m3.argtypes = [vp, i64, i64, i64, ctypes.c_int, ctypes.c_int,
                                            ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
         L.orc_sr_quantize_e4m3.restype = ctypes.c_int
+        L.orc_e4m_max.argtypes = [ctypes.c_int]
+        L.orc_e4m_max.restype = ctypes.c_double
+        L.orc_quantize_e4m_scalar.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_uint32]
+        L.orc_quantize_e4m_scalar.restype = ctypes.c_uint8
+        L.orc_scale_e4m.argtypes = [ctypes.c_float, ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+        L.orc_scale_e4m.restype = None
+        L.orc_sr_quantize_e4m.argtypes = [vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                          ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
+        L.orc_sr_quantize_e4m.restype = ctypes.c_int
         L.orc_gemm_e4m3_nt.argtypes = [vp, vp, i64, i64, i64, vp, ctypes.c_int, vp, ctypes.c_int, vp, vp]
         L.orc_gemm_e4m3_nt.restype = None
         L.orc_requantize.argtypes = [vp, i64, i64, ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_uint64,
@@ -295,8 +304,26 @@ def quantize_e4m3_scalar(x: float, inv: float, round_mode: int, u24: int = 0) ->
     return int(lib().orc_quantize_e4m3_scalar(ctypes.c_float(x), ctypes.c_float(inv), round_mode, u24))
 
 
+def e4m_max(mant: int) -> float:
+    """Largest value of the E4Mk grid (k = mant mantissa bits)."""
+    return float(lib().orc_e4m_max(mant))
+
+
+def scale_e4m(m: float, mant: int):
+    d, inv = ctypes.c_float(), ctypes.c_float()
+    lib().orc_scale_e4m(ctypes.c_float(m), mant, ctypes.byref(d), ctypes.byref(inv))
+    return np.float32(d.value), np.float32(inv.value)
+
+
+def quantize_e4m_scalar(x: float, inv: float, mant: int, round_mode: int, u24: int = 0) -> int:
+    return int(lib().orc_quantize_e4m_scalar(ctypes.c_float(x), ctypes.c_float(inv), mant, round_mode, u24))
+
+
 def sr_quantize_e4m3(x, q: QSpec, want_rm: bool = True, want_tr: bool = False):
-    """Def. 1-3 on the E4M3 grid (q.bits is ignored); returns (codes_rm, scale_rm, codes_tr, scale_tr)."""
+    """Def. 1-3 on the E4Mk grid, k = q.bits - 5 mantissa bits (8: E4M3, 7: E4M2, 6: E4M1, 5: E4M0);
+    codes are E4M3 bytes; returns (codes_rm, scale_rm, codes_tr, scale_tr)."""
+    mant = q.bits - 5
+    assert 0 <= mant <= 3
     x = _f32_2d(x)
     rows, cols = x.shape
     ld = x.strides[0] // 4
@@ -308,8 +335,8 @@ def sr_quantize_e4m3(x, q: QSpec, want_rm: bool = True, want_tr: bool = False):
     if want_tr:
         ctr = np.zeros((cols, rows), dtype=np.uint8)
         strr = np.zeros(cols if per_row else 1, dtype=np.float32)
-    lib().orc_sr_quantize_e4m3(_ptr(x), rows, cols, ld, q.scale_mode, q.round_mode, q.seed, q.tensor_id,
-                               q.index_offset, _ptr(crm), _ptr(srm), _ptr(ctr), _ptr(strr))
+    lib().orc_sr_quantize_e4m(_ptr(x), rows, cols, ld, mant, q.scale_mode, q.round_mode, q.seed, q.tensor_id,
+                              q.index_offset, _ptr(crm), _ptr(srm), _ptr(ctr), _ptr(strr))
     return crm, srm, ctr, strr
 
 

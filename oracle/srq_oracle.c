@@ -490,18 +490,31 @@ static uint8_t orc_e4m3_encode_on_grid(double v)
 }
 
 /*
- * Def. 1 on the E4M3 grid.  The grid is uniform inside each binade, so the
+ * The narrower members E4M2, E4M1, E4M0 (the formats of the paper's experiments section, which
+ * names them without defining them).  Reading used here: E4Mk keeps the sign, the four exponent
+ * bits and the bias of E4M3 and has k mantissa bits, i.e. its values are the E4M3 values whose
+ * low 3 - k mantissa bits are zero: inside binade e the spacing is 2^(e-k), the subnormal
+ * spacing (below 2^-6) is 2^(-6-k), and the largest finite value is the largest such E4M3
+ * value: 448 for k = 3 and 2 (1.75 2^8), 384 for k = 1 (1.5 2^8), 256 for k = 0 (2^8).
+ * Codes are stored as E4M3 bytes, so that one product routine serves all four.
+ */
+double orc_e4m_max(int mant)
+{
+    return mant >= 2 ? 448.0 : (mant == 1 ? 384.0 : 256.0);
+}
+
+/*
+ * Def. 1 on the E4Mk grid.  The grid is uniform inside each binade, so the
  * precision level of Def. 1 is taken locally: for t = x * inv with
  * 2^e <= |t| < 2^(e+1) (e clamped to [-6, 8]; below 2^-6 the subnormal spacing
- * continues) the step is D = 2^(e-3), and Q_D(t, eps) = D floor(t/D) if
- * frac(t/D) < eps... i.e. exactly the rule of orc_quantize_scalar applied to
- * u = t / D: round up (toward +infinity) iff eps < frac(u) for SR, iff
- * frac(u) >= 1/2 for RTN.  Both neighbours D floor(u) and D (floor(u) + 1) are
- * E4M3 values (a binade's upper end is the next binade's first value).
- * Scaling by D is exact, and the comparison is evaluated in binary64 where
- * every term is exact.  Returns the code byte.
+ * continues) the step is D = 2^(e-k), and Q_D(t, eps) is exactly the rule of
+ * orc_quantize_scalar applied to u = t / D: round up (toward +infinity) iff
+ * eps < frac(u) for SR, iff frac(u) >= 1/2 for RTN.  Both neighbours D floor(u)
+ * and D (floor(u) + 1) are grid values (a binade's upper end is the next
+ * binade's first value).  Scaling by D is exact, and the comparison is
+ * evaluated in binary64 where every term is exact.  Returns the E4M3 code byte.
  */
-uint8_t orc_quantize_e4m3_scalar(float x, float inv, int round_mode, uint32_t u24)
+uint8_t orc_quantize_e4m_scalar(float x, float inv, int mant, int round_mode, uint32_t u24)
 {
     float t = x * inv;
     double td = (double)t, a = fabs(td);
@@ -511,29 +524,41 @@ uint8_t orc_quantize_e4m3_scalar(float x, float inv, int round_mode, uint32_t u2
     int e = ex2 - 1;
     if (e < -6) e = -6;
     if (e > 8) e = 8;
-    double u = ldexp(td, 3 - e);                 /* t / D, exact */
+    double u = ldexp(td, mant - e);              /* t / D, exact */
     double f = floor(u);
     int up;
     if (round_mode == ORC_SR || round_mode == ORC_SR8)
         up = ((double)u24 + f * 0x1p24) < u * 0x1p24;
     else
         up = (f * 0x1p24 + 0x1p23) <= u * 0x1p24;
-    double v = ldexp(f + up, e - 3);
-    if (v > 448.0) v = 448.0;                    /* unreachable with inv from orc_scale_e4m3 */
-    if (v < -448.0) v = -448.0;
+    double v = ldexp(f + up, e - mant);
+    double top = orc_e4m_max(mant);
+    if (v > top) v = top;                        /* unreachable with inv from orc_scale_e4m */
+    if (v < -top) v = -top;
     return orc_e4m3_encode_on_grid(v);
 }
 
-/* Step size D = m / 448 (round to nearest) and the reciprocal multiplied in,
- * 448 / m rounded toward zero, so that |x * inv| <= 448 for the whole group
+uint8_t orc_quantize_e4m3_scalar(float x, float inv, int round_mode, uint32_t u24)
+{
+    return orc_quantize_e4m_scalar(x, inv, 3, round_mode, u24);
+}
+
+/* Step size D = m / top (round to nearest), top the largest value of the grid, and the reciprocal
+ * multiplied in, top / m rounded toward zero, so that |x * inv| <= top for the whole group
  * (same reasoning as orc_scale_from_absmax). */
+void orc_scale_e4m(float m, int mant, float *delta, float *inv)
+{
+    float top = (float)orc_e4m_max(mant);
+    float r = (m == 0.0f) ? 0.0f : top / m;
+    if (isinf(r) || r != r) r = 0.0f;
+    if (r != 0.0f && (double)r * (double)m > (double)top) r = nextafterf(r, 0.0f);
+    *inv = r;
+    *delta = (r == 0.0f) ? 0.0f : m / top;
+}
+
 void orc_scale_e4m3(float m, float *delta, float *inv)
 {
-    float r = (m == 0.0f) ? 0.0f : 448.0f / m;
-    if (isinf(r) || r != r) r = 0.0f;
-    if (r != 0.0f && (double)r * (double)m > 448.0) r = nextafterf(r, 0.0f);
-    *inv = r;
-    *delta = (r == 0.0f) ? 0.0f : m / 448.0f;
+    orc_scale_e4m(m, 3, delta, inv);
 }
 
 /*
@@ -541,11 +566,11 @@ void orc_scale_e4m3(float m, float *delta, float *inv)
  * or per-row step sizes, one threshold per element by flat source index);
  * codes are E4M3 bytes.
  */
-int orc_sr_quantize_e4m3(const float *x, int64_t rows, int64_t cols, int64_t ld,
-                         int scale_mode, int round_mode,
-                         uint64_t seed, uint64_t tensor_id, uint64_t index_offset,
-                         uint8_t *codes_rm, float *scale_rm,
-                         uint8_t *codes_tr, float *scale_tr)
+int orc_sr_quantize_e4m(const float *x, int64_t rows, int64_t cols, int64_t ld,
+                        int mant, int scale_mode, int round_mode,
+                        uint64_t seed, uint64_t tensor_id, uint64_t index_offset,
+                        uint8_t *codes_rm, float *scale_rm,
+                        uint8_t *codes_tr, float *scale_tr)
 {
     float m_tensor = 0.0f;
     if (scale_mode == ORC_PER_TENSOR) orc_absmax_tensor(x, rows, cols, ld, &m_tensor);
@@ -554,33 +579,43 @@ int orc_sr_quantize_e4m3(const float *x, int64_t rows, int64_t cols, int64_t ld,
 #pragma omp parallel for schedule(static)
         for (int64_t r = 0; r < rows; ++r) {
             float delta, inv;
-            orc_scale_e4m3(scale_mode == ORC_PER_TENSOR ? m_tensor : scale_rm[r], &delta, &inv);
+            orc_scale_e4m(scale_mode == ORC_PER_TENSOR ? m_tensor : scale_rm[r], mant, &delta, &inv);
             if (scale_mode == ORC_PER_ROW) scale_rm[r] = delta;
             else if (r == 0) scale_rm[0] = delta;
             for (int64_t c = 0; c < cols; ++c) {
                 uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
                 uint32_t u24 = orc_threshold(round_mode, seed, tensor_id, i);
-                codes_rm[r * cols + c] = orc_quantize_e4m3_scalar(x[r * ld + c], inv, round_mode, u24);
+                codes_rm[r * cols + c] = orc_quantize_e4m_scalar(x[r * ld + c], inv, mant, round_mode, u24);
             }
         }
-        if (scale_mode == ORC_PER_TENSOR && rows == 0) { float d, iv; orc_scale_e4m3(m_tensor, &d, &iv); scale_rm[0] = d; }
+        if (scale_mode == ORC_PER_TENSOR && rows == 0) { float d, iv; orc_scale_e4m(m_tensor, mant, &d, &iv); scale_rm[0] = d; }
     }
     if (codes_tr) {
         if (scale_mode == ORC_PER_ROW) orc_absmax_cols(x, rows, cols, ld, scale_tr);
 #pragma omp parallel for schedule(static)
         for (int64_t c = 0; c < cols; ++c) {
             float delta, inv;
-            orc_scale_e4m3(scale_mode == ORC_PER_TENSOR ? m_tensor : scale_tr[c], &delta, &inv);
+            orc_scale_e4m(scale_mode == ORC_PER_TENSOR ? m_tensor : scale_tr[c], mant, &delta, &inv);
             if (scale_mode == ORC_PER_ROW) scale_tr[c] = delta;
             else if (c == 0) scale_tr[0] = delta;
             for (int64_t r = 0; r < rows; ++r) {
                 uint64_t i = index_offset + (uint64_t)r * (uint64_t)cols + (uint64_t)c;
                 uint32_t u24 = orc_threshold(round_mode, seed, tensor_id, i);
-                codes_tr[c * rows + r] = orc_quantize_e4m3_scalar(x[r * ld + c], inv, round_mode, u24);
+                codes_tr[c * rows + r] = orc_quantize_e4m_scalar(x[r * ld + c], inv, mant, round_mode, u24);
             }
         }
     }
     return 0;
+}
+
+int orc_sr_quantize_e4m3(const float *x, int64_t rows, int64_t cols, int64_t ld,
+                         int scale_mode, int round_mode,
+                         uint64_t seed, uint64_t tensor_id, uint64_t index_offset,
+                         uint8_t *codes_rm, float *scale_rm,
+                         uint8_t *codes_tr, float *scale_tr)
+{
+    return orc_sr_quantize_e4m(x, rows, cols, ld, 3, scale_mode, round_mode, seed, tensor_id, index_offset,
+                               codes_rm, scale_rm, codes_tr, scale_tr);
 }
 
 /*

@@ -156,3 +156,104 @@ def test_product_is_the_binary64_matmul_of_the_decoded_codes():
     want = oracle.e4m3_decode(a) @ oracle.e4m3_decode(b).T
     assert np.array_equal(acc, want)            # sums of this length are exact in binary64
     assert np.array_equal(out, want * (s_row[:, None] * s_col[None, :]).astype(np.float32).astype(np.float64))
+
+
+# ---------------------------------------------------------------------------------------------
+# E4M2, E4M1, E4M0: the E4M3 values with fewer mantissa bits (same exponent field and bias)
+# ---------------------------------------------------------------------------------------------
+import pytest
+
+
+def _grid_k(k):
+    """Sorted finite values of a format with 1 sign, 4 exponent (bias 7) and k mantissa bits,
+    subnormals at exponent field 0, written from that definition (no oracle code).  For k = 3 the
+    all-ones code is NaN and is left out."""
+    vals = set()
+    for ex in range(16):
+        for man in range(2 ** k):
+            if k == 3 and ex == 15 and man == 7:
+                continue
+            v = Fraction(man, 2 ** k) * Fraction(1, 64) if ex == 0 else (1 + Fraction(man, 2 ** k)) * Fraction(2) ** (ex - 7)
+            vals.add(v)
+            vals.add(-v)
+    return sorted(vals)
+
+
+@pytest.mark.parametrize("k", [0, 1, 2, 3])
+def test_narrow_grids_are_subsets_of_e4m3_with_the_stated_maxima(k):
+    g3, gk = set(_grid_k(3)), _grid_k(k)
+    assert set(gk) <= g3                                  # every value has an E4M3 code
+    assert max(gk) == Fraction(oracle.e4m_max(k)) == {0: 256, 1: 384, 2: 448, 3: 448}[k]
+    # grid values never move, whatever the threshold, and their codes have the low mantissa bits clear
+    for v in gk:
+        for u in (0, 2 ** 23, 2 ** 24 - 1):
+            c = oracle.quantize_e4m_scalar(float(v), 1.0, k, SR, u)
+            assert Fraction(float(oracle.e4m3_decode([c])[0])) == v and (c & ((1 << (3 - k)) - 1)) == 0
+        assert Fraction(float(oracle.e4m3_decode([oracle.quantize_e4m_scalar(float(v), 1.0, k, RTN)])[0])) == v
+
+
+@pytest.mark.parametrize("k", [0, 1, 2])
+def test_narrow_grids_round_to_a_neighbour_with_the_exact_probability(k):
+    grid = _grid_k(k)
+    top = float(max(grid))
+    rng = np.random.default_rng(10 + k)
+    ts = np.concatenate([rng.uniform(-top, top, 300), rng.normal(0, 1, 300), rng.normal(0, 0.01, 200)]).astype(np.float32)
+    for t in ts:
+        T = Fraction(float(t))
+        lo = max(g for g in grid if g <= T)
+        hi = min(g for g in grid if g >= T)
+        if lo == hi:
+            continue
+        P = (T - lo) / (hi - lo) * 2 ** 24
+        kk = -(-P.numerator // P.denominator)          # ceil(P): thresholds 0 .. kk-1 go up
+        for u, up in ((0, kk > 0), (kk - 1, True), (kk, False), (2 ** 24 - 1, False)):
+            if 0 <= u < 2 ** 24:
+                v = Fraction(float(oracle.e4m3_decode([oracle.quantize_e4m_scalar(float(t), 1.0, k, SR, u)])[0]))
+                assert v == (hi if up else lo), (k, float(t), u)
+        # Def. 2: the nearer neighbour, the upper one at a tie
+        v = Fraction(float(oracle.e4m3_decode([oracle.quantize_e4m_scalar(float(t), 1.0, k, RTN)])[0]))
+        assert v == (hi if (T - lo) >= (hi - T) else lo), (k, float(t))
+
+
+@pytest.mark.parametrize("k", [0, 1, 2])
+def test_narrow_grid_scale_rule_and_matrix_form(k):
+    top = oracle.e4m_max(k)
+    rng = np.random.default_rng(20 + k)
+    for m in rng.uniform(1e-3, 100, 200).astype(np.float32):
+        d, inv = oracle.scale_e4m(float(m), k)
+        exact = Fraction(top) / Fraction(float(m))
+        assert Fraction(float(inv)) <= exact < Fraction(float(np.nextafter(inv, np.float32(np.inf))))
+        assert d == np.float32(m) / np.float32(top) and np.float32(m) * inv <= top
+    assert oracle.scale_e4m(0.0, k) == (0, 0)
+    # matrix form against the restatement in exact rationals, both layouts, per row
+    grid = _grid_k(k)
+    x = (rng.normal(0, 1, (7, 10)) * rng.choice([1, 1, 30], (7, 10))).astype(np.float32)
+    x[3] = 0
+    q = QSpec(5 + k, PER_ROW, SR, seed=5, tensor_id=2, index_offset=9)
+    crm, srm, ctr, stt = oracle.sr_quantize_e4m3(x, q, True, True)
+    u = thresholds_u24(5, 2, 9, 7, 10)
+    for codes, maxima, axis in ((crm, np.abs(x).max(axis=1), 0), (ctr.T, np.abs(x).max(axis=0), 1)):
+        for idx in np.ndindex(x.shape):
+            inv = oracle.scale_e4m(float(maxima[idx[axis]]), k)[1]
+            T = Fraction(float(np.float32(x[idx] * np.float32(inv))))
+            lo = max(g for g in grid if g <= T)
+            hi = min(g for g in grid if g >= T)
+            want = lo if lo == hi or not Fraction(int(u[idx]), 2 ** 24) < (T - lo) / (hi - lo) else hi
+            assert Fraction(float(oracle.e4m3_decode([codes[idx]])[0])) == want
+    assert np.array_equal(srm, np.array([oracle.scale_e4m(float(m), k)[0] for m in np.abs(x).max(axis=1)], dtype=np.float32))
+
+
+def test_sr_is_unbiased_on_e4m1():
+    rng = np.random.default_rng(31)
+    x = rng.normal(0, 1, (1, 256)).astype(np.float32)
+    draws = 2000
+    acc = np.zeros((1, 256))
+    for seed in range(draws):
+        c, s, _, _ = oracle.sr_quantize_e4m3(x, QSpec(6, PER_TENSOR, SR, seed, 1))
+        acc += oracle.e4m3_decode(c)
+    d, inv = oracle.scale_e4m(float(np.abs(x).max()), 1)
+    t = x.astype(np.float64) * float(inv)
+    step = 2.0 ** (np.maximum(np.floor(np.log2(np.abs(t))), -6) - 1)
+    p = t / step - np.floor(t / step)
+    sigma = step * np.sqrt(p * (1 - p) / draws)
+    assert np.all(np.abs(acc / draws - t) <= 5 * sigma + 1e-12)
