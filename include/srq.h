@@ -79,15 +79,19 @@ typedef enum { SRQ_PER_TENSOR = 0, SRQ_PER_ROW = 1 } srq_scale_t;
  * byte (i & 3) of word ((i >> 2) & 3) of Philox block i >> 4, so that one block serves 16 elements.
  * P(round up) is the fraction rounded to the nearest 1/256.  Integer grid only. */
 typedef enum { SRQ_SR = 0, SRQ_RTN = 1, SRQ_SR8 = 2 } srq_round_t;
-/* Grid of a quantization point: integers times the step size (bits 2..8), or the E4M3 8-bit
- * floating-point values times the step size (1 sign, 4 exponent, 3 mantissa bits, bias 7, no
- * infinities, largest value 448; `bits` is ignored). */
+/* Grid of a quantization point: integers times the step size (bits 2..8), or 8-bit floating-point
+ * values times the step size.  SRQ_GRID_E4M3 with bits = 8 is E4M3 (1 sign, 4 exponent, 3 mantissa
+ * bits, bias 7, no infinities, largest value 448); bits = 7, 6, 5 select E4M2, E4M1, E4M0, the
+ * formats of the paper's experiments section, taken as the E4M3 values with 2, 1, 0 mantissa bits
+ * (largest values 448, 384, 256; Def. 1 with the binade's own step).  Their codes are E4M3 bytes
+ * with the low mantissa bits clear, so one product (kind::f8f6f4) serves all four. */
 typedef enum { SRQ_GRID_INT = 0, SRQ_GRID_E4M3 = 1, SRQ_GRID_NONE = 2 /* operand left unquantized */ } srq_grid_t;
 
 /* One quantization point: the paper's (D, eps) pair for one operand of one pass
  * (five per layer: A and W forward; A, W and dY backward). */
 typedef struct {
-    int32_t bits;          /* 2..8; codes are stored one per int8 whatever the width */
+    int32_t bits;          /* integer grid: 2..8 (codes are stored one per int8 whatever the width);
+                              floating-point grid: 8, 7, 6, 5 = E4M3, E4M2, E4M1, E4M0 */
     int32_t scale;         /* srq_scale_t */
     int32_t round;         /* srq_round_t */
     int32_t format;        /* srq_grid_t; 0 = integer grid */

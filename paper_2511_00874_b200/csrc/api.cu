@@ -12,6 +12,7 @@ srq_status_t check_qspec(const srq_qspec_t* q) {
     if (!q) return SRQ_ERR_INVALID_ARG;
     if (q->format != SRQ_GRID_INT && q->format != SRQ_GRID_E4M3) return SRQ_ERR_INVALID_ARG;
     if (q->format == SRQ_GRID_INT && (q->bits < 2 || q->bits > 8)) return SRQ_ERR_UNSUPPORTED;
+    if (q->format == SRQ_GRID_E4M3 && (q->bits < 5 || q->bits > 8)) return SRQ_ERR_UNSUPPORTED;   // E4M0 .. E4M3
     if (q->scale != SRQ_PER_TENSOR && q->scale != SRQ_PER_ROW) return SRQ_ERR_INVALID_ARG;
     if (q->round != SRQ_SR && q->round != SRQ_RTN && q->round != SRQ_SR8) return SRQ_ERR_INVALID_ARG;
     if (q->round == SRQ_SR8 && q->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;

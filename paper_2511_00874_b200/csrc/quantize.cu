@@ -314,10 +314,12 @@ __device__ __forceinline__ uint32_t quantize_sum(float x, float inv, uint32_t wo
 // field (next binade), |q| < 8 only occurs for E = 121 and gives the subnormal codes, q = 0 gives +0.
 // Returns the code in the low byte.
 template <int MODE>
-__device__ __forceinline__ uint32_t quantize_e4m3(float x, float inv, uint32_t word) {
+__device__ __forceinline__ uint32_t quantize_e4m3(float x, float inv, uint32_t word, uint32_t sh) {
+    // sh = 3 - k for the E4Mk grid (k mantissa bits; 0 for E4M3 itself): the step of binade e is
+    // 2^(e-k), q counts those steps, and q << sh is the same value in the E4M3 code's units of 2^(e-3)
     const float t = __fmul_rn(x, inv);
     const uint32_t E = max((__float_as_uint(t) >> 23) & 0xFFu, 121u);          // |t| <= 448: E <= 135
-    const float s = __fmul_rn(t, __uint_as_float((281u - E) << 23));            // t 2^(3-e) 2^24, exact
+    const float s = __fmul_rn(t, __uint_as_float((281u - sh - E) << 23));       // t 2^(k-e) 2^24, exact
     uint32_t sum;
     if constexpr ((MODE & MODE_SR) != 0) {
         const int c = __float2int_ru(s);
@@ -326,7 +328,7 @@ __device__ __forceinline__ uint32_t quantize_e4m3(float x, float inv, uint32_t w
         sum = (uint32_t)__float2int_rd(s) + 0x00800000u;
     }
     const int q = (int)sum >> 24;
-    return ((uint32_t)q & 0x80u) | ((E << 3) + (uint32_t)abs(q) - 968u);
+    return ((uint32_t)q & 0x80u) | ((E << 3) + ((uint32_t)abs(q) << sh) - 968u);
 }
 
 // 8-random-bit mode: the threshold words of four consecutive elements from the stream word that holds
@@ -339,12 +341,12 @@ __device__ __forceinline__ void sr8_words(uint32_t w, uint32_t rnd[4]) {
 // Four codes packed into one word, first element in the low byte.
 template <int MODE>
 __device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3,
-                                              const uint32_t rnd[4]) {
+                                              const uint32_t rnd[4], uint32_t sh) {
     if constexpr ((MODE & MODE_SR8) != 0) {
-        return quantize4<MODE_SR>(v, i0, i1, i2, i3, rnd);
+        return quantize4<MODE_SR>(v, i0, i1, i2, i3, rnd, sh);
     } else if constexpr ((MODE & MODE_E4M3) != 0) {
-        const uint32_t c0 = quantize_e4m3<MODE>(v[0], i0, rnd[0]), c1 = quantize_e4m3<MODE>(v[1], i1, rnd[1]);
-        const uint32_t c2 = quantize_e4m3<MODE>(v[2], i2, rnd[2]), c3 = quantize_e4m3<MODE>(v[3], i3, rnd[3]);
+        const uint32_t c0 = quantize_e4m3<MODE>(v[0], i0, rnd[0], sh), c1 = quantize_e4m3<MODE>(v[1], i1, rnd[1], sh);
+        const uint32_t c2 = quantize_e4m3<MODE>(v[2], i2, rnd[2], sh), c3 = quantize_e4m3<MODE>(v[3], i3, rnd[3], sh);
         return __byte_perm(__byte_perm(c0, c1, 0x0040), __byte_perm(c2, c3, 0x0040), 0x5410);
     } else {
         const uint32_t s0 = quantize_sum<MODE>(v[0], i0, rnd[0]), s1 = quantize_sum<MODE>(v[1], i1, rnd[1]);
@@ -355,13 +357,13 @@ __device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float 
 
 // Same with the mode chosen at run time (general path).
 __device__ __forceinline__ uint32_t quantize4_rt(int mode, const float v[4], float i0, float i1, float i2, float i3,
-                                                 const uint32_t rnd[4]) {
+                                                 const uint32_t rnd[4], uint32_t sh) {
     switch (mode) {
-        case 0: return quantize4<0>(v, i0, i1, i2, i3, rnd);
-        case 1: return quantize4<1>(v, i0, i1, i2, i3, rnd);
-        case 2: return quantize4<2>(v, i0, i1, i2, i3, rnd);
-        case 3: return quantize4<3>(v, i0, i1, i2, i3, rnd);
-        default: return quantize4<MODE_SR>(v, i0, i1, i2, i3, rnd);      // MODE_SR8: thresholds already in word form
+        case 0: return quantize4<0>(v, i0, i1, i2, i3, rnd, sh);
+        case 1: return quantize4<1>(v, i0, i1, i2, i3, rnd, sh);
+        case 2: return quantize4<2>(v, i0, i1, i2, i3, rnd, sh);
+        case 3: return quantize4<3>(v, i0, i1, i2, i3, rnd, sh);
+        default: return quantize4<MODE_SR>(v, i0, i1, i2, i3, rnd, sh);      // MODE_SR8: thresholds already in word form
     }
 }
 
@@ -382,6 +384,7 @@ struct QuantParams {
     PhiloxKeys keys;
     int sr;                       // 1 = SR, 0 = RTN
     int mode;                     // MODE_SR | MODE_E4M3
+    uint32_t e4m_shift;           // E4Mk grid: 3 - k (0 for E4M3 and for the integer grid)
     int per_row;                  // step size per row of each layout
     int8_t* codes_rm; int64_t ld_rm;
     int8_t* codes_tr; int64_t ld_tr;
@@ -521,9 +524,9 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
             }
             if constexpr (WANT_RM || !TWO_STEPS) {
                 const float ir = (PER_ROW && WANT_RM) ? inv_cur[i] : inv_tensor;
-                wr[i] = quantize4<MODE>(v, ir, ir, ir, ir, rnd);
+                wr[i] = quantize4<MODE>(v, ir, ir, ir, ir, rnd, P.e4m_shift);
             }
-            if constexpr (TWO_STEPS) wt[i] = quantize4<MODE>(v, ic[0], ic[1], ic[2], ic[3], rnd);
+            if constexpr (TWO_STEPS) wt[i] = quantize4<MODE>(v, ic[0], ic[1], ic[2], ic[3], rnd, P.e4m_shift);
             else wt[i] = wr[i];
             if constexpr (WANT_RM) {
                 if (FULL || (col_ok && r0 + tr < P.rows)) *reinterpret_cast<uint32_t*>(out_rm + tr * ld_rm) = wr[i];
@@ -661,7 +664,7 @@ quantize_rows_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
                 const uint32_t lo = (uint32_t)jb + g;
                 philox_rounds(lo, (uint32_t)(jb >> 32) + (lo < g ? 1u : 0u), P.keys, rnd);
             }
-            w[k] = quantize4<MODE>(v, inv, inv, inv, inv, rnd);
+            w[k] = quantize4<MODE>(v, inv, inv, inv, inv, rnd, P.e4m_shift);
         }
 #pragma unroll
         for (int k = 0; k < G; ++k) {
@@ -764,9 +767,9 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
                 }
                 const float inv_r = P.per_row ? P.inv_rm[want_rm ? r : 0] : inv_tensor;
                 if (want_rm || !two_steps)
-                    wr[i] = quantize4_rt(P.mode, v, inv_r, inv_r, inv_r, inv_r, rnd);
+                    wr[i] = quantize4_rt(P.mode, v, inv_r, inv_r, inv_r, inv_r, rnd, P.e4m_shift);
                 if (two_steps)
-                    wt[i] = quantize4_rt(P.mode, v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], rnd);
+                    wt[i] = quantize4_rt(P.mode, v, inv_c[0], inv_c[1], inv_c[2], inv_c[3], rnd, P.e4m_shift);
                 else
                     wt[i] = wr[i];
                 if (want_rm) {
@@ -871,7 +874,9 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     const int64_t rows = a.rows, cols = a.cols;
     if (rows == 0 || cols == 0 || (!want_rm && !want_tr)) return cudaSuccess;
     const bool e4m3 = a.q.format == SRQ_GRID_E4M3;
-    const float qmax = e4m3 ? 448.0f : (float)((1 << (a.q.bits - 1)) - 1);
+    // E4Mk grid: bits = 5 + k; the largest value with k mantissa bits is 448 (k = 3, 2), 384 (k = 1), 256 (k = 0)
+    const int mant = e4m3 ? a.q.bits - 5 : 3;
+    const float qmax = e4m3 ? (mant >= 2 ? 448.0f : (mant == 1 ? 384.0f : 256.0f)) : (float)((1 << (a.q.bits - 1)) - 1);
     const size_t esize = a.dt == SRQ_F32 ? 4 : 2;
 
     // group counts and where each layout's absmax lives; per tensor both layouts share word 0
@@ -895,6 +900,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     P.sr = a.q.round == SRQ_SR;
     const bool sr8 = a.q.round == SRQ_SR8;
     P.mode = sr8 ? MODE_SR8 : ((P.sr ? MODE_SR : 0) | (e4m3 ? MODE_E4M3 : 0));
+    P.e4m_shift = (uint32_t)(3 - mant);
     P.per_row = per_row;
     P.codes_rm = a.codes_rm; P.ld_rm = a.ld_rm;
     P.codes_tr = a.codes_tr; P.ld_tr = a.ld_tr;

@@ -14,8 +14,8 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-5
 
 
-def _q(scale, rnd, seed=0, tid=0, off=0):
-    return srq.QSpec(8, scale, rnd, seed, tid, off, srq.GRID_E4M3)
+def _q(scale, rnd, seed=0, tid=0, off=0, bits=8):
+    return srq.QSpec(bits, scale, rnd, seed, tid, off, srq.GRID_E4M3)
 
 
 def _oq(q):
@@ -154,3 +154,53 @@ def test_operands_of_one_product_must_share_the_grid():
     with pytest.raises(srq.SrqError) as e:
         srq.qlinear_fwd(A, W, _q(srq.PER_TENSOR, srq.SR), srq.QSpec(8), Y)
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("bits", [7, 6, 5])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_narrow_formats_e4m2_e4m1_e4m0(bits, dtype):
+    """The E4M3 values with 2, 1, 0 mantissa bits: codes and step sizes bit for bit, both layouts,
+    fast and general quantizer paths, the one-pass per-row kernel; every code has its low mantissa
+    bits clear; the layer passes run on the same product as E4M3."""
+    low = (1 << (8 - bits)) - 1
+    for shape, off in (((300, 388), 0), ((131, 259), 3), ((40, 1024), 4)):
+        x = synth.with_outliers(shape, seed=bits, dtype=dtype, device="cuda")
+        x[1] = 0
+        for scale in (srq.PER_TENSOR, srq.PER_ROW):
+            for rnd in (srq.SR, srq.RTN):
+                q = _q(scale, rnd, seed=6, tid=2 ** 33 + 1, off=off, bits=bits)
+                _check_quantizer(x, q)
+                crm = _quantize_gpu(x, q, True, False)[0]          # rows of 1024: one-pass per-row kernel
+                assert not (crm & low).any()
+                ref = oracle.sr_quantize_e4m3(x.float().cpu().numpy(), _oq(q), True, False)
+                assert np.array_equal(crm, ref[0])
+    T, N, K = 136, 264, 200
+    A, W, dY = synth.layer_inputs(T, N, K, seed=2, dtype=dtype, device="cuda", std_dy=1e-3)
+    qa, qw, qdy = (_q(srq.PER_ROW, srq.SR, seed=1, tid=i, bits=bits) for i in range(3))
+    f = lambda t: t.float().cpu().numpy()
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
+    Y = torch.empty((T, N), device="cuda")
+    dbg = srq.DebugOut(torch.empty((T, K), dtype=torch.int8, device="cuda"), torch.empty(T, device="cuda"),
+                       torch.empty((N, K), dtype=torch.int8, device="cuda"), torch.empty(N, device="cuda"), None)
+    srq.qlinear_fwd(A, W, qa, qw, Y, dbg, ws)
+    assert srq.srq_poll_status(ws) == 0
+    ref = oracle.qlinear_fwd_e4m3(f(A), f(W), _oq(qa), _oq(qw))
+    assert np.array_equal(dbg.codes_a.view(torch.uint8).cpu().numpy(), ref.codes_a)
+    assert np.array_equal(dbg.codes_b.view(torch.uint8).cpu().numpy(), ref.codes_b)
+    _, out_b = _bound(ref.codes_a, ref.codes_b, ref.scale_a, ref.scale_b)
+    assert np.all(np.abs(Y.cpu().numpy().astype(np.float64) - ref.out) <= out_b * 1.001 + np.abs(ref.out) * 2e-7)
+    dW = torch.empty((N, K), device="cuda")
+    srq.qlinear_bwd_weight(dY, A, qdy, qa, dW, None, ws)
+    assert srq.srq_poll_status(ws) == 0
+    ref = oracle.qlinear_bwd_weight_e4m3(f(dY), f(A), _oq(qdy), _oq(qa))
+    _, out_b = _bound(ref.codes_a, ref.codes_b, ref.scale_a, ref.scale_b)
+    assert np.all(np.abs(dW.cpu().numpy().astype(np.float64) - ref.out) <= out_b * 1.001 + np.abs(ref.out) * 2e-7)
+
+
+def test_floating_point_grid_rejects_other_widths():
+    x = synth.normal((64, 64), 1.0, seed=1, device="cuda")
+    c = torch.empty((64, 64), dtype=torch.int8, device="cuda")
+    sc = torch.empty(1, device="cuda")
+    with pytest.raises(srq.SrqError) as e:
+        srq.sr_quantize(x, _q(srq.PER_TENSOR, srq.SR, bits=4), c, sc, None, None)
+    assert e.value.status == 2
