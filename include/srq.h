@@ -98,11 +98,15 @@ typedef struct {
     uint64_t seed;         /* Philox key; one per training step */
     uint64_t tensor_id;    /* Philox counter words 2-3; one per (layer, operand, pass) */
     uint64_t index_offset; /* added to the flat index; first_row*cols for a row shard */
-    const float *absmax;   /* optional, DEVICE pointer to one float: max |x| of the operand when the
-                            * caller already knows it (srq_absmax, or an all-reduced maximum over
-                            * token shards).  The absmax pass over the operand is then skipped.  Only
-                            * with SRQ_PER_TENSOR.  The value must not be smaller than the true
-                            * maximum (codes are unspecified otherwise).  NULL: compute it. */
+    const float *absmax;   /* optional, DEVICE pointer.  SRQ_PER_TENSOR: one float, max |x| of the operand
+                            * when the caller already knows it (srq_absmax, or an all-reduced maximum
+                            * over token shards); the absmax pass over the operand is then skipped.
+                            * SRQ_PER_ROW: [cols] floats, max |x[:, c]| of every column of the source
+                            * matrix (srq_absmax_cols, max-reduced over token shards), used for the
+                            * step sizes of the TRANSPOSED layout, whose groups run over the rows,
+                            * i.e. over tokens other shards may hold; the row-major layout's row
+                            * maxima are always computed here.  Values must not be smaller than the
+                            * true maxima (codes are unspecified otherwise).  NULL: compute them. */
 } srq_qspec_t;
 
 /* Optional copies of what a layer pass fed to its product: dense code matrices in the layout
@@ -172,6 +176,12 @@ srq_status_t sr_quantize_static(const void *x, srq_dtype_t dt, int64_t rows, int
  * all-reduce it over token shards, through srq_qspec_t.absmax.  Needs no workspace. */
 srq_status_t srq_absmax(const void *x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
                         float *absmax, void *cuda_stream);
+
+/* max |x[:, c]| of every column into absmax_cols (device, [cols] floats, overwritten): what a token
+ * shard contributes to the per-row step sizes of the transposed layout (the operands of the
+ * weight-gradient product); max-reduce it over the shards and pass it through srq_qspec_t.absmax. */
+srq_status_t srq_absmax_cols(const void *x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld,
+                             float *absmax_cols, void *cuda_stream);
 
 /*
  * The product of two quantized matrices (mixed-precision matmul subsection): int8 codes

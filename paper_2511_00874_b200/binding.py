@@ -26,7 +26,7 @@ SR, RTN, SR8 = 0, 1, 2
 GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
-           "sr_quantize", "sr_quantize_static", "srq_absmax", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
+           "sr_quantize", "sr_quantize_static", "srq_absmax", "srq_absmax_cols", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
            "srq_gemm_i8_ex", "qlinear_fwd_ex", "qlinear_bwd_ex",
            "srq_poll_status", "srq_status_string", "srq_launch_count", "srq_selftest_bounded_wait", "srq_plan_splits"]
 
@@ -98,6 +98,8 @@ def lib() -> ctypes.CDLL:
     L.sr_quantize.restype = ctypes.c_int
     L.srq_absmax.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, vp]
     L.srq_absmax.restype = ctypes.c_int
+    L.srq_absmax_cols.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, vp]
+    L.srq_absmax_cols.restype = ctypes.c_int
     L.sr_quantize_static.argtypes = [vp, ctypes.c_int, i64, i64, i64, qp, vp, i64, vp, vp, i64, vp, vp, vp]
     L.sr_quantize_static.restype = ctypes.c_int
     L.srq_gemm_i8.argtypes = [vp, i64, vp, i64, i64, i64, i64, vp, i32, vp, i32, vp, i64, vp, vp, sz, vp]
@@ -204,6 +206,15 @@ def srq_absmax(x: torch.Tensor, absmax: torch.Tensor) -> None:
     _dev2d(x, "x")
     st = lib().srq_absmax(x.data_ptr(), _dtype_of(x), x.shape[0], x.shape[1], x.stride(0), absmax.data_ptr(), _stream())
     _check(st, "srq_absmax")
+
+
+def srq_absmax_cols(x: torch.Tensor, absmax_cols: torch.Tensor) -> None:
+    """max |x[:, c]| of every column into the float32 CUDA tensor ``absmax_cols`` ([cols])."""
+    _dev2d(x, "x")
+    if absmax_cols.numel() < x.shape[1] or absmax_cols.dtype != torch.float32:
+        raise ValueError("absmax_cols must hold cols float32 values")
+    st = lib().srq_absmax_cols(x.data_ptr(), _dtype_of(x), x.shape[0], x.shape[1], x.stride(0), absmax_cols.data_ptr(), _stream())
+    _check(st, "srq_absmax_cols")
 
 
 def sr_quantize_static(x: torch.Tensor, q: QSpec, codes_rm: Optional[torch.Tensor] = None,

@@ -16,7 +16,7 @@ srq_status_t check_qspec(const srq_qspec_t* q) {
     if (q->scale != SRQ_PER_TENSOR && q->scale != SRQ_PER_ROW) return SRQ_ERR_INVALID_ARG;
     if (q->round != SRQ_SR && q->round != SRQ_RTN && q->round != SRQ_SR8) return SRQ_ERR_INVALID_ARG;
     if (q->round == SRQ_SR8 && q->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;
-    if (q->absmax && (q->scale != SRQ_PER_TENSOR || ((uintptr_t)q->absmax % 4) != 0)) return SRQ_ERR_INVALID_ARG;
+    if (q->absmax && ((uintptr_t)q->absmax % 4) != 0) return SRQ_ERR_INVALID_ARG;
     return SRQ_OK;
 }
 
@@ -387,6 +387,14 @@ srq_status_t srq_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t col
     if (dt != SRQ_F32 && dt != SRQ_BF16) return SRQ_ERR_INVALID_ARG;
     if (!aligned_to(x, 16) || !aligned_to(absmax, 4)) return SRQ_ERR_INVALID_ARG;
     return launch_absmax(x, dt, rows, cols, ld, absmax, (cudaStream_t)cuda_stream) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+}
+
+srq_status_t srq_absmax_cols(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax_cols,
+                             void* cuda_stream) {
+    if (!x || !absmax_cols || rows < 0 || cols < 0 || ld < cols) return SRQ_ERR_INVALID_ARG;
+    if (dt != SRQ_F32 && dt != SRQ_BF16) return SRQ_ERR_INVALID_ARG;
+    if (!aligned_to(x, 16) || !aligned_to(absmax_cols, 4)) return SRQ_ERR_INVALID_ARG;
+    return launch_absmax_cols(x, dt, rows, cols, ld, absmax_cols, (cudaStream_t)cuda_stream) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
 }
 
 srq_status_t srq_gemm_i8(const int8_t* a, int64_t lda, const int8_t* b, int64_t ldb, int64_t M, int64_t N, int64_t Kc,

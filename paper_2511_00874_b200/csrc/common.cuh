@@ -89,6 +89,9 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& scratch, uin
 
 // max |x| of the whole matrix into *absmax (device float, overwritten).
 cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax, cudaStream_t stream);
+// absmax_cols[c] = max over the rows of |x[r, c]| (device [cols], overwritten).
+cudaError_t launch_absmax_cols(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax_cols,
+                               cudaStream_t stream);
 
 // int8 codes as bfloat16 integers (pitches in elements); *one receives 1.0f.
 cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, int64_t ld, void* out_bf16, int64_t ld_out,

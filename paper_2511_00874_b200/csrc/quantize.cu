@@ -856,6 +856,19 @@ cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t c
     return cudaGetLastError();
 }
 
+// Column maxima: absmax_cols[c] = max_r |x[r, c]| (binary32, written from zero).
+cudaError_t launch_absmax_cols(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax_cols,
+                               cudaStream_t stream) {
+    if (cols == 0) return cudaSuccess;
+    cudaError_t e = cudaMemsetAsync(absmax_cols, 0, (size_t)cols * sizeof(float), stream);
+    if (e != cudaSuccess || rows == 0) return e;
+    const ScaleStep none = {};
+    if (dt == SRQ_F32) launch_amax<float>(x, rows, cols, ld, nullptr, false, (uint32_t*)absmax_cols, true, none, stream);
+    else launch_amax<__nv_bfloat16>(x, rows, cols, ld, nullptr, false, (uint32_t*)absmax_cols, true, none, stream);
+    ++g_launches;
+    return cudaGetLastError();
+}
+
 // SM count of the current device (asked once per device).
 static int sm_count() {
     static int cached[64] = {0};
@@ -888,7 +901,10 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     float* inv_tr = per_row ? s.inv_tr : s.inv_rm;
 
     const bool vec_in = ((uintptr_t)a.x % (4 * esize) == 0) && (a.ld % 4 == 0);
-    const bool given = a.q.absmax != nullptr && !per_row;   // a known absmax is only taken per tensor
+    const bool given = a.q.absmax != nullptr && !per_row;   // per tensor: one known maximum for the whole operand
+    // per row: known column maxima [cols] for the transposed layout (its groups run over the rows, i.e.
+    // over the tokens, which other shards may hold); the row-major layout's row maxima are local
+    const bool given_cols = a.q.absmax != nullptr && per_row && want_tr;
     // per tensor: one group feeds both layouts' scale outputs
     const int64_t n0 = per_row ? n_rm : 1;
     const int64_t n1 = per_row ? n_tr : ((want_tr && a.scale_tr) ? 1 : 0);
@@ -919,7 +935,24 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         return cudaGetLastError();
     }
 
-    if (given) {
+    if (given_cols) {
+        const int threads = 256;
+        if (want_rm) {                                  // row maxima of this shard, then their step sizes
+            if (!scratch_zeroed) {
+                cudaError_t e = cudaMemsetAsync(s.counter, 0, (size_t)((char*)s.inv_rm - (char*)s.counter), stream);
+                if (e != cudaSuccess) return e;
+            }
+            const ScaleStep none = {};
+            if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, amax_rm, true, nullptr, false, none, stream);
+            else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, amax_rm, true, nullptr, false, none, stream);
+            ++g_launches;
+        }
+        const uint32_t* col_bits = (const uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
+        const int64_t n = n0 > n1 ? n0 : n1;
+        scales_kernel<<<(unsigned)((n + threads - 1) / threads), threads, 0, stream>>>(
+            amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr, col_bits, n1, inv_tr, a.scale_tr, qmax, status);
+        ++g_launches;
+    } else if (given) {
         amax_rm = amax_tr = (uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
         const int64_t n = n0 > n1 ? n0 : n1;
         const int threads = 256;

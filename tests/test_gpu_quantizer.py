@@ -180,9 +180,6 @@ def test_absmax_entry_point_and_a_known_absmax(dtype):
     ref = oracle.sr_quantize(xs, oracle.QSpec(6, 0, 0, 3, 4), True, True)
     assert np.array_equal(got[0], ref[0][:300]) and np.array_equal(got[1], ref[1])
     assert np.array_equal(got[2], ref[2][:, :300])
-    with pytest.raises(srq.SrqError):                    # only with one step size per tensor
-        srq.sr_quantize(x, srq.QSpec(8, srq.PER_ROW, absmax=m), torch.empty((300, 388), dtype=torch.int8, device="cuda"),
-                        torch.empty(300, device="cuda"))
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
@@ -221,3 +218,55 @@ def test_one_pass_per_row_path_matches_the_oracle(dtype, shape, off):
     one = _run_gpu(x, q, True, False)
     two = _run_gpu(x, q, True, True)
     assert np.array_equal(one[0], two[0]) and np.array_equal(one[1], two[1])
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("shape", [(300, 388), (262, 131)])
+def test_token_shards_with_per_row_steps_share_their_column_maxima(dtype, shape):
+    """Per-row mode, transposed layout: its groups are the columns of the source, which run over the
+    tokens.  Two token shards that exchange their column maxima (srq_absmax_cols, then an element-wise
+    maximum as an all-reduce would form it) produce exactly the columns of codes, and the step sizes,
+    that one device produces on the whole tensor; row-major codes need no exchange."""
+    rows, cols = shape
+    x = synth.with_outliers(shape, seed=21, dtype=dtype, device="cuda")
+    x[:, 3] = 0
+    cut = 136
+    shards = [x[:cut].contiguous(), x[cut:].contiguous()]
+    cm = [torch.full((cols,), -1.0, device="cuda") for _ in shards]
+    for sh, m in zip(shards, cm):
+        srq.srq_absmax_cols(sh, m)
+        assert torch.equal(m, sh.float().abs().amax(dim=0))
+    shared = torch.maximum(cm[0], cm[1])
+    for bits, rnd in ((8, srq.SR), (4, srq.RTN)):
+        whole = oracle.sr_quantize(x.float().cpu().numpy(), oracle.QSpec(bits, oracle.PER_ROW, rnd, 5, 9), True, True)
+        first = 0
+        for sh in shards:
+            q = srq.QSpec(bits, srq.PER_ROW, rnd, 5, 9, index_offset=first * cols, absmax=shared)
+            for want_rm in (True, False):
+                got = _run_gpu(sh, q, want_rm, True)
+                n = sh.shape[0]
+                assert np.array_equal(got[2], whole[2][:, first:first + n]), "transposed codes of the shard"
+                assert np.array_equal(got[3], whole[3]), "column step sizes"
+                if want_rm:
+                    assert np.array_equal(got[0], whole[0][first:first + n]) and np.array_equal(got[1], whole[1][first:first + n])
+            first += sh.shape[0]
+    # the weight-gradient product of the shards then adds up to the unsharded one, int32 sums exactly
+    A = synth.normal((rows, 72), 1.0, seed=3, dtype=dtype, device="cuda")
+    ma, mx = torch.empty(72, device="cuda"), torch.empty(cols, device="cuda")
+    srq.srq_absmax_cols(A, ma)
+    srq.srq_absmax_cols(x, mx)
+    f = lambda t: t.float().cpu().numpy()
+    ref = oracle.qlinear_bwd_weight(f(x), f(A), oracle.QSpec(8, oracle.PER_ROW, oracle.SR, 1, 4), oracle.QSpec(8, oracle.PER_ROW, oracle.SR, 1, 2))
+    total = np.zeros_like(ref.acc, dtype=np.int64)
+    first = 0
+    for lo, hi in ((0, cut), (cut, rows)):
+        T = hi - lo
+        dW = torch.empty((cols, 72), device="cuda")
+        acc = torch.empty((cols, 72), dtype=torch.int32, device="cuda")
+        dbg = srq.DebugOut(None, torch.empty(cols, device="cuda"), None, torch.empty(72, device="cuda"), acc)
+        srq.qlinear_bwd_weight(x[lo:hi].contiguous(), A[lo:hi].contiguous(),
+                               srq.QSpec(8, srq.PER_ROW, srq.SR, 1, 4, index_offset=lo * cols, absmax=mx),
+                               srq.QSpec(8, srq.PER_ROW, srq.SR, 1, 2, index_offset=lo * 72, absmax=ma), dW, dbg)
+        assert np.array_equal(dbg.scale_a.cpu().numpy(), ref.scale_a) and np.array_equal(dbg.scale_b.cpu().numpy(), ref.scale_b)
+        total += acc.cpu().numpy()
+    assert np.array_equal(total, ref.acc.astype(np.int64))
