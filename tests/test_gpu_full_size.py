@@ -2,7 +2,8 @@
 
 Linear layer 4096 -> 4096 with 65536 tokens, fp32 inputs, 8-bit per-tensor SR: the workload
 `bench.py` times, called the way it calls it (no debug copies, so the products run as CTA pairs
-and store their results as whole blocks).  The oracle cannot form 3 x 1.1e12 products in a test,
+and store their results as whole blocks); and the largest layer of the per-row configuration
+(2048 -> 5632, 65536 tokens, bf16 inputs, 8-bit forward, 4-bit backward).  The oracle cannot form 3 x 1.1e12 products in a test,
 so the comparison is:
   - every int8 code and step size of all operands against the oracle's quantizer (bit for bit);
   - sampled rows of Y, dA and dW against oracle products of the oracle's codes (bit for bit);
@@ -20,8 +21,6 @@ from paper_2511_00874_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-T, N, K = 65536, 4096, 4096
-
 
 def _oq(q):
     return oracle.QSpec(q.bits, q.scale, q.round, q.seed, q.tensor_id, q.index_offset)
@@ -29,11 +28,13 @@ def _oq(q):
 
 def _codes(x, q, rm, tr):
     rows, cols = x.shape
+    per_row = q.scale == srq.PER_ROW
     crm = torch.empty((rows, cols), dtype=torch.int8, device="cuda") if rm else None
     ctr = torch.empty((cols, rows), dtype=torch.int8, device="cuda") if tr else None
-    s1, s2 = torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
+    s1 = torch.empty(rows if per_row else 1, device="cuda")
+    s2 = torch.empty(cols if per_row else 1, device="cuda")
     srq.sr_quantize(x, q, crm, s1 if rm else None, ctr, s2 if tr else None)
-    return crm, ctr, (s1 if rm else s2)
+    return crm, ctr, s1 if rm else None, s2 if tr else None
 
 
 def _freivalds(acc, qa, qb, rng):
@@ -50,11 +51,22 @@ def _freivalds(acc, qa, qb, rng):
             assert torch.equal(lhs[i:i + 8192], qa[i:i + 8192].double() @ right)
 
 
-def test_benchmark_layer_at_full_size():
-    A = synth.normal((T, K), 1.0, 1000, torch.float32, "cuda")
-    dY = synth.normal((T, N), 1e-3, 1001, torch.float32, "cuda")
-    W = synth.normal((N, K), 0.02, 7, torch.float32, "cuda")
-    q = {k: srq.QSpec(8, srq.PER_TENSOR, srq.SR, 3, i) for i, k in enumerate(["a_f", "w_f", "a_b", "w_b", "dy"])}
+CASES = {
+    # the benchmark workload: linear 4096 -> 4096, fp32, 8-bit per-tensor SR
+    "bench": (65536, 4096, 4096, torch.float32, srq.PER_TENSOR, 8, 8),
+    # the largest Llama-style layer of the per-row configuration: bf16, 8-bit forward, 4-bit backward
+    "gate_up": (65536, 5632, 2048, torch.bfloat16, srq.PER_ROW, 8, 4),
+}
+
+
+@pytest.mark.parametrize("case", list(CASES))
+def test_layer_at_full_size(case):
+    T, N, K, dtype, scale, bits_f, bits_b = CASES[case]
+    A = synth.normal((T, K), 1.0, 1000, dtype, "cuda")
+    dY = synth.normal((T, N), 1e-3, 1001, dtype, "cuda")
+    W = synth.normal((N, K), 0.02, 7, dtype, "cuda")
+    bits = {"a_f": bits_f, "w_f": bits_f, "a_b": bits_b, "w_b": bits_b, "dy": bits_b}
+    q = {k: srq.QSpec(bits[k], scale, srq.SR, 3, i) for i, k in enumerate(["a_f", "w_f", "a_b", "w_b", "dy"])}
     ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
     Y = torch.empty((T, N), device="cuda")
     dA = torch.empty((T, K), device="cuda")
@@ -64,21 +76,21 @@ def test_benchmark_layer_at_full_size():
     assert srq.srq_poll_status(ws) == 0
 
     # ---- codes and step sizes of every operand, whole tensors, against the oracle
-    hA, hW, hdY = A.cpu().numpy(), W.cpu().numpy(), dY.cpu().numpy()
+    hA, hW, hdY = A.float().cpu().numpy(), W.float().cpu().numpy(), dY.float().cpu().numpy()
     o_af = oracle.sr_quantize(hA, _oq(q["a_f"]), True, False)
     o_wf = oracle.sr_quantize(hW, _oq(q["w_f"]), True, False)
     o_dy = oracle.sr_quantize(hdY, _oq(q["dy"]), True, True)
     o_wb = oracle.sr_quantize(hW, _oq(q["w_b"]), False, True)
     o_ab = oracle.sr_quantize(hA, _oq(q["a_b"]), False, True)
-    g_af, _, s_af = _codes(A, q["a_f"], True, False)
-    g_wf, _, s_wf = _codes(W, q["w_f"], True, False)
-    g_dy, g_dyt, s_dy = _codes(dY, q["dy"], True, True)
-    _, g_wbt, s_wb = _codes(W, q["w_b"], False, True)
-    _, g_abt, s_ab = _codes(A, q["a_b"], False, True)
+    g_af, _, s_af, _ = _codes(A, q["a_f"], True, False)
+    g_wf, _, s_wf, _ = _codes(W, q["w_f"], True, False)
+    g_dy, g_dyt, s_dy, s_dyt = _codes(dY, q["dy"], True, True)
+    _, g_wbt, _, s_wb = _codes(W, q["w_b"], False, True)
+    _, g_abt, _, s_ab = _codes(A, q["a_b"], False, True)
     for name, g, o in (("A fwd", g_af, o_af[0]), ("W fwd", g_wf, o_wf[0]), ("dY", g_dy, o_dy[0]),
                        ("dY^T", g_dyt, o_dy[2]), ("W^T bwd", g_wbt, o_wb[2]), ("A^T bwd", g_abt, o_ab[2])):
         assert np.array_equal(g.cpu().numpy(), o), name + ": codes"
-    for name, g, o in (("A fwd", s_af, o_af[1]), ("W fwd", s_wf, o_wf[1]), ("dY", s_dy, o_dy[1]),
+    for name, g, o in (("A fwd", s_af, o_af[1]), ("W fwd", s_wf, o_wf[1]), ("dY", s_dy, o_dy[1]), ("dY^T", s_dyt, o_dy[3]),
                        ("W bwd", s_wb, o_wb[3]), ("A bwd", s_ab, o_ab[3])):
         assert np.array_equal(g.cpu().numpy(), o), name + ": step size"
 
@@ -86,19 +98,20 @@ def test_benchmark_layer_at_full_size():
     rng = np.random.default_rng(0)
     rows_t = np.sort(rng.choice(T, 48, replace=False))
     rows_n = np.sort(rng.choice(N, 12, replace=False))
-    ref = oracle.dequant(oracle.gemm_i8_nt(o_af[0][rows_t], o_wf[0]), o_af[1], o_wf[1])
+    pick = lambda sc, rows: sc if sc.size == 1 else sc[rows]
+    ref = oracle.dequant(oracle.gemm_i8_nt(o_af[0][rows_t], o_wf[0]), pick(o_af[1], rows_t), o_wf[1])
     assert np.array_equal(Y[torch.from_numpy(rows_t).cuda()].cpu().numpy(), ref), "Y rows"
-    ref = oracle.dequant(oracle.gemm_i8_nt(o_dy[0][rows_t], o_wb[2]), o_dy[1], o_wb[3])
+    ref = oracle.dequant(oracle.gemm_i8_nt(o_dy[0][rows_t], o_wb[2]), pick(o_dy[1], rows_t), o_wb[3])
     assert np.array_equal(dA[torch.from_numpy(rows_t).cuda()].cpu().numpy(), ref), "dA rows"
-    ref = oracle.dequant(oracle.gemm_i8_nt(o_dy[2][rows_n], o_ab[2]), o_dy[3], o_ab[3])
+    ref = oracle.dequant(oracle.gemm_i8_nt(o_dy[2][rows_n], o_ab[2]), pick(o_dy[3], rows_n), o_ab[3])
     assert np.array_equal(dW[torch.from_numpy(rows_n).cuda()].cpu().numpy(), ref), "dW rows"
     del hA, hW, hdY, o_af, o_wf, o_dy, o_wb, o_ab
 
     # ---- whole outputs: the element-wise path on the same codes gives the same values, and its
     # int32 sums pass exact Freivalds checks
-    gws = srq.new_workspace(srq.srq_gemm_workspace_bytes(N, K))
+    gws = srq.new_workspace(srq.srq_gemm_workspace_bytes(max(T, N), max(N, K)))
     for name, qa, qb, sa, sb, out in (("Y", g_af, g_wf, s_af, s_wf, Y), ("dA", g_dy, g_wbt, s_dy, s_wb, dA),
-                                      ("dW", g_dyt, g_abt, s_dy, s_ab, dW)):
+                                      ("dW", g_dyt, g_abt, s_dyt, s_ab, dW)):
         acc = torch.empty(out.shape, dtype=torch.int32, device="cuda")
         out2 = torch.empty_like(out)
         srq.srq_gemm_i8(qa, qb, sa, sb, out2, acc, gws)
