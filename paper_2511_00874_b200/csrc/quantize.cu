@@ -591,9 +591,10 @@ quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
 // takes whole rows; each thread holds its 4-element groups of the row in registers (G per thread,
 // groups tid, tid + 256, ...), the row maximum is reduced over the CTA (two barriers per row), the
 // step size is derived exactly as in the two-pass path, and the codes are formed from the registers,
-// so that the input is read once (e + 1 bytes per element instead of 2 e + 1).  The next row's loads
-// are issued before the current row is processed.  Same conditions as the fast path (groups of four
-// line up with the flat index), same arithmetic, same codes.
+// so that the input is read once (e + 1 bytes per element instead of 2 e + 1).  Several CTAs per SM
+// hide one another's load latency (holding the next row in registers as well cost more in occupancy
+// than it gained).  Same conditions as the fast path (groups of four line up with the flat index),
+// same arithmetic, same codes.
 __device__ __forceinline__ uint32_t abs_max4(const float4& q) {
     return max(max(__float_as_uint(q.x) & 0x7FFFFFFFu, __float_as_uint(q.y) & 0x7FFFFFFFu),
                max(__float_as_uint(q.z) & 0x7FFFFFFFu, __float_as_uint(q.w) & 0x7FFFFFFFu));
@@ -615,7 +616,7 @@ quantize_rows_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
     __shared__ float row_inv[2];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t ngroups = (uint32_t)(P.cols >> 2);
-    Raw cur[G], nxt[G];
+    Raw cur[G];
     auto load_row = [&](int64_t r, Raw raw[G]) {
         const Raw* src = reinterpret_cast<const Raw*>(x + r * P.ld);
 #pragma unroll
@@ -625,9 +626,8 @@ quantize_rows_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
         }
     };
     int64_t r = blockIdx.x;
-    if (r < P.rows) load_row(r, cur);
     for (uint32_t it = 0; r < P.rows; r += gridDim.x, ++it) {
-        if (r + gridDim.x < P.rows) load_row(r + gridDim.x, nxt);
+        load_row(r, cur);
         uint32_t m = 0u;
 #pragma unroll
         for (int k = 0; k < G; ++k) m = max(m, abs_max4(cur[k]));
@@ -671,8 +671,6 @@ quantize_rows_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
             const uint32_t g = (uint32_t)tid + (uint32_t)(k * Q_THREADS);
             if (g < ngroups) out[g] = w[k];
         }
-#pragma unroll
-        for (int k = 0; k < G; ++k) cur[k] = nxt[k];
     }
 }
 
