@@ -266,6 +266,13 @@ srq_status_t qlinear_bwd(const void *dY, const void *A, const void *W, srq_dtype
  *   accumulate  1: out += result (one binary32 addition per element) instead of out = result.
  *               The paper emulates large batches by accumulating gradients over micro-batches
  *               (hardware-considerations section); this is that accumulation for dW.
+ *               2: the int32 sums are accumulated instead: acc_out += sums (the call's acc_out /
+ *               dbg->acc matrix is required and holds the running sums; zero it before the first
+ *               micro-batch) and out = float(acc_out) * (s_row * s_col) is written from the total.
+ *               Exact - the result equals one product over the concatenated contraction - as
+ *               long as every micro-batch uses the same step sizes (srq_qspec_t.absmax) and the
+ *               totals fit int32; a wrap is reported as SRQ_ERR_ACC_OVERFLOW by srq_poll_status.
+ *               Integer grid only.
  *   q, step, codes, ld_codes
  *               also write Q(result) as int8 codes [M, ld_codes] for the layer that consumes the
  *               result (the next layer's Q(A_in) of Alg. 1, the previous layer's Q(dA_out) of
@@ -282,7 +289,7 @@ srq_status_t qlinear_bwd(const void *dY, const void *A, const void *W, srq_dtype
  *               float *; its pitch counts bfloat16 elements): each binary32 result is rounded to
  *               the nearest bfloat16, ties to even, as it is stored, which halves the bytes the
  *               product writes.  Codes and absmax still come from the binary32 result.  Not with
- *               accumulate (SRQ_ERR_UNSUPPORTED): running sums stay in binary32.
+ *               accumulate = 1 (SRQ_ERR_UNSUPPORTED): running binary32 sums stay in binary32.
  * Products with q or absmax set are never split along the contraction.
  */
 typedef struct {

@@ -371,7 +371,7 @@ class Output:
     """Output options of a product (srq_output_t): accumulate into out, codes of Q(result) with a
     caller-supplied step (q, step, codes), absmax of the result.  A bfloat16 output tensor passed
     to one of the *_ex calls sets the struct's out_bf16 member."""
-    accumulate: bool = False
+    accumulate: int = 0        # 1 (or True): out += result in binary32; 2: running int32 sums in acc_out
     q: Optional[QSpec] = None
     step: Optional[torch.Tensor] = None
     codes: Optional[torch.Tensor] = None
@@ -432,18 +432,24 @@ def qlinear_fwd_ex(A: torch.Tensor, W: torch.Tensor, qA: QSpec, qW: QSpec, Y: Op
 
 def qlinear_bwd_ex(dY: torch.Tensor, A: torch.Tensor, W: torch.Tensor, qdY: QSpec, qA: QSpec, qW: QSpec,
                    dA: Optional[torch.Tensor], dW: Optional[torch.Tensor], output_dA: Optional[Output] = None,
-                   output_dW: Optional[Output] = None, ws: Optional[torch.Tensor] = None) -> None:
-    """qlinear_bwd with output options for dA and dW."""
+                   output_dW: Optional[Output] = None, ws: Optional[torch.Tensor] = None,
+                   dbg_input: Optional[DebugOut] = None, dbg_weight: Optional[DebugOut] = None) -> None:
+    """qlinear_bwd with output options for dA and dW (dbg_weight.acc holds the running int32 sums of
+    dW when output_dW.accumulate is 2)."""
     T, N = dY.shape
     K = A.shape[1]
     if ws is None:
         ws = new_workspace(srq_workspace_bytes(T, N, K), dY.device)
     c0, c1, c2 = qdY.c(), qA.c(), qW.c()
     o0, o1 = _opt(output_dA, dA), _opt(output_dW, dW)
+    d0 = dbg_input.c() if dbg_input is not None else None
+    d1 = dbg_weight.c() if dbg_weight is not None else None
     st = lib().qlinear_bwd_ex(dY.data_ptr(), A.data_ptr(), W.data_ptr(), _dtype_of(dY), T, N, K,
                               ctypes.byref(c0), ctypes.byref(c1), ctypes.byref(c2), _ptr(dA), _ptr(dW),
                               ctypes.byref(o0) if o0 is not None else None,
-                              ctypes.byref(o1) if o1 is not None else None, None, None,
+                              ctypes.byref(o1) if o1 is not None else None,
+                              ctypes.byref(d0) if d0 is not None else None,
+                              ctypes.byref(d1) if d1 is not None else None,
                               ws.data_ptr(), ws.numel(), _stream())
     _check(st, "qlinear_bwd_ex")
 

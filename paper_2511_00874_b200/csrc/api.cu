@@ -24,10 +24,10 @@ srq_status_t check_qspec(const srq_qspec_t* q) {
 srq_status_t make_out_options(const srq_output_t* o, int64_t N, bool have_out, OutOptions* r) {
     *r = OutOptions();
     if (!o) return have_out ? SRQ_OK : SRQ_ERR_INVALID_ARG;
-    if (o->accumulate != 0 && o->accumulate != 1) return SRQ_ERR_INVALID_ARG;
+    if (o->accumulate < 0 || o->accumulate > 2) return SRQ_ERR_INVALID_ARG;
     if (o->accumulate && !have_out) return SRQ_ERR_INVALID_ARG;
     if (o->out_bf16 != 0 && o->out_bf16 != 1) return SRQ_ERR_INVALID_ARG;
-    if (o->out_bf16 && o->accumulate) return SRQ_ERR_UNSUPPORTED;   // sums are kept in binary32
+    if (o->out_bf16 && o->accumulate == 1) return SRQ_ERR_UNSUPPORTED;   // running binary32 sums stay in binary32
     r->accumulate = o->accumulate;
     r->out_bf16 = o->out_bf16;
     if (o->q) {

@@ -599,7 +599,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0 && wrow < P.M && col0 < P.N) {
-                        if (P.opt.accumulate) tma_reduce_add_2d(&map_out, stage, col0, wrow);   // binary32 adds in memory
+                        if (P.opt.accumulate == 1) tma_reduce_add_2d(&map_out, stage, col0, wrow);   // binary32 adds in memory
                         else tma_store_2d(&map_out, stage, col0, wrow);
                         bulk_commit();
                     }
@@ -618,9 +618,25 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const float* sc = &T->s_col[buf][j * 32];
                         if (P.acc_out) {
                             int32_t* ad = P.acc_out + row * P.N + col0;
+                            if (P.opt.accumulate == 2) {
+                                // running int32 sums over calls (exact while they fit): acc_out += sums, and the
+                                // result below is formed from the total
+                                bool wrapped = false;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (col0 + i < P.N) ad[i] = (int32_t)v[i];
+                                for (int i = 0; i < 32; ++i)
+                                    if (col0 + i < P.N) {
+                                        const int32_t before = ad[i], add = (int32_t)v[i];
+                                        const int32_t total = (int32_t)((uint32_t)before + (uint32_t)add);
+                                        wrapped |= ((before ^ total) & (add ^ total)) < 0;
+                                        ad[i] = total;
+                                        v[i] = (uint32_t)total;
+                                    }
+                                if (wrapped) record_status(P.status, SRQ_ERR_ACC_OVERFLOW);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (col0 + i < P.N) ad[i] = (int32_t)v[i];
+                            }
                         }
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
@@ -638,7 +654,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 for (int q = 0; q < 8; ++q) {
                                     float4 o = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
                                                            __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
-                                    if (P.opt.accumulate) {
+                                    if (P.opt.accumulate == 1) {
                                         const float4 p = *reinterpret_cast<const float4*>(dst + 4 * q);
                                         o.x = __fadd_rn(p.x, o.x); o.y = __fadd_rn(p.y, o.y); o.z = __fadd_rn(p.z, o.z); o.w = __fadd_rn(p.w, o.w);
                                     }
@@ -648,7 +664,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                                 for (int i = 0; i < 32; ++i)
                                     if (col0 + i < P.N)
-                                        dst[i] = P.opt.accumulate ? __fadd_rn(dst[i], __uint_as_float(v[i])) : __uint_as_float(v[i]);
+                                        dst[i] = P.opt.accumulate == 1 ? __fadd_rn(dst[i], __uint_as_float(v[i])) : __uint_as_float(v[i]);
                             }
                         }
                     }
@@ -703,7 +719,7 @@ __global__ void __launch_bounds__(256)
 dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_tile, int32_t tiles_n, int32_t tile_rows,
                int64_t M, int64_t N, const float* __restrict__ s_row, int32_t row_stride,
                const float* __restrict__ s_col, int32_t col_stride, float* __restrict__ out, int64_t ldo,
-               int32_t* __restrict__ acc_out, int vec, int accumulate, int out_bf16) {
+               int32_t* __restrict__ acc_out, int vec, int accumulate, int out_bf16, uint32_t* status) {
     const int64_t per_tile = (int64_t)tile_rows * (BN / 4);
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_tiles * per_tile; g += (int64_t)gridDim.x * blockDim.x) {
         const int64_t t = g / per_tile, in_tile = g % per_tile;
@@ -712,7 +728,15 @@ dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_
         const int64_t c = (tile % tiles_n) * BN + (in_tile % (BN / 4)) * 4;
         if (r >= M || c >= N) continue;
         const int4 a = __ldcg(reinterpret_cast<const int4*>(part + g * 4));
-        const int32_t av[4] = {a.x, a.y, a.z, a.w};
+        int32_t av[4] = {a.x, a.y, a.z, a.w};
+        if (accumulate == 2) {             // running int32 sums over calls: the result is formed from the total
+            for (int e = 0; e < 4 && c + e < N; ++e) {
+                const int32_t before = acc_out[r * N + c + e];
+                const int32_t total = (int32_t)((uint32_t)before + (uint32_t)av[e]);
+                if (((before ^ total) & (av[e] ^ total)) < 0) record_status(status, SRQ_ERR_ACC_OVERFLOW);
+                av[e] = total;
+            }
+        }
         const float sr = s_row[r * row_stride];
         float o[4];
 #pragma unroll
@@ -732,13 +756,13 @@ dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_
         float* dst = out + r * ldo + c;
         if (vec && c + 4 <= N) {
             float4 w = make_float4(o[0], o[1], o[2], o[3]);
-            if (accumulate) {
+            if (accumulate == 1) {
                 const float4 p = *reinterpret_cast<const float4*>(dst);
                 w.x = __fadd_rn(p.x, w.x); w.y = __fadd_rn(p.y, w.y); w.z = __fadd_rn(p.z, w.z); w.w = __fadd_rn(p.w, w.w);
             }
             *reinterpret_cast<float4*>(dst) = w;
         } else {
-            for (int e = 0; e < 4 && c + e < N; ++e) dst[e] = accumulate ? __fadd_rn(dst[e], o[e]) : o[e];
+            for (int e = 0; e < 4 && c + e < N; ++e) dst[e] = accumulate == 1 ? __fadd_rn(dst[e], o[e]) : o[e];
         }
         if (acc_out)
             for (int e = 0; e < 4 && c + e < N; ++e) acc_out[r * N + c + e] = av[e];
@@ -886,6 +910,7 @@ static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, cons
 }
 
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream) {
+    if (g.opt.accumulate == 2 && (g.acc_out == nullptr || g.kind != 0)) return SRQ_ERR_INVALID_ARG;   // int32 sums need their matrix
     if (g.M == 0 || g.N == 0) return SRQ_OK;
     DeviceInfo* dev = nullptr;
     if (!device_info(&dev)) return SRQ_ERR_CUDA;
@@ -954,7 +979,7 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
         const unsigned grid = (unsigned)(blocks < 8 * (int64_t)dev->sms ? blocks : 8 * (int64_t)dev->sms);
         dequant_kernel<<<grid, 256, 0, stream>>>(P.part, split_tiles, P.full_tiles, P.tiles_n, BM * ctas, g.M, g.N, g.s_row,
                                                  g.row_stride, g.s_col, g.col_stride, g.out, g.ldo, g.acc_out, vec,
-                                                 g.opt.accumulate, g.opt.out_bf16);
+                                                 g.opt.accumulate, g.opt.out_bf16, status);
         ++g_launches;
         if (cudaGetLastError() != cudaSuccess) return SRQ_ERR_CUDA;
     }

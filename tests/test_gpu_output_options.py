@@ -192,3 +192,59 @@ def test_bfloat16_output_cannot_accumulate():
     with pytest.raises(srq.SrqError) as e:
         srq.srq_gemm_i8_ex(a, b, s, s, out, srq.Output(accumulate=True))
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("M,N,Kc", [(300, 520, 384), (64, 256, 4096)])
+def test_int32_accumulation_over_micro_batches_equals_the_product_over_all_of_them(M, N, Kc):
+    """accumulate = 2: the raw sums of three micro-batches are added in int32 and the output is formed
+    from the total, which is the product over the concatenated contraction, exactly (same step
+    sizes for every micro-batch).  The second shape runs the split contraction, whose finishing
+    pass does the adding.  A total that does not fit int32 is reported."""
+    parts_a = [_codes(M, Kc, 10 + i) for i in range(3)]
+    parts_b = [_codes(N, Kc, 20 + i) for i in range(3)]
+    s_row = (torch.rand(M) * 0.02 + 1e-3).cuda()
+    s_col = (torch.rand(1) * 0.02 + 1e-3).cuda()
+    acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    out = torch.full((M, N), float("nan"), device="cuda")
+    ws = srq.new_workspace(srq.srq_gemm_workspace_bytes(M, N))
+    for a, b in zip(parts_a, parts_b):
+        srq.srq_gemm_i8_ex(a, b, s_row, s_col, out, srq.Output(accumulate=2), acc, ws)
+        assert srq.srq_poll_status(ws) == 0
+    ref_acc = oracle.gemm_i8_nt(np.concatenate([a.cpu().numpy() for a in parts_a], 1), np.concatenate([b.cpu().numpy() for b in parts_b], 1))
+    assert np.array_equal(acc.cpu().numpy(), ref_acc)
+    assert np.array_equal(out.cpu().numpy(), oracle.dequant(ref_acc, s_row.cpu().numpy(), s_col.cpu().numpy()))
+    # running sums need their matrix
+    with pytest.raises(srq.SrqError) as e:
+        srq.srq_gemm_i8_ex(parts_a[0], parts_b[0], s_row, s_col, out, srq.Output(accumulate=2), None, ws)
+    assert e.value.status == 1
+    # a total beyond int32 wraps and is reported
+    acc.fill_(2 ** 31 - 5)
+    ones_a = torch.ones((M, 16), dtype=torch.int8, device="cuda")
+    ones_b = torch.ones((N, 16), dtype=torch.int8, device="cuda")
+    srq.srq_gemm_i8_ex(ones_a, ones_b, s_row, s_col, out, srq.Output(accumulate=2), acc, ws)
+    assert srq.srq_poll_status(ws) == 4
+
+
+def test_layer_weight_gradient_accumulated_in_int32():
+    """qlinear_bwd_ex with accumulate = 2 for dW and shared step sizes (srq_qspec_t.absmax of the
+    whole batch): two micro-batches give the int32 sums, and dW, of one pass over all tokens."""
+    T, N, K = 264, 136, 200
+    A, W, dY = synth.layer_inputs(T, N, K, seed=8, device="cuda", std_dy=1e-3)
+    mA, mdY = torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
+    srq.srq_absmax(A, mA)
+    srq.srq_absmax(dY, mdY)
+    f = lambda t: t.cpu().numpy()
+    ref = oracle.qlinear_bwd_weight(f(dY), f(A), oracle.QSpec(8, 0, 0, 2, 4), oracle.QSpec(8, 0, 0, 2, 2))
+    acc = torch.zeros((N, K), dtype=torch.int32, device="cuda")
+    dW = torch.empty((N, K), device="cuda")
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
+    for lo, hi in ((0, 128), (128, T)):
+        qdy = srq.QSpec(8, 0, 0, 2, 4, index_offset=lo * N, absmax=mdY)
+        qa = srq.QSpec(8, 0, 0, 2, 2, index_offset=lo * K, absmax=mA)
+        dbg = srq.DebugOut(None, None, None, None, acc)
+        dA = torch.empty((hi - lo, K), device="cuda")
+        srq.qlinear_bwd_ex(dY[lo:hi].contiguous(), A[lo:hi].contiguous(), W, qdy, qa, srq.QSpec(8, 0, 0, 2, 3), dA, dW,
+                           None, srq.Output(accumulate=2), ws, dbg_weight=dbg)
+        assert srq.srq_poll_status(ws) == 0
+    assert np.array_equal(acc.cpu().numpy(), ref.acc)
+    assert np.array_equal(dW.cpu().numpy(), ref.out)
