@@ -270,3 +270,19 @@ def test_token_shards_with_per_row_steps_share_their_column_maxima(dtype, shape)
         assert np.array_equal(dbg.scale_a.cpu().numpy(), ref.scale_a) and np.array_equal(dbg.scale_b.cpu().numpy(), ref.scale_b)
         total += acc.cpu().numpy()
     assert np.array_equal(total, ref.acc.astype(np.int64))
+
+
+def test_one_pass_per_row_path_reports_nonfinite_input():
+    x = synth.normal((40, 1024), 1.0, seed=5, device="cuda")
+    x[7, 900] = float("nan")
+    ws = srq.new_workspace(srq.srq_quantize_workspace_bytes(40, 1024))
+    c = torch.empty((40, 1024), dtype=torch.int8, device="cuda")
+    s = torch.empty(40, device="cuda")
+    srq.sr_quantize(x, srq.QSpec(scale=srq.PER_ROW), c, s, ws=ws)
+    assert srq.srq_poll_status(ws) == 6
+    x[7, 900] = float("-inf")
+    srq.sr_quantize(x, srq.QSpec(scale=srq.PER_ROW, round=srq.RTN), c, s, ws=ws)
+    assert srq.srq_poll_status(ws) == 6
+    x[7, 900] = 0.5
+    srq.sr_quantize(x, srq.QSpec(scale=srq.PER_ROW), c, s, ws=ws)
+    assert srq.srq_poll_status(ws) == 0
