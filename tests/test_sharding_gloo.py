@@ -90,3 +90,65 @@ def test_token_shards_reproduce_the_unsharded_layer():
         p.join(120)
         assert p.exitcode == 0
     assert out.get(timeout=5) == []
+
+
+def _worker_per_row(rank, world, port, out):
+    """Per-row step sizes: the operands of dW are scaled per column of dY / A, i.e. over the tokens.
+    Each rank finds the column maxima of its shard, the ranks max-reduce them, and every rank
+    quantizes with the reduced maxima (handed to the oracle as one extra row holding them, which
+    makes its own column maxima the global ones; that row's codes are dropped)."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        A, W, dY = _inputs()
+        rows = T // world
+        r0 = rank * rows
+        a, dy = A[r0:r0 + rows], dY[r0:r0 + rows]
+        col_a = torch.from_numpy(np.abs(a).max(axis=0))
+        col_dy = torch.from_numpy(np.abs(dy).max(axis=0))
+        dist.all_reduce(col_a, op=dist.ReduceOp.MAX)
+        dist.all_reduce(col_dy, op=dist.ReduceOp.MAX)
+        from oracle import PER_ROW
+        qa = QSpec(8, PER_ROW, SR, 11, 2, index_offset=r0 * K)
+        qdy = QSpec(8, PER_ROW, SR, 11, 4, index_offset=r0 * N)
+        # transposed layouts of the shard with the reduced maxima
+        _, _, ca, sa = oracle.sr_quantize(np.concatenate([a, col_a.numpy()[None, :]], 0), qa, False, True)
+        _, _, cdy, sdy = oracle.sr_quantize(np.concatenate([dy, col_dy.numpy()[None, :]], 0), qdy, False, True)
+        ca, cdy = ca[:, :rows], cdy[:, :rows]
+        acc = torch.from_numpy(oracle.gemm_i8_nt(cdy, ca).copy())
+        dist.all_reduce(acc)
+        gathered = [None] * world
+        dist.gather_object((ca, cdy, sa, sdy, col_a.numpy(), col_dy.numpy()), gathered if rank == 0 else None)
+        if rank == 0:
+            full = oracle.qlinear_bwd_weight(dY, A, QSpec(8, PER_ROW, SR, 11, 4), QSpec(8, PER_ROW, SR, 11, 2))
+            bad = []
+            if not (np.array_equal(gathered[0][4], np.abs(A).max(axis=0)) and np.array_equal(gathered[0][5], np.abs(dY).max(axis=0))):
+                bad.append("max-reduced column maxima")
+            if not np.array_equal(np.concatenate([g[1] for g in gathered], axis=1), full.codes_a):
+                bad.append("codes of dY^T [N, T]")
+            if not np.array_equal(np.concatenate([g[0] for g in gathered], axis=1), full.codes_b):
+                bad.append("codes of A^T [K, T]")
+            if not all(np.array_equal(g[3], full.scale_a) and np.array_equal(g[2], full.scale_b) for g in gathered):
+                bad.append("column step sizes")
+            if not np.array_equal(acc.numpy(), full.acc):
+                bad.append("all-reduced int32 sums of dW")
+            out.put(bad)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_token_shards_with_per_row_steps_exchange_column_maxima():
+    oracle.build()
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_worker_per_row, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    assert out.get(timeout=5) == []
