@@ -18,18 +18,19 @@
  *     device memory and keeps no state between calls.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL
  *     for the default stream) and the call returns without waiting.
- *   - Errors the host can see (null pointer, bits outside 2..8, a pitch or
+ *   - Errors the host can see (null pointer, bits outside the grid's range, a pitch or
  *     pointer that breaks the alignment rules below, workspace too small,
  *     a contraction long enough to overflow int32) return a status at once
  *     and enqueue nothing.  Conditions only the device can see (an input
  *     that is not finite, a bounded wait inside a kernel that ran out) are
  *     recorded in a status word at the start of the workspace; read it with
  *     srq_poll_status.  After such a condition the outputs are unspecified.
- *   - Outputs are overwritten, never accumulated into.
- *   - Both operands of a layer pass use the same grid (srq_qspec_t.format).  With the E4M3
- *     grid the codes are E4M3 bytes, D_g = absmax_g / 448, the products run in kind::f8f6f4
- *     with binary32 accumulation, and the `acc` member of the debug struct receives binary32
- *     sums (same size as int32).
+ *   - Outputs are overwritten, unless a srq_output_t (the *_ex entry points) asks for accumulation.
+ *   - Both operands of a layer pass use the same grid (srq_qspec_t.format).  With the
+ *     floating-point grid (E4M3, or E4M2 / E4M1 / E4M0 by `bits`) the codes are E4M3 bytes,
+ *     D_g = absmax_g / (largest value of the grid: 448, 448, 384, 256), the products run in
+ *     kind::f8f6f4 with binary32 accumulation, and the `acc` member of the debug struct receives
+ *     binary32 sums (same size as int32).
  *   - Alignment: input base pointers 16-byte aligned; input pitch `ld` in
  *     elements; fp32 outputs 16-byte aligned; the workspace 256-byte aligned.
  *     Inputs whose pitch or extent is not a multiple of 4 elements take a
@@ -64,7 +65,7 @@ extern "C" {
 typedef enum {
     SRQ_OK = 0,
     SRQ_ERR_INVALID_ARG = 1,   /* null pointer, bad enum, bad extent, misaligned pointer/pitch */
-    SRQ_ERR_UNSUPPORTED = 2,   /* bits outside 2..8 */
+    SRQ_ERR_UNSUPPORTED = 2,   /* bits outside 2..8 (5..8 on the floating-point grid); options that do not combine */
     SRQ_ERR_WORKSPACE = 3,     /* workspace smaller than srq_*_workspace_bytes says */
     SRQ_ERR_ACC_OVERFLOW = 4,  /* contraction length * qmax_a * qmax_b >= 2^31 */
     SRQ_ERR_CUDA = 5,          /* a CUDA call failed (launch, tensor-map encode, copy) */
