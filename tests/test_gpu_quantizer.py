@@ -286,3 +286,31 @@ def test_one_pass_per_row_path_reports_nonfinite_input():
     x[7, 900] = 0.5
     srq.sr_quantize(x, srq.QSpec(scale=srq.PER_ROW), c, s, ws=ws)
     assert srq.srq_poll_status(ws) == 0
+
+
+@pytest.mark.parametrize("case", range(32))
+def test_random_shapes_pitches_offsets_and_modes(case):
+    """Seeded random cases over extents (ragged and aligned, rows long enough for the one-pass per-row
+    kernel included), input pitches, index offsets, widths, grids of modes and layouts."""
+    rng = np.random.default_rng(1000 + case)
+    rows = int(rng.integers(1, 260))
+    cols = int(rng.choice([rng.integers(1, 200), rng.integers(500, 1200), 4 * rng.integers(128, 300), 1024, 2048]))
+    ld = cols + int(rng.choice([0, 0, 4, 8, 3]))
+    dtype = [torch.float32, torch.bfloat16][int(rng.integers(2))]
+    scale = [srq.PER_TENSOR, srq.PER_ROW][int(rng.integers(2))]
+    rnd = [srq.SR, srq.RTN, srq.SR8][int(rng.integers(3))]
+    bits = int(rng.integers(2, 9))
+    off = int(rng.choice([0, 4, 16, 5, 2 ** 32 - 8, 2 ** 35 + 12]))
+    want_rm, want_tr = [(True, True), (True, False), (False, True)][int(rng.integers(3))]
+    base = synth.with_outliers((rows, ld), seed=case, dtype=dtype, device="cuda")
+    x = base[:, :cols]
+    if case % 5 == 0:
+        x[rows // 2] = 0
+    q = srq.QSpec(bits, scale, rnd, seed=case, tensor_id=2 ** 32 + case, index_offset=off)
+    got = _run_gpu(x, q, want_rm, want_tr, pad_rm=int(rng.choice([0, 4, 7])), pad_tr=int(rng.choice([0, 4, 5])))
+    ref = oracle.sr_quantize(x.float().cpu().numpy(), oracle.QSpec(bits, scale, rnd, case, 2 ** 32 + case, off), want_rm, want_tr)
+    for name, g, r in zip(("codes_rm", "scale_rm", "codes_tr", "scale_tr"), got, ref):
+        if r is None:
+            continue
+        bad = np.argwhere(g != r)
+        assert bad.size == 0, f"{name}: {len(bad)} mismatches, first at {bad[0]} ({rows}x{cols}, ld {ld}, {dtype}, scale {scale}, round {rnd}, bits {bits}, off {off})"
