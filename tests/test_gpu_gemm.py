@@ -170,3 +170,38 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
     one = torch.ones(1, device="cuda")
     out, acc = _run(a, b, one, one)
     assert np.array_equal(acc, oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy()))
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_products(case):
+    """Seeded random products: extents from one element to several tiles (one-CTA and CTA-pair
+    tiles, split and unsplit contractions), output pitches, per-tensor and per-row step sizes,
+    fp32 or bfloat16 results, with and without the raw sums."""
+    rng = np.random.default_rng(500 + case)
+    M = int(rng.choice([rng.integers(1, 129), rng.integers(129, 700), 256, 512]))
+    N = int(rng.choice([rng.integers(1, 300), rng.integers(300, 800), 256, 768]))
+    Kc = int(rng.choice([rng.integers(1, 300), 16 * rng.integers(8, 400), 4096]))
+    a, b = _codes(M, Kc, 2 * case), _codes(N, Kc, 2 * case + 1)
+    per_row = bool(rng.integers(2))
+    s_row = (torch.rand(M if per_row else 1) * 0.1 + 1e-3).cuda()
+    s_col = (torch.rand(N if per_row else 1) * 0.1 + 1e-3).cuda()
+    bf16 = bool(rng.integers(2))
+    want_acc = bool(rng.integers(2))
+    pad = int(rng.choice([0, 0, 8, 3]))
+    full = torch.full((M, N + pad), 7.0, dtype=torch.bfloat16 if bf16 else torch.float32, device="cuda")
+    out = full[:, :N]
+    acc = torch.full((M, N), -1, dtype=torch.int32, device="cuda") if want_acc else None
+    ws = srq.new_workspace(srq.srq_gemm_workspace_bytes(M, N))
+    srq.srq_gemm_i8_ex(a, b, s_row, s_col, out, None, acc, ws)
+    assert srq.srq_poll_status(ws) == 0
+    ref_acc = oracle.gemm_i8_nt(a.cpu().numpy(), b.cpu().numpy())
+    ref = oracle.dequant(ref_acc, s_row.cpu().numpy(), s_col.cpu().numpy())
+    tag = f"M {M} N {N} Kc {Kc} per_row {per_row} bf16 {bf16} acc {want_acc} pad {pad}"
+    if want_acc:
+        assert np.array_equal(acc.cpu().numpy(), ref_acc), tag
+    if bf16:
+        assert np.array_equal(out.contiguous().view(torch.uint16).cpu().numpy(), oracle.to_bf16(ref)), tag
+    else:
+        assert np.array_equal(out.cpu().numpy(), ref), tag
+    if pad:
+        assert bool((full[:, N:] == 7.0).all()), tag + ": pad columns written"
