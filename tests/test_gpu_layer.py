@@ -180,3 +180,19 @@ def test_layer_with_eight_random_bits_per_element():
     T, N, K = 264, 400, 336
     A, W, dY = synth.layer_inputs(T, N, K, seed=6, device="cuda", std_dy=1e-3)
     all_passes(A, W, dY, layer_specs(srq.PER_TENSOR, srq.SR8, seed=4, bits_fwd=8, bits_bwd=4))
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_layers(case):
+    """Seeded random layers: extents (aligned and odd, rows long enough for the one-pass per-row
+    quantizer included), input type, step-size mode, rounding mode, forward and backward widths."""
+    rng = np.random.default_rng(300 + case)
+    T = int(rng.choice([rng.integers(1, 300), 8 * rng.integers(4, 60)]))
+    N = int(rng.choice([rng.integers(1, 300), 8 * rng.integers(4, 60)]))
+    K = int(rng.choice([rng.integers(1, 300), 8 * rng.integers(4, 60), 1024]))
+    dtype = [torch.float32, torch.bfloat16][int(rng.integers(2))]
+    scale = [srq.PER_TENSOR, srq.PER_ROW][int(rng.integers(2))]
+    rnd = [srq.SR, srq.RTN, srq.SR8][int(rng.integers(3))]
+    A, W, dY = synth.layer_inputs(T, N, K, seed=case, dtype=dtype, device="cuda", std_dy=1e-3)
+    q = layer_specs(scale, rnd, seed=case, bits_fwd=int(rng.integers(3, 9)), bits_bwd=int(rng.integers(2, 9)))
+    all_passes(A, W, dY, q)
