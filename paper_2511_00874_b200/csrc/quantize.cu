@@ -674,6 +674,79 @@ quantize_rows_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
     }
 }
 
+// The same one-pass scheme with a WARP per row, for rows short enough that a lane can hold its share
+// in registers (GW groups of four elements per lane, groups lane, lane + 32, ...): no barriers at all,
+// the row maximum is one warp reduction and every lane derives the step size itself, so the warps of
+// an SM run independently and hide one another's load latency.
+template <typename T, int MODE, int GW>
+__global__ void __launch_bounds__(Q_THREADS)
+quantize_rows_warp_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P, float* __restrict__ delta_out,
+                          float qmax, uint32_t* status) {
+    using Raw = typename Raw4<T>::type;
+    constexpr bool SRM = (MODE & MODE_SR) != 0;
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (Q_THREADS / 32);
+    const uint32_t ngroups = (uint32_t)(P.cols >> 2);
+    for (int64_t r = (int64_t)blockIdx.x * (Q_THREADS / 32) + (threadIdx.x >> 5); r < P.rows; r += warps) {
+        const Raw* src = reinterpret_cast<const Raw*>(x + r * P.ld);
+        Raw cur[GW];
+#pragma unroll
+        for (int k = 0; k < GW; ++k) {
+            const uint32_t g = (uint32_t)lane + 32u * k;
+            cur[k] = g < ngroups ? __ldcs(src + g) : Raw{};
+        }
+        uint32_t m = 0u;
+#pragma unroll
+        for (int k = 0; k < GW; ++k) m = max(m, abs_max4(cur[k]));
+        m = __reduce_max_sync(0xFFFFFFFFu, m);
+        float delta, inv;
+        scale_from_bits(m, qmax, &delta, &inv, status);
+        if (lane == 0 && delta_out) delta_out[r] = delta;
+        const uint64_t jb = (P.index_offset + (uint64_t)r * (uint64_t)P.cols) >> 2;
+        uint32_t* out = reinterpret_cast<uint32_t*>(P.codes_rm + r * P.ld_rm);
+#pragma unroll
+        for (int k = 0; k < GW; ++k) {
+            const uint32_t g = (uint32_t)lane + 32u * k;
+            float v[4];
+            widen(cur[k], v);
+            uint32_t rnd[4] = {0u, 0u, 0u, 0u};
+            if constexpr (SRM) {
+                const uint32_t lo = (uint32_t)jb + g;
+                philox_rounds(lo, (uint32_t)(jb >> 32) + (lo < g ? 1u : 0u), P.keys, rnd);
+            }
+            const uint32_t w = quantize4<MODE>(v, inv, inv, inv, inv, rnd, P.e4m_shift);
+            if (g < ngroups) out[g] = w;
+        }
+    }
+}
+
+template <typename T, int MODE, int GW>
+static void launch_rows_warp_one(const T* p, const QuantParams& P, float* delta_out, float qmax, uint32_t* status,
+                                 int sms, cudaStream_t st) {
+    static int per_sm = 0;
+    if (per_sm == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_rows_warp_kernel<T, MODE, GW>, Q_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+        per_sm = n;
+    }
+    const int64_t resident = (int64_t)sms * per_sm;
+    const int64_t need = (P.rows + Q_THREADS / 32 - 1) / (Q_THREADS / 32);
+    quantize_rows_warp_kernel<T, MODE, GW><<<(unsigned)(need < resident ? need : resident), Q_THREADS, 0, st>>>(p, P, delta_out, qmax, status);
+}
+
+// Groups per lane a warp may hold: 64 data registers at most.
+template <typename T> constexpr int rows_warp_max_groups() { return sizeof(T) == 4 ? 16 : 32; }
+
+template <typename T, int MODE>
+static void launch_rows_warp_g(int gw, const void* x, const QuantParams& P, float* delta_out, float qmax, uint32_t* status,
+                               int sms, cudaStream_t st) {
+    const T* p = (const T*)x;
+    if (gw <= 4) launch_rows_warp_one<T, MODE, 4>(p, P, delta_out, qmax, status, sms, st);
+    else if (gw <= 8) launch_rows_warp_one<T, MODE, 8>(p, P, delta_out, qmax, status, sms, st);
+    else if (gw <= 16) launch_rows_warp_one<T, MODE, 16>(p, P, delta_out, qmax, status, sms, st);
+    else if constexpr (rows_warp_max_groups<T>() >= 32) launch_rows_warp_one<T, MODE, 32>(p, P, delta_out, qmax, status, sms, st);
+}
+
 // One wave of CTAs: as many as are resident at once (asked once per kernel), at most one per row.
 template <typename T, int MODE, int G>
 static void launch_rows_one(const T* p, const QuantParams& P, float* delta_out, float qmax, uint32_t* status,
@@ -702,6 +775,17 @@ static void launch_rows_g(int g, const void* x, const QuantParams& P, float* del
 static void launch_rows(srq_dtype_t dt, int mode, const void* x, const QuantParams& P, float* delta_out, float qmax,
                         uint32_t* status, int sms, cudaStream_t st) {
     const int g = (int)(((P.cols >> 2) + Q_THREADS - 1) / Q_THREADS);
+    const int gw = (int)(((P.cols >> 2) + 31) / 32);          // groups per lane with a warp per row
+#define SRQ_ROWS_WARP(T)                                                                          \
+    switch (mode) {                                                                               \
+        case 0: launch_rows_warp_g<T, 0>(gw, x, P, delta_out, qmax, status, sms, st); break;      \
+        case 1: launch_rows_warp_g<T, 1>(gw, x, P, delta_out, qmax, status, sms, st); break;      \
+        case 2: launch_rows_warp_g<T, 2>(gw, x, P, delta_out, qmax, status, sms, st); break;      \
+        default: launch_rows_warp_g<T, 3>(gw, x, P, delta_out, qmax, status, sms, st); break;     \
+    }
+    if (dt == SRQ_F32 && gw <= rows_warp_max_groups<float>()) { SRQ_ROWS_WARP(float) return; }
+    if (dt != SRQ_F32 && gw <= rows_warp_max_groups<__nv_bfloat16>()) { SRQ_ROWS_WARP(__nv_bfloat16) return; }
+#undef SRQ_ROWS_WARP
 #define SRQ_ROWS(T)                                                                          \
     switch (mode) {                                                                          \
         case 0: launch_rows_g<T, 0>(g, x, P, delta_out, qmax, status, sms, st);  break;      \
