@@ -28,7 +28,7 @@ T_FULL, N_FULL, K_FULL = 65536, 4096, 4096
 
 # DRAM bytes (read + write) of one gemm_i8_kernel launch of this workload, from the ncu capture
 # summarised in profiles/gemm_i8_kernel_M8192_N4096_K4096.md (its bench-size section).
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = 1326607104   # forward-shaped launch, M=65536 N=4096 K=4096
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 1338072320   # forward-shaped launch, M=65536 N=4096 K=4096
 
 
 def layer_ops(T, N, K):

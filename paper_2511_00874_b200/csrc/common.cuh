@@ -21,6 +21,28 @@ __host__ __device__ inline size_t align_up(size_t v, size_t a = kAlign) { return
 
 extern unsigned long long g_launches;   // kernels launched by this process (host counter)
 
+// Programmatic dependent launch.  Every kernel of the library waits for the results of the work before
+// it as its first act (griddepcontrol.wait returns once the preceding grids have finished and their
+// writes are visible; it returns at once for a kernel launched the ordinary way) and then lets the
+// kernel after it be launched, so that the successor's launch and start-up overlap this kernel's
+// execution instead of following it.  Nothing is read or written before the wait, so the order of the
+// stream is kept; a kernel two places ahead has finished as well, because the one in between only
+// finishes after its own wait.
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ void record_status(uint32_t* status, uint32_t code) {
     atomicCAS(status, 0u, code);
 }

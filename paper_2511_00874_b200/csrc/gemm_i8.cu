@@ -362,6 +362,7 @@ template <int CTAS, int KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_part, const GemmParams P) {
+    pdl_enter();
     using C = Cfg<CTAS>;
     constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES;
     using Tail = SharedTail<STAGES>;
@@ -720,6 +721,7 @@ dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_
                int64_t M, int64_t N, const float* __restrict__ s_row, int32_t row_stride,
                const float* __restrict__ s_col, int32_t col_stride, float* __restrict__ out, int64_t ldo,
                int32_t* __restrict__ acc_out, int vec, int accumulate, int out_bf16, uint32_t* status) {
+    pdl_enter();
     const int64_t per_tile = (int64_t)tile_rows * (BN / 4);
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_tiles * per_tile; g += (int64_t)gridDim.x * blockDim.x) {
         const int64_t t = g / per_tile, in_tile = g % per_tile;
@@ -903,9 +905,10 @@ static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, cons
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(groups * CTAS); cfg.blockDim = dim3(GEMM_THREADS);
     cfg.dynamicSmemBytes = gemm_smem<CTAS>(); cfg.stream = stream;
-    cudaLaunchAttribute at;
-    at.id = cudaLaunchAttributeClusterDimension; at.val.clusterDim.x = CTAS; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
-    cfg.attrs = &at; cfg.numAttrs = 1;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = CTAS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization; at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, gemm_i8_kernel<CTAS, KIND>, map_a, map_b, map_out, map_part, P);
 }
 
@@ -977,7 +980,7 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
         const int64_t work = split_tiles * BM * ctas * (BN / 4);
         const int64_t blocks = (work + 255) / 256;
         const unsigned grid = (unsigned)(blocks < 8 * (int64_t)dev->sms ? blocks : 8 * (int64_t)dev->sms);
-        dequant_kernel<<<grid, 256, 0, stream>>>(P.part, split_tiles, P.full_tiles, P.tiles_n, BM * ctas, g.M, g.N, g.s_row,
+        launch_pdl(dequant_kernel, dim3(grid), dim3(256), 0, stream, P.part, split_tiles, P.full_tiles, P.tiles_n, BM * ctas, g.M, g.N, g.s_row,
                                                  g.row_stride, g.s_col, g.col_stride, g.out, g.ldo, g.acc_out, vec,
                                                  g.opt.accumulate, g.opt.out_bf16, status);
         ++g_launches;

@@ -129,6 +129,7 @@ template <typename T, bool ROWS, bool COLS>
 __global__ void __launch_bounds__(AMAX_THREADS, COLS ? 3 : 4)
 amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok,
             uint32_t* __restrict__ amax_rm, uint32_t* __restrict__ amax_tr, const ScaleStep S) {
+    pdl_enter();
     constexpr int EPL = 16 / (int)sizeof(T);                   // elements per 16-byte group
     constexpr int TILE_C = 32 * AMAX_GROUPS * EPL;
     __shared__ uint32_t col_max[COLS ? TILE_C : 1];
@@ -245,10 +246,10 @@ static void launch_amax(const void* x, int64_t rows, int64_t cols, int64_t ld, u
     constexpr int tile_c = 32 * AMAX_GROUPS * (16 / (int)sizeof(T));
     const unsigned grid = (unsigned)(((cols + tile_c - 1) / tile_c) * ((rows + AMAX_TILE_R - 1) / AMAX_TILE_R));
     const bool vec_ok = ((uintptr_t)x % 16 == 0) && ((ld * (int64_t)sizeof(T)) % 16 == 0);
-    if (want_rows && want_cols) amax_kernel<T, true, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
-    else if (want_rows) amax_kernel<T, true, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
-    else if (want_cols) amax_kernel<T, false, true><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
-    else amax_kernel<T, false, false><<<grid, AMAX_THREADS, 0, st>>>(p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
+    if (want_rows && want_cols) launch_pdl(amax_kernel<T, true, true>, dim3(grid), dim3(AMAX_THREADS), 0, st, p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
+    else if (want_rows) launch_pdl(amax_kernel<T, true, false>, dim3(grid), dim3(AMAX_THREADS), 0, st, p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
+    else if (want_cols) launch_pdl(amax_kernel<T, false, true>, dim3(grid), dim3(AMAX_THREADS), 0, st, p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
+    else launch_pdl(amax_kernel<T, false, false>, dim3(grid), dim3(AMAX_THREADS), 0, st, p, rows, cols, ld, vec_ok, amax_rm, amax_tr, S);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -258,6 +259,7 @@ static void launch_amax(const void* x, int64_t rows, int64_t cols, int64_t ld, u
 __global__ void scales_kernel(const uint32_t* amax_rm, int64_t n_rm, float* inv_rm, float* delta_rm,
                               const uint32_t* amax_tr, int64_t n_tr, float* inv_tr, float* delta_tr,
                               float qmax, uint32_t* status) {
+    pdl_enter();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n_rm) {
         float d, r;
@@ -572,6 +574,7 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
 template <typename T, int MODE, int LAYOUT, bool PER_ROW>
 __global__ void __launch_bounds__(Q_THREADS)
 quantize_fast_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P) {
+    pdl_enter();
     __shared__ uint32_t tileT[(LAYOUT & 2) ? Q_TILE * (Q_TILE / 4) : 1];
     const int64_t n_tc = (P.cols + Q_TILE - 1) / Q_TILE;
     const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * Q_TILE;
@@ -610,6 +613,7 @@ template <typename T, int MODE, int G>
 __global__ void __launch_bounds__(Q_THREADS)
 quantize_rows_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P, float* __restrict__ delta_out,
                      float qmax, uint32_t* status) {
+    pdl_enter();
     using Raw = typename Raw4<T>::type;
     constexpr bool SRM = (MODE & MODE_SR) != 0;
     __shared__ uint32_t warp_max[2][Q_THREADS / 32];
@@ -682,6 +686,7 @@ template <typename T, int MODE, int GW>
 __global__ void __launch_bounds__(Q_THREADS)
 quantize_rows_warp_kernel(const T* __restrict__ x, const __grid_constant__ QuantParams P, float* __restrict__ delta_out,
                           float qmax, uint32_t* status) {
+    pdl_enter();
     using Raw = typename Raw4<T>::type;
     constexpr bool SRM = (MODE & MODE_SR) != 0;
     const int lane = threadIdx.x & 31;
@@ -731,7 +736,7 @@ static void launch_rows_warp_one(const T* p, const QuantParams& P, float* delta_
     }
     const int64_t resident = (int64_t)sms * per_sm;
     const int64_t need = (P.rows + Q_THREADS / 32 - 1) / (Q_THREADS / 32);
-    quantize_rows_warp_kernel<T, MODE, GW><<<(unsigned)(need < resident ? need : resident), Q_THREADS, 0, st>>>(p, P, delta_out, qmax, status);
+    launch_pdl(quantize_rows_warp_kernel<T, MODE, GW>, dim3((unsigned)(need < resident ? need : resident)), dim3(Q_THREADS), 0, st, p, P, delta_out, qmax, status);
 }
 
 // Groups per lane a warp may hold: 64 data registers at most.
@@ -759,7 +764,7 @@ static void launch_rows_one(const T* p, const QuantParams& P, float* delta_out, 
     }
     const int64_t resident = (int64_t)sms * per_sm;
     const unsigned grid = (unsigned)(P.rows < resident ? P.rows : resident);
-    quantize_rows_kernel<T, MODE, G><<<grid, Q_THREADS, 0, st>>>(p, P, delta_out, qmax, status);
+    launch_pdl(quantize_rows_kernel<T, MODE, G>, dim3(grid), dim3(Q_THREADS), 0, st, p, P, delta_out, qmax, status);
 }
 
 template <typename T, int MODE>
@@ -802,6 +807,7 @@ static void launch_rows(srq_dtype_t dt, int mode, const void* x, const QuantPara
 template <typename T>
 __global__ void __launch_bounds__(Q_THREADS)
 quantize_kernel(const T* __restrict__ x, const QuantParams P) {
+    pdl_enter();
     // transposed tile: column c of the tile holds 128 row codes = 32 words; the word index is
     // XOR-ed with (c >> 2) & 31 so that both the column-wise writes and the row-wise reads
     // touch 32 different banks.
@@ -883,8 +889,8 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
 // ------------------------------------------------------------------------------------------
 template <typename T, int MODE, int LAYOUT>
 static void launch_fast_pr(bool per_row, const void* x, const QuantParams& P, unsigned grid, cudaStream_t st) {
-    if (per_row) quantize_fast_kernel<T, MODE, LAYOUT, true><<<grid, Q_THREADS, 0, st>>>((const T*)x, P);
-    else quantize_fast_kernel<T, MODE, LAYOUT, false><<<grid, Q_THREADS, 0, st>>>((const T*)x, P);
+    if (per_row) launch_pdl(quantize_fast_kernel<T, MODE, LAYOUT, true>, dim3(grid), dim3(Q_THREADS), 0, st, (const T*)x, P);
+    else launch_pdl(quantize_fast_kernel<T, MODE, LAYOUT, false>, dim3(grid), dim3(Q_THREADS), 0, st, (const T*)x, P);
 }
 template <typename T, int MODE>
 static void launch_fast_layout(int layout, bool per_row, const void* x, const QuantParams& P, unsigned grid, cudaStream_t st) {
@@ -912,6 +918,7 @@ static void launch_fast(srq_dtype_t dt, int mode, int layout, bool per_row, cons
 // of unquantized bfloat16 activations with a quantized weight.  Also writes 1.0f to *one.
 __global__ void widen_codes_kernel(const int8_t* __restrict__ codes, int64_t rows, int64_t cols, int64_t ld,
                                    uint16_t* __restrict__ out, int64_t ld_out, float* one) {
+    pdl_enter();
     if (blockIdx.x == 0 && threadIdx.x == 0) *one = 1.0f;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < rows * cols; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t r = i / cols, c = i % cols;
@@ -923,7 +930,7 @@ cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, 
                                float* one, cudaStream_t stream) {
     const int64_t n = rows * cols;
     const unsigned grid = (unsigned)(n / 256 + 1 < 4096 ? n / 256 + 1 : 4096);
-    widen_codes_kernel<<<grid, 256, 0, stream>>>(codes, rows, cols, ld, (uint16_t*)out_bf16, ld_out, one);
+    launch_pdl(widen_codes_kernel, dim3(grid), dim3(256), 0, stream, codes, rows, cols, ld, (uint16_t*)out_bf16, ld_out, one);
     ++g_launches;
     return cudaGetLastError();
 }
@@ -1031,14 +1038,14 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         }
         const uint32_t* col_bits = (const uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
         const int64_t n = n0 > n1 ? n0 : n1;
-        scales_kernel<<<(unsigned)((n + threads - 1) / threads), threads, 0, stream>>>(
+        launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
             amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr, col_bits, n1, inv_tr, a.scale_tr, qmax, status);
         ++g_launches;
     } else if (given) {
         amax_rm = amax_tr = (uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
         const int64_t n = n0 > n1 ? n0 : n1;
         const int threads = 256;
-        scales_kernel<<<(unsigned)((n + threads - 1) / threads), threads, 0, stream>>>(
+        launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
             amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
             amax_tr, n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status);
         ++g_launches;
@@ -1059,7 +1066,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         if (!few) {
             const int64_t n = n0 > n1 ? n0 : n1;
             const int threads = 256;
-            scales_kernel<<<(unsigned)((n + threads - 1) / threads), threads, 0, stream>>>(
+            launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
                 amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
                 amax_tr, n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status);
             ++g_launches;
@@ -1068,8 +1075,8 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     {
         const unsigned grid = (unsigned)(((cols + Q_TILE - 1) / Q_TILE) * ((rows + Q_TILE - 1) / Q_TILE));
         if (fast) launch_fast(a.dt, P.mode, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);
-        else if (a.dt == SRQ_F32) quantize_kernel<float><<<grid, Q_THREADS, 0, stream>>>((const float*)a.x, P);
-        else quantize_kernel<__nv_bfloat16><<<grid, Q_THREADS, 0, stream>>>((const __nv_bfloat16*)a.x, P);
+        else if (a.dt == SRQ_F32) launch_pdl(quantize_kernel<float>, dim3(grid), dim3(Q_THREADS), 0, stream, (const float*)a.x, P);
+        else launch_pdl(quantize_kernel<__nv_bfloat16>, dim3(grid), dim3(Q_THREADS), 0, stream, (const __nv_bfloat16*)a.x, P);
         ++g_launches;
     }
     return cudaGetLastError();
