@@ -908,7 +908,7 @@ static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, cons
     cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = CTAS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization; at[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = at; cfg.numAttrs = 2;
+    cfg.attrs = at; cfg.numAttrs = pdl_allowed(stream) ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, gemm_i8_kernel<CTAS, KIND>, map_a, map_b, map_out, map_part, P);
 }
 
