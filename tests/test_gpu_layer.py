@@ -196,3 +196,38 @@ def test_random_layers(case):
     A, W, dY = synth.layer_inputs(T, N, K, seed=case, dtype=dtype, device="cuda", std_dy=1e-3)
     q = layer_specs(scale, rnd, seed=case, bits_fwd=int(rng.integers(3, 9)), bits_bwd=int(rng.integers(2, 9)))
     all_passes(A, W, dY, q)
+
+
+@pytest.mark.parametrize("scale,dtype", [(srq.PER_TENSOR, torch.float32), (srq.PER_ROW, torch.bfloat16)])
+def test_a_layer_step_recorded_in_a_cuda_graph_replays_the_same_results(scale, dtype):
+    """The calls only enqueue work on the caller's stream, so forward + backward can be recorded once in
+    a CUDA graph (after one call outside the capture, which does the one-time device set-up) and
+    replayed; the replay gives the oracle's results, again after the inputs have changed."""
+    T, N, K = 264, 392, 1024
+    q = layer_specs(scale, srq.SR, seed=3)
+    A, W, dY = synth.layer_inputs(T, N, K, seed=1, dtype=dtype, device="cuda", std_dy=1e-3)
+    Y, dA, dW = torch.empty((T, N), device="cuda"), torch.empty((T, K), device="cuda"), torch.empty((N, K), device="cuda")
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
+
+    def step():
+        srq.qlinear_fwd(A, W, q["a_fwd"], q["w_fwd"], Y, None, ws)
+        srq.qlinear_bwd(dY, A, W, q["dy_bwd"], q["a_bwd"], q["w_bwd"], dA, dW, None, None, ws)
+
+    step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    oq = lambda s: oracle.QSpec(s.bits, s.scale, s.round, s.seed, s.tensor_id, s.index_offset)
+    f = lambda t: t.float().cpu().numpy()
+    for rep in range(2):
+        if rep == 1:                             # new inputs in the same buffers: the graph reads them at replay
+            A2, W2, dY2 = synth.layer_inputs(T, N, K, seed=2, dtype=dtype, device="cuda", std_dy=1e-3)
+            A.copy_(A2); W.copy_(W2); dY.copy_(dY2)
+        for t in (Y, dA, dW):
+            t.fill_(float("nan"))
+        g.replay()
+        assert srq.srq_poll_status(ws) == 0
+        assert np.array_equal(Y.cpu().numpy(), oracle.qlinear_fwd(f(A), f(W), oq(q["a_fwd"]), oq(q["w_fwd"])).out)
+        assert np.array_equal(dA.cpu().numpy(), oracle.qlinear_bwd_input(f(dY), f(W), oq(q["dy_bwd"]), oq(q["w_bwd"])).out)
+        assert np.array_equal(dW.cpu().numpy(), oracle.qlinear_bwd_weight(f(dY), f(A), oq(q["dy_bwd"]), oq(q["a_bwd"])).out)
