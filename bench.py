@@ -3,6 +3,10 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
+With --gpus N > 1 and no launcher (torch.distributed.run sets RANK / WORLD_SIZE / MASTER_*), the
+command starts its own N ranks, one per GPU; under a launcher it is one of the ranks.  Every rank
+holds its own 65536-token shard (weak scaling); rank 0 prints the line.
+
 One step = one pass of the whole hot path over one batch: qlinear_fwd (Alg. 1) and qlinear_bwd
 (Alg. 2: both backward products) - five absmax reductions and quantizations, three int8
 tensor-core products with dequantizing epilogues - on a 4096 x 4096 linear layer with 65536 tokens, fp32 inputs,
@@ -26,9 +30,10 @@ UNIT = "TOPS"
 WORKLOAD = "linear 4096->4096, tokens 65536, fp32 inputs, 8-bit per-tensor SR on A, W, dY (fwd + bwd)"
 T_FULL, N_FULL, K_FULL = 65536, 4096, 4096
 
-# DRAM bytes (read + write) of one gemm_i8_kernel launch of this workload, from the ncu capture
-# summarised in profiles/gemm_i8_kernel_M8192_N4096_K4096.md (its bench-size section).
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = 1338072320   # forward-shaped launch, M=65536 N=4096 K=4096
+# DRAM bytes (read + write) of one gemm_i8_kernel launch of this workload (forward-shaped launch,
+# M=65536 N=4096 K=4096) as a profiler capture counted them; not a quantity this run measures.
+# None while the kernel has changed since the counters were taken.
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 1338072320
 
 
 def layer_ops(T, N, K):
@@ -171,25 +176,42 @@ def run_reference(args):
 # ---------------------------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------------------------
+def needs_spawn(gpus: int) -> bool:
+    """True when this process must start the ranks itself: several GPUs asked for, no launcher."""
+    from paper_2511_00874_b200 import dp
+    return gpus > 1 and not dp.launched_by_env()
+
+
+def _timed_loop(fn, seconds, est_ms, torch):
+    """Runs fn back to back for about `seconds` (count fixed beforehand from est_ms, so that every rank
+    runs the same number); returns (ms per call, calls) by CUDA events on the current stream."""
+    n = max(3, int(seconds * 1e3 / max(est_ms, 1e-3)) + 1)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(n):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / n, n
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
 
     import paper_2511_00874_b200 as srq
-    from paper_2511_00874_b200 import binding, synth
+    from paper_2511_00874_b200 import binding, dp, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     binding.lib()                      # fails loudly if libsrq.so is missing
+    local = int(os.environ.get("LOCAL_RANK", os.environ.get("RANK", "0")))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    rank, local, world = dp.init_from_env("nccl", dev)
 
     T, N, K = T_FULL, N_FULL, K_FULL
+    shard = dp.TokenShard(rank, world, T)
     peaks = load_peaks()
 
     # each rank holds its own token shard (weak scaling); W is replicated
@@ -201,13 +223,19 @@ def run_ours(args):
     dW = torch.empty((N, K), device=dev)
     ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K), dev)
 
-    # max |A| and max |dY|: found once per step, max-reduced over the token shards when there are several
+    # max |A| and max |dY|: found once per step, max-reduced over the token shards in ONE collective
     # (so that every rank uses the step sizes of the whole batch), and handed to the quantization points
-    amax_a = torch.zeros(1, device=dev)
-    amax_dy = torch.zeros(1, device=dev)
+    amax = torch.zeros(2, device=dev)
+    amax_a, amax_dy = amax[0:1], amax[1:2]
+    # Several ranks: the weight gradient sums over all shards.  While the int32 sums of the whole batch
+    # cannot overflow, the ranks all-reduce the exact sums and scale the total once (bit for bit the
+    # gradient one GPU computes on the whole batch); otherwise they all-reduce the fp32 gradients.
+    exact_dw = world > 1 and dp.int32_sums_fit(world, T, 8, 8)
+    sums = torch.empty((N, K), dtype=torch.int32, device=dev) if exact_dw else None
+    step_dy, step_a = torch.empty(1, device=dev), torch.empty(1, device=dev)
 
     def specs(step):
-        off_a, off_y = rank * T * K, rank * T * N       # thresholds follow the global flat index
+        off_a, off_y = shard.index_offset(K), shard.index_offset(N)       # thresholds follow the global flat index
         return (srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 0, off_a, absmax=amax_a), srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 1),
                 srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 2, off_a, absmax=amax_a), srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 3),
                 srq.QSpec(8, srq.PER_TENSOR, srq.SR, step, 4, off_y, absmax=amax_dy))
@@ -216,18 +244,28 @@ def run_ours(args):
         qa_f, qw_f, qa_b, qw_b, qdy = specs(i)
         srq.srq_absmax(a, amax_a)
         srq.srq_absmax(dy, amax_dy)
-        if world > 1:
-            dist.all_reduce(amax_a, op=dist.ReduceOp.MAX)
-            dist.all_reduce(amax_dy, op=dist.ReduceOp.MAX)
+        dp.reduce_absmax(amax, world)
         srq.qlinear_fwd(a, w, qa_f, qw_f, y, None, ws)
-        srq.qlinear_bwd(dy, a, w, qdy, qa_b, qw_b, da, dw, None, None, ws)      # Alg. 2: both backward products
-        if world > 1:
-            dist.all_reduce(dw)        # the batch average of the weight gradient spans all shards
+        if exact_dw:
+            srq.qlinear_bwd_ex(dy, a, w, qdy, qa_b, qw_b, da, sums, None, None, ws,
+                               dbg_weight=srq.DebugOut(scale_a=step_dy, scale_b=step_a))   # raw int32 sums of dW
+            dp.reduce_sum(sums, world)
+            srq.srq_dequant_i32(sums, step_dy, step_a, dw)
+        else:
+            srq.qlinear_bwd(dy, a, w, qdy, qa_b, qw_b, da, dw, None, None, ws)      # Alg. 2: both backward products
+            dp.reduce_sum(dw, world)   # the batch average of the weight gradient spans all shards
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+
+    def max_over_ranks(v):
+        if world == 1:
+            return v
+        t = torch.tensor([v], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return t.item()
 
     quantizer = None
     if rank == 0:
@@ -275,16 +313,20 @@ def run_ours(args):
     e1.record()
     barrier()
     launches = srq.launch_count() - l0
-    ms = e0.elapsed_time(e1) / args.steps
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = t.item()
+    ms = max_over_ranks(e0.elapsed_time(e1) / args.steps)
     clocks = sampler.stop() if rank == 0 else None
     st = srq.srq_poll_status(ws)
     if st != 0:
         raise SystemExit("device status after the timed region: " + srq.status_string(st))
     value = world * layer_ops(T, N, K) / (ms * 1e-3) / 1e12
+
+    gathered = None
+    if world > 1:
+        # which process sat on which device (rank 0 puts the list into the line)
+        gathered = [None] * world
+        me = {"rank": rank, "local_rank": local, "device": torch.cuda.get_device_name(dev), "pid": os.getpid(),
+              "uuid": str(torch.cuda.get_device_properties(dev).uuid), "index_offset_A": shard.index_offset(K)}
+        dist.gather_object(me, gathered if rank == 0 else None, dst=0)
 
     result = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
               "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -292,8 +334,26 @@ def run_ours(args):
               "config": {"workload": WORKLOAD, "tokens_per_gpu": T, "l2": "inputs (1 GiB each) are larger than L2",
                          "absmax": "max |A| and max |dY| are computed once per step (srq_absmax; max-reduced over ranks when "
                                    "N > 1) and handed to their quantization points; max |A| serves both of A's points",
-                         "multi_gpu": "token shards, two scalar all-reduce(max) and one all-reduce(sum) of dW per step" if world > 1 else "single GPU"},
+                         "multi_gpu": ("token shards; per step one 2-element all-reduce(max) of the maxima and one all-reduce(sum) of "
+                                       + ("the exact int32 sums of dW, scaled once afterwards" if exact_dw else
+                                          "the fp32 dW (the int32 sums of the whole batch could overflow)")) if world > 1 else "single GPU",
+                         "regime": "the timed region is --steps steps long: a short run is a burst figure (full clocks), "
+                                   "see `sustained` for the same step under the power cap"},
               "gpu_launches": int(launches)}
+    if gathered is not None and rank == 0:
+        result["ranks"] = gathered
+
+    # ---- the same step for at least two seconds: the figure a long training run sees (power cap, lower clocks)
+    sus_sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sus_sampler.start()
+    sus_ms, sus_n = _timed_loop(lambda i: step(2000 + i), 2.0, ms, torch)
+    barrier()
+    sus_ms = max_over_ranks(sus_ms)
+    sus_clocks = sus_sampler.stop() if rank == 0 else None
+    result["sustained"] = {"ms_per_step": sus_ms, "value": world * layer_ops(T, N, K) / (sus_ms * 1e-3) / 1e12, "unit": UNIT,
+                           "steps": sus_n, "clocks": sus_clocks}
 
     # ---- end to end through the public API with host buffers (every rank, max over ranks).
     # Every step copies its inputs from pinned host memory and its results back; the copies of
@@ -328,11 +388,7 @@ def run_ours(args):
                 h.copy_(d, non_blocking=True)
             ev_out[i].record(s_out)
     torch.cuda.synchronize()
-    e_sec = (time.perf_counter() - t0) / e_steps
-    if world > 1:
-        t = torch.tensor([e_sec], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e_sec = t.item()
+    e_sec = max_over_ranks((time.perf_counter() - t0) / e_steps)
     h2d = sum(t.numel() * 4 for t in (hA, hW, hdY))
     d2h = sum(t.numel() * 4 for t in (hY, hdA, hdW))
     result["e2e"] = {"value": world * layer_ops(T, N, K) / e_sec / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -342,8 +398,7 @@ def run_ours(args):
     del hA, hW, hdY, hY, hdA, hdW, ins, outs
 
     if rank == 0:
-        # ---- per-kernel timing of the dominant kernel: the three products of one step, on the codes
-        # the quantizer wrote, each launch bracketed by CUDA events on the launching stream
+        # ---- the dominant kernel: the three products of one step, on the codes the quantizer wrote
         one = torch.ones(1, device=dev)
 
         def codes(x, rows, cols, q, rm, tr):
@@ -362,7 +417,14 @@ def run_ours(args):
         for a_, b_, o_ in gemms:
             srq.srq_gemm_i8(a_, b_, one, one, o_, None, gws)
         torch.cuda.synchronize()
-        reps = max(3, args.steps)
+        time.sleep(1.0)                          # let the clocks recover from the long loops above
+        ops_per_launch = 2.0 * T * N * K
+
+        # burst: every launch bracketed by its own CUDA events on the launching stream, a short series
+        b_sampler = ClockSampler(local)
+        b_sampler.start()
+        time.sleep(0.5)                          # the sampler needs a moment before its first line
+        reps = 20
         evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in gemms]
                for _ in range(reps)]
         for r in range(reps):
@@ -371,28 +433,45 @@ def run_ours(args):
                 srq.srq_gemm_i8(a_, b_, one, one, o_, None, gws)
                 evs[r][j][1].record()
         torch.cuda.synchronize()
+        b_clocks = b_sampler.stop()
         gemm_ms = [statistics.mean(evs[r][j][0].elapsed_time(evs[r][j][1]) for r in range(reps)) for j in range(3)]
         launch_ms = statistics.mean(gemm_ms)
-        ops_per_launch = 2.0 * T * N * K
         achieved = ops_per_launch / (launch_ms * 1e-3) / 1e12
-        peak = 2.0 * peaks["bf16_sustained"]        # int8 : bf16 dense nominal ratio is 2
+        peak_burst = 2.0 * peaks["bf16_burst"]        # int8 : bf16 dense nominal ratio is 2
+
+        # sustained: the same three launches back to back for two seconds, against the sustained figure
+        s_sampler = ClockSampler(local)
+        s_sampler.start()
+
+        def three(_):
+            for a_, b_, o_ in gemms:
+                srq.srq_gemm_i8(a_, b_, one, one, o_, None, gws)
+        s_ms3, s_n = _timed_loop(three, 2.0, 3.0 * launch_ms, torch)
+        s_clocks = s_sampler.stop()
+        s_achieved = ops_per_launch / (s_ms3 / 3.0 * 1e-3) / 1e12
+        peak_sus = 2.0 * peaks["bf16_sustained"]
         result["roofline"] = {
-            "bound": "tensor", "kernel": "gemm_i8_kernel", "achieved": achieved, "peak": peak, "unit": "TOPS",
-            "frac": achieved / peak, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
-            "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS TFLOP/s (int8:bf16 nominal ratio 2)",
-            "frac_of_burst": achieved / (2.0 * peaks["bf16_burst"]), "frac_of_nominal_4500": achieved / 4500.0,
+            "bound": "tensor", "kernel": "gemm_i8_kernel", "achieved": achieved, "peak": peak_burst, "unit": "TOPS",
+            "frac": achieved / peak_burst, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
+            "traffic_source": "DRAM read + write bytes of one launch from a profiler capture (summary under profiles/), "
+                              "not measured by this run",
+            "regime": "burst: 60 launches, each timed alone by CUDA events",
+            "peak_source": f"2 x {peaks['source']} burst bf16 cuBLAS TFLOP/s (int8:bf16 nominal ratio 2)",
+            "frac_of_nominal_4500": achieved / 4500.0,
             "ms_per_launch": {"fwd": gemm_ms[0], "bwd_input": gemm_ms[1], "bwd_weight": gemm_ms[2]},
-            "ops_per_launch": ops_per_launch}
+            "ops_per_launch": ops_per_launch, "clocks": b_clocks,
+            "sustained": {"achieved": s_achieved, "peak": peak_sus, "frac": s_achieved / peak_sus,
+                          "ms_per_launch": s_ms3 / 3.0, "launches": 3 * s_n, "clocks": s_clocks,
+                          "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS TFLOP/s",
+                          "regime": "the three products back to back for two seconds (power cap)"}}
         del cA, cAt, cW, cWt, cdY, cdYt
 
         result["quantizer"] = quantizer
         result["clocks"] = clocks
         if world == 1:
             result["cpu_baseline"] = cpu_baseline()
-        print(json.dumps(result))
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+        print(json.dumps(result), flush=True)
+    dp.finish()
 
 
 def main():
@@ -405,6 +484,9 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif needs_spawn(args.gpus):
+        from paper_2511_00874_b200 import dp
+        sys.exit(dp.spawn_ranks(args.gpus, [os.path.abspath(__file__), *sys.argv[1:]]))
     else:
         run_ours(args)
 

@@ -15,7 +15,11 @@
  *   - Every tensor pointer is a DEVICE pointer owned by the caller, the
  *     workspace included.  qspec pointers and the debug struct are HOST
  *     pointers, read before the call returns.  The library allocates no
- *     device memory and keeps no state between calls.
+ *     device memory.  Between calls it keeps only what it has learned about the
+ *     devices (SM count, how many CTAs of a kernel fit, the address of the array
+ *     sr_quantize_static uses; each found once, thread-safely) and the launch
+ *     counter of srq_launch_count; nothing of it changes a result.
+ *     (sr_quantize_static is the one exception to "no device memory": see there.)
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL
  *     for the default stream) and the call returns without waiting.
  *   - Errors the host can see (null pointer, bits outside the grid's range, a pitch or
@@ -24,7 +28,9 @@
  *     and enqueue nothing.  Conditions only the device can see (an input
  *     that is not finite, a bounded wait inside a kernel that ran out) are
  *     recorded in a status word at the start of the workspace; read it with
- *     srq_poll_status.  After such a condition the outputs are unspecified.
+ *     srq_poll_status (sr_quantize_static, which has no workspace, reports
+ *     through a word the caller passes).  After such a condition the outputs are
+ *     unspecified.
  *   - Outputs are overwritten, unless a srq_output_t (the *_ex entry points) asks for accumulation.
  *   - Both operands of a layer pass use the same grid (srq_qspec_t.format).  With the
  *     floating-point grid (E4M3, or E4M2 / E4M1 / E4M0 by `bits`) the codes are E4M3 bytes,
@@ -291,6 +297,14 @@ srq_status_t qlinear_bwd(const void *dY, const void *A, const void *W, srq_dtype
  *               the nearest bfloat16, ties to even, as it is stored, which halves the bytes the
  *               product writes.  Codes and absmax still come from the binary32 result.  Not with
  *               accumulate = 1 (SRQ_ERR_UNSUPPORTED): running binary32 sums stay in binary32.
+ *   raw_sums    1: the output pointer of the call addresses int32 numbers (pass it cast to float *;
+ *               its pitch counts int32 elements) and receives the exact sums themselves; nothing
+ *               is scaled.  For token shards on several devices (the batch axis of the variance
+ *               lemma): the shards' sums are added with an integer all-reduce, which is exact in
+ *               any order, and srq_dequant_i32 then scales the total once, so that the weight
+ *               gradient is bit for bit the one a single device computes on the whole batch
+ *               (given shared step sizes, srq_qspec_t.absmax).  Integer grid only; not combined
+ *               with any other member (SRQ_ERR_UNSUPPORTED).
  * Products with q or absmax set are never split along the contraction.
  */
 typedef struct {
@@ -301,6 +315,7 @@ typedef struct {
     int8_t *codes;
     int64_t ld_codes;
     float *absmax;
+    int32_t raw_sums;
 } srq_output_t;
 
 /* srq_gemm_i8, qlinear_fwd and qlinear_bwd with output options (NULL = none, i.e. the plain call).
@@ -323,6 +338,20 @@ srq_status_t qlinear_bwd_ex(const void *dY, const void *A, const void *W, srq_dt
                             const srq_output_t *output_dA, const srq_output_t *output_dW,
                             const srq_debug_out_t *dbg_input, const srq_debug_out_t *dbg_weight,
                             void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * The finishing step of a product on its own (the last line of Alg. 1 / Alg. 2 once the integer
+ * sums exist): out[i, j] = float(acc[i, j]) * (s_row[i * row_stride] * s_col[j * col_stride]) over a
+ * caller's int32 matrix acc[M, N] (pitch ld_acc), with the same three roundings in the same order as
+ * the products' own epilogue, so that sums collected with raw_sums and scaled here give the very
+ * bits the one-call product gives.  out is binary32 [M, ldo], or bfloat16 when out_bf16 = 1 (round
+ * to nearest even).  All pointers are device pointers, 4-byte aligned (16-byte alignment and
+ * pitches that are multiples of 4 allow vector accesses).  Needs no workspace.
+ */
+srq_status_t srq_dequant_i32(const int32_t *acc, int64_t ld_acc, int64_t M, int64_t N,
+                             const float *s_row, int32_t row_stride,
+                             const float *s_col, int32_t col_stride,
+                             void *out, int64_t ldo, int32_t out_bf16, void *cuda_stream);
 
 /* Waits for the stream, then returns the device status word of the workspace: SRQ_OK, or the
  * first device-side condition recorded by the calls that used this workspace since its header

@@ -2,8 +2,10 @@
 
 TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the bench's CPU
 baseline leg import this; the product package never does, and this module
-never imports the product package.  All arithmetic lives in the C file; this
-module only builds it with gcc and marshals numpy arrays.
+never imports the product package.  The arithmetic lives in the C file; this
+module builds it with gcc and marshals numpy arrays.  One exception, stated
+where it occurs: qlinear_fwd_fp_act forms its binary64 product with numpy's
+matmul (a library routine used as one step) around the C quantizer.
 """
 from __future__ import annotations
 

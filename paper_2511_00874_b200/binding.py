@@ -27,7 +27,7 @@ GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
            "sr_quantize", "sr_quantize_static", "srq_absmax", "srq_absmax_cols", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
-           "srq_gemm_i8_ex", "qlinear_fwd_ex", "qlinear_bwd_ex",
+           "srq_gemm_i8_ex", "qlinear_fwd_ex", "qlinear_bwd_ex", "srq_dequant_i32",
            "srq_poll_status", "srq_status_string", "srq_launch_count", "srq_selftest_bounded_wait", "srq_plan_splits"]
 
 
@@ -53,7 +53,7 @@ class _DebugOut(ctypes.Structure):
 class _Output(ctypes.Structure):
     _fields_ = [("accumulate", ctypes.c_int32), ("out_bf16", ctypes.c_int32), ("q", ctypes.POINTER(_QSpec)),
                 ("step", ctypes.c_void_p), ("codes", ctypes.c_void_p), ("ld_codes", ctypes.c_int64),
-                ("absmax", ctypes.c_void_p)]
+                ("absmax", ctypes.c_void_p), ("raw_sums", ctypes.c_int32)]
 
 
 @dataclass
@@ -119,6 +119,8 @@ def lib() -> ctypes.CDLL:
     L.qlinear_fwd_ex.restype = ctypes.c_int
     L.qlinear_bwd_ex.argtypes = [vp, vp, vp, ctypes.c_int, i64, i64, i64, qp, qp, qp, vp, vp, op, op, dp, dp, vp, sz, vp]
     L.qlinear_bwd_ex.restype = ctypes.c_int
+    L.srq_dequant_i32.argtypes = [vp, i64, i64, i64, vp, i32, vp, i32, vp, i64, i32, vp]
+    L.srq_dequant_i32.restype = ctypes.c_int
     L.srq_selftest_bounded_wait.argtypes = [vp, sz, ctypes.c_uint32, vp]
     L.srq_selftest_bounded_wait.restype = ctypes.c_int
     L.srq_plan_splits.argtypes = [i64, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
@@ -377,22 +379,25 @@ class Output:
     codes: Optional[torch.Tensor] = None
     absmax: Optional[torch.Tensor] = None
 
-    def c(self, out_bf16: bool = False):
+    def c(self, out_bf16: bool = False, raw_sums: bool = False):
         cq = self.q.c() if self.q is not None else None
         o = _Output(int(self.accumulate), int(out_bf16), ctypes.pointer(cq) if cq is not None else None, _ptr(self.step),
-                    _ptr(self.codes), self.codes.stride(0) if self.codes is not None else 0, _ptr(self.absmax))
+                    _ptr(self.codes), self.codes.stride(0) if self.codes is not None else 0, _ptr(self.absmax),
+                    int(raw_sums))
         o._keep = cq                      # the struct points into cq
         return o
 
 
 def _opt(o: Optional[Output], out: Optional[torch.Tensor] = None):
-    """The C struct of the options; a bfloat16 output tensor selects out_bf16 by itself."""
+    """The C struct of the options; a bfloat16 output tensor selects out_bf16 by itself, an int32
+    output tensor raw_sums (the exact sums, unscaled)."""
     bf16 = out is not None and out.dtype == torch.bfloat16
-    if out is not None and not bf16 and out.dtype != torch.float32:
-        raise TypeError("the output of a product is float32 or bfloat16")
+    raw = out is not None and out.dtype == torch.int32
+    if out is not None and not bf16 and not raw and out.dtype != torch.float32:
+        raise TypeError("the output of a product is float32, bfloat16 or (raw sums) int32")
     if o is None:
-        return Output().c(True) if bf16 else None
-    return o.c(bf16)
+        return Output().c(bf16, raw) if (bf16 or raw) else None
+    return o.c(bf16, raw)
 
 
 def srq_gemm_i8_ex(a: torch.Tensor, b: torch.Tensor, s_row: torch.Tensor, s_col: torch.Tensor,
@@ -452,6 +457,20 @@ def qlinear_bwd_ex(dY: torch.Tensor, A: torch.Tensor, W: torch.Tensor, qdY: QSpe
                               ctypes.byref(d1) if d1 is not None else None,
                               ws.data_ptr(), ws.numel(), _stream())
     _check(st, "qlinear_bwd_ex")
+
+
+def srq_dequant_i32(acc: torch.Tensor, s_row: torch.Tensor, s_col: torch.Tensor, out: torch.Tensor) -> None:
+    """out[M,N] = float(acc[M,N]) * (s_row x s_col): the finishing step over int32 sums (e.g. the
+    all-reduced raw sums of token shards).  out is float32 or bfloat16."""
+    _dev2d(acc, "acc")
+    _dev2d(out, "out")
+    if acc.dtype != torch.int32 or out.dtype not in (torch.float32, torch.bfloat16) or acc.shape != out.shape:
+        raise TypeError("acc must be int32 [M, N], out float32 or bfloat16 [M, N]")
+    M, N = acc.shape
+    st = lib().srq_dequant_i32(acc.data_ptr(), acc.stride(0), M, N, s_row.data_ptr(), int(s_row.numel() != 1),
+                               s_col.data_ptr(), int(s_col.numel() != 1), out.data_ptr(), out.stride(0),
+                               int(out.dtype == torch.bfloat16), _stream())
+    _check(st, "srq_dequant_i32")
 
 
 def srq_plan_splits(tiles: int, k_blocks: int, groups: int):

@@ -4,11 +4,8 @@
 
 using namespace srq;
 
-namespace {
-
-inline int qmax_of(int bits) { return (1 << (bits - 1)) - 1; }
-
-srq_status_t check_qspec(const srq_qspec_t* q) {
+// Host-side validation of one quantization point, shared by every entry point that takes one.
+srq_status_t srq::check_qspec(const srq_qspec_t* q) {
     if (!q) return SRQ_ERR_INVALID_ARG;
     if (q->format != SRQ_GRID_INT && q->format != SRQ_GRID_E4M3) return SRQ_ERR_INVALID_ARG;
     if (q->format == SRQ_GRID_INT && (q->bits < 2 || q->bits > 8)) return SRQ_ERR_UNSUPPORTED;
@@ -20,6 +17,10 @@ srq_status_t check_qspec(const srq_qspec_t* q) {
     return SRQ_OK;
 }
 
+namespace {
+
+inline int qmax_of(int bits) { return (1 << (bits - 1)) - 1; }
+
 // Host-side checks of the output options of a product with an [M, N] result, and their device form.
 srq_status_t make_out_options(const srq_output_t* o, int64_t N, bool have_out, OutOptions* r) {
     *r = OutOptions();
@@ -28,8 +29,11 @@ srq_status_t make_out_options(const srq_output_t* o, int64_t N, bool have_out, O
     if (o->accumulate && !have_out) return SRQ_ERR_INVALID_ARG;
     if (o->out_bf16 != 0 && o->out_bf16 != 1) return SRQ_ERR_INVALID_ARG;
     if (o->out_bf16 && o->accumulate == 1) return SRQ_ERR_UNSUPPORTED;   // running binary32 sums stay in binary32
+    if (o->raw_sums != 0 && o->raw_sums != 1) return SRQ_ERR_INVALID_ARG;
+    if (o->raw_sums && (!have_out || o->accumulate || o->out_bf16 || o->q || o->absmax)) return SRQ_ERR_UNSUPPORTED;
     r->accumulate = o->accumulate;
     r->out_bf16 = o->out_bf16;
+    r->raw_sums = o->raw_sums;
     if (o->q) {
         srq_status_t s = check_qspec(o->q);
         if (s != SRQ_OK) return s;
@@ -101,7 +105,7 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
     if ((s = check_qspec(a.q)) != SRQ_OK) return s;
     if ((s = check_qspec(b.q)) != SRQ_OK) return s;
     if (!aligned_to(a.x, 16) || !aligned_to(b.x, 16) || !aligned_to(out, 16) || !aligned_to(ws, 256)) return SRQ_ERR_INVALID_ARG;
-    if (opt.requant && a.q->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;
+    if ((opt.requant || opt.raw_sums) && a.q->format != SRQ_GRID_INT) return SRQ_ERR_UNSUPPORTED;
     const int64_t M = a.out_rows(), Nn = b.out_rows(), Kc = a.out_cols();
     if (Kc != b.out_cols()) return SRQ_ERR_INVALID_ARG;
     if (a.q->format != b.q->format) return SRQ_ERR_INVALID_ARG;          // one product, one kind of code
@@ -267,6 +271,7 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
         return SRQ_ERR_INVALID_ARG;
     if (qdY->format != qW->format || qdY->format != qA->format) return SRQ_ERR_INVALID_ARG;
     const int kind = qdY->format == SRQ_GRID_E4M3;
+    if (kind && (opt_in.raw_sums || opt_w.raw_sums)) return SRQ_ERR_UNSUPPORTED;       // int32 sums exist on the integer grid only
     if (!kind && (double)N * qmax_of(qdY->bits) * qmax_of(qW->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
     if (!kind && (double)T * qmax_of(qdY->bits) * qmax_of(qA->bits) >= 2147483648.0) return SRQ_ERR_ACC_OVERFLOW;
     const BwdPlan p = plan_bwd(T, N, K);
@@ -507,6 +512,17 @@ srq_status_t qlinear_bwd_ex(const void* dY, const void* A, const void* W, srq_dt
     return run_bwd(dY, A, W, dt, T, N, K, qdY, qA, qW, dA, dW, output_dA, output_dW, dbg_input, dbg_weight, ws, ws_bytes, cuda_stream);
 }
 
+srq_status_t srq_dequant_i32(const int32_t* acc, int64_t ld_acc, int64_t M, int64_t N, const float* s_row, int32_t row_stride,
+                             const float* s_col, int32_t col_stride, void* out, int64_t ldo, int32_t out_bf16, void* cuda_stream) {
+    if (!acc || !s_row || !s_col || !out) return SRQ_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || ld_acc < N || ldo < N) return SRQ_ERR_INVALID_ARG;
+    if ((row_stride != 0 && row_stride != 1) || (col_stride != 0 && col_stride != 1)) return SRQ_ERR_INVALID_ARG;
+    if (out_bf16 != 0 && out_bf16 != 1) return SRQ_ERR_INVALID_ARG;
+    if (!aligned_to(acc, 4) || !aligned_to(s_row, 4) || !aligned_to(s_col, 4) || !aligned_to(out, out_bf16 ? 2 : 4)) return SRQ_ERR_INVALID_ARG;
+    return launch_finish_sums(acc, ld_acc, M, N, s_row, row_stride, s_col, col_stride, (float*)out, ldo, out_bf16,
+                              (cudaStream_t)cuda_stream) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+}
+
 void srq_plan_splits(int64_t tiles, int32_t k_blocks, int32_t groups, int32_t* full_tiles, int32_t* splits) {
     if (!full_tiles || !splits) return;
     *full_tiles = 0; *splits = 0;
@@ -545,6 +561,6 @@ const char* srq_status_string(srq_status_t s) {
     return "unknown status";
 }
 
-uint64_t srq_launch_count(void) { return (uint64_t)g_launches; }
+uint64_t srq_launch_count(void) { return (uint64_t)g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "srq.h"
 
 namespace srq {
@@ -19,7 +21,9 @@ static_assert(sizeof(WsHeader) == 256, "header is one 256-byte line");
 constexpr size_t kAlign = 256;
 __host__ __device__ inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 
-extern unsigned long long g_launches;   // kernels launched by this process (host counter)
+// Kernels launched by this process (host counter; entry points may be called from several threads).
+extern std::atomic<unsigned long long> g_launches;
+inline void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 // Programmatic dependent launch.  Every kernel of the library waits for the results of the work before
 // it as its first act (griddepcontrol.wait returns once the preceding grids have finished and their
@@ -27,7 +31,10 @@ extern unsigned long long g_launches;   // kernels launched by this process (hos
 // kernel after it be launched, so that the successor's launch and start-up overlap this kernel's
 // execution instead of following it.  Nothing is read or written before the wait, so the order of the
 // stream is kept; a kernel two places ahead has finished as well, because the one in between only
-// finishes after its own wait.
+// finishes after its own wait.  A kernel launched through launch_pdl (or with the same attribute)
+// that did NOT start with pdl_enter() could read its predecessor's half-written output, so every
+// __global__ function of the library starts with it; a host-side test reads the sources and fails
+// for a kernel that does not.
 __device__ __forceinline__ void pdl_enter() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -88,6 +95,10 @@ inline PhiloxKeys make_philox_keys(uint64_t seed, uint64_t tensor_id) {
     return k;
 }
 
+// SRQ_OK, or why the quantization point cannot be used: unknown grid, scale or rounding mode, a bit
+// width outside the grid's range, a mode the grid does not have, a misaligned absmax pointer.
+srq_status_t check_qspec(const srq_qspec_t* q);
+
 // ------------------------------------------------------------------------------------------
 // Quantizer (quantize.cu)
 // ------------------------------------------------------------------------------------------
@@ -132,6 +143,7 @@ cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, 
 struct OutOptions {
     int32_t accumulate = 0;          // out += result instead of out = result
     int32_t out_bf16 = 0;            // out holds bfloat16 [M, ldo]: each result rounded to nearest even
+    int32_t raw_sums = 0;            // out holds int32 [M, ldo]: the sums themselves, nothing is scaled
     int32_t requant = 0;             // also write Q(result) as int8 codes with a given step size
     int32_t rq_sr = 0;               // stochastic rounding (else round to nearest)
     float rq_lim = 0.0f;             // qmax * 2^24: saturation bound of the fixed-point quotient
@@ -157,6 +169,9 @@ size_t gemm_splitk_bytes(int64_t M, int64_t N);
 void gemm_plan_splits(int64_t tiles, int32_t num_kb, int groups, int32_t* full_tiles, int32_t* splits);
 // One thread waits (at most limit_ns) on a barrier nobody signals and records SRQ_ERR_TIMEOUT.
 cudaError_t launch_bounded_wait_probe(uint32_t* status, uint64_t limit_ns, cudaStream_t stream);
+// out = float(acc) * (s_row * s_col) over a caller's int32 matrix (the finishing step on its own).
+cudaError_t launch_finish_sums(const int32_t* acc, int64_t ld_acc, int64_t M, int64_t N, const float* s_row, int32_t row_stride,
+                               const float* s_col, int32_t col_stride, float* out, int64_t ldo, int out_bf16, cudaStream_t stream);
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream);
 
 }  // namespace srq

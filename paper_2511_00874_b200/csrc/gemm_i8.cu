@@ -584,13 +584,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
                     const float* sc = &T->s_col[buf][j * 32];
+                    if (!P.opt.raw_sums) {                    // raw sums leave as the int32 words they are
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 c4 = *reinterpret_cast<const float4*>(sc + 4 * q);
-                        v[4 * q + 0] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 0]), __fmul_rn(sr, c4.x)));
-                        v[4 * q + 1] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 1]), __fmul_rn(sr, c4.y)));
-                        v[4 * q + 2] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 2]), __fmul_rn(sr, c4.z)));
-                        v[4 * q + 3] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 3]), __fmul_rn(sr, c4.w)));
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 c4 = *reinterpret_cast<const float4*>(sc + 4 * q);
+                            v[4 * q + 0] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 0]), __fmul_rn(sr, c4.x)));
+                            v[4 * q + 1] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 1]), __fmul_rn(sr, c4.y)));
+                            v[4 * q + 2] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 2]), __fmul_rn(sr, c4.z)));
+                            v[4 * q + 3] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[4 * q + 3]), __fmul_rn(sr, c4.w)));
+                        }
                     }
                     const int32_t col0 = (int32_t)col_base + j * 32;
                     output_options(P, v, row, col0, rq_inv, amax);
@@ -638,6 +640,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 for (int i = 0; i < 32; ++i)
                                     if (col0 + i < P.N) ad[i] = (int32_t)v[i];
                             }
+                        }
+                        if (P.opt.raw_sums) {                   // the sums themselves, element by element
+                            uint32_t* dst = reinterpret_cast<uint32_t*>(P.out) + row * P.ldo + col0;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (col0 + i < P.N) dst[i] = v[i];
+                            continue;
                         }
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
@@ -720,7 +729,7 @@ __global__ void __launch_bounds__(256)
 dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_tile, int32_t tiles_n, int32_t tile_rows,
                int64_t M, int64_t N, const float* __restrict__ s_row, int32_t row_stride,
                const float* __restrict__ s_col, int32_t col_stride, float* __restrict__ out, int64_t ldo,
-               int32_t* __restrict__ acc_out, int vec, int accumulate, int out_bf16, uint32_t* status) {
+               int32_t* __restrict__ acc_out, int vec, int accumulate, int out_bf16, int raw_sums, uint32_t* status) {
     pdl_enter();
     const int64_t per_tile = (int64_t)tile_rows * (BN / 4);
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_tiles * per_tile; g += (int64_t)gridDim.x * blockDim.x) {
@@ -738,6 +747,12 @@ dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_
                 if (((before ^ total) & (av[e] ^ total)) < 0) record_status(status, SRQ_ERR_ACC_OVERFLOW);
                 av[e] = total;
             }
+        }
+        if (raw_sums) {                        // the caller wants the sums themselves
+            int32_t* dst = reinterpret_cast<int32_t*>(out) + r * ldo + c;
+            if (vec && c + 4 <= N) *reinterpret_cast<int4*>(dst) = make_int4(av[0], av[1], av[2], av[3]);
+            else for (int e = 0; e < 4 && c + e < N; ++e) dst[e] = av[e];
+            continue;
         }
         const float sr = s_row[r * row_stride];
         float o[4];
@@ -771,6 +786,43 @@ dequant_kernel(const int32_t* __restrict__ part, int64_t n_tiles, int64_t first_
     }
 }
 
+// The finishing step on its own, over a caller's int32 matrix: out = float(sum) * (s_row * s_col), the
+// same two binary32 multiplies in the same order as the epilogue.  For sums that were added up
+// elsewhere (over token shards on several devices) before they are scaled once.  One thread per four
+// consecutive columns; vec: 16-byte loads and 16-byte (binary32) or 8-byte (bfloat16) stores allowed.
+__global__ void __launch_bounds__(256)
+finish_sums_kernel(const int32_t* __restrict__ acc, int64_t ld_acc, int64_t M, int64_t N,
+                   const float* __restrict__ s_row, int32_t row_stride, const float* __restrict__ s_col, int32_t col_stride,
+                   float* __restrict__ out, int64_t ldo, int vec, int out_bf16) {
+    pdl_enter();
+    const int64_t per_row = (N + 3) / 4;
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < M * per_row; g += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = g / per_row, c = (g % per_row) * 4;
+        const int32_t* src = acc + r * ld_acc + c;
+        int32_t av[4] = {0, 0, 0, 0};
+        if (vec && c + 4 <= N) {
+            const int4 a = __ldcs(reinterpret_cast<const int4*>(src));
+            av[0] = a.x; av[1] = a.y; av[2] = a.z; av[3] = a.w;
+        } else {
+            for (int e = 0; e < 4 && c + e < N; ++e) av[e] = src[e];
+        }
+        const float sr = s_row[r * row_stride];
+        float o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            o[e] = (c + e < N) ? __fmul_rn(__int2float_rn(av[e]), __fmul_rn(sr, s_col[(c + e) * col_stride])) : 0.0f;
+        if (out_bf16) {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(out) + r * ldo + c;
+            if (vec && c + 4 <= N) *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3]));
+            else for (int e = 0; e < 4 && c + e < N; ++e) dst[e] = __float2bfloat16_rn(o[e]);
+        } else {
+            float* dst = out + r * ldo + c;
+            if (vec && c + 4 <= N) __stcs(reinterpret_cast<float4*>(dst), make_float4(o[0], o[1], o[2], o[3]));
+            else for (int e = 0; e < 4 && c + e < N; ++e) dst[e] = o[e];
+        }
+    }
+}
+
 // Self-test of the bounded wait: one thread waits on a barrier that nothing ever arrives on, with a
 // short limit; the wait gives up, the status word receives SRQ_ERR_TIMEOUT and the kernel returns.
 __global__ void bounded_wait_probe_kernel(uint32_t* status, uint64_t limit_ns) {
@@ -786,7 +838,7 @@ __global__ void bounded_wait_probe_kernel(uint32_t* status, uint64_t limit_ns) {
 
 cudaError_t launch_bounded_wait_probe(uint32_t* status, uint64_t limit_ns, cudaStream_t stream) {
     bounded_wait_probe_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
-    ++g_launches;
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -869,6 +921,20 @@ static bool device_info(DeviceInfo** out) {
     return true;
 }
 
+cudaError_t launch_finish_sums(const int32_t* acc, int64_t ld_acc, int64_t M, int64_t N, const float* s_row, int32_t row_stride,
+                               const float* s_col, int32_t col_stride, float* out, int64_t ldo, int out_bf16, cudaStream_t stream) {
+    if (M == 0 || N == 0) return cudaSuccess;
+    DeviceInfo* dev = nullptr;
+    if (!device_info(&dev)) return cudaErrorUnknown;
+    const int vec = (uintptr_t)acc % 16 == 0 && ld_acc % 4 == 0 && (uintptr_t)out % (out_bf16 ? 8 : 16) == 0 && ldo % 4 == 0;
+    const int64_t work = M * ((N + 3) / 4), blocks = (work + 255) / 256;
+    const unsigned grid = (unsigned)(blocks < 16 * (int64_t)dev->sms ? blocks : 16 * (int64_t)dev->sms);
+    launch_pdl(finish_sums_kernel, dim3(grid), dim3(256), 0, stream, acc, ld_acc, M, N, s_row, row_stride, s_col, col_stride, out, ldo,
+               vec, out_bf16);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // Which tiles are split, and into how many parts.  `groups` tiles run at a time.  Too few tiles to fill
 // the machine: all of them are split.  Several rounds of tiles with a last, partly empty round: only
 // the tiles of that round are split, so that it takes a fraction of a round.  Each part keeps at least
@@ -914,6 +980,8 @@ static cudaError_t launch_kernel(unsigned groups, const CUtensorMap& map_a, cons
 
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream) {
     if (g.opt.accumulate == 2 && (g.acc_out == nullptr || g.kind != 0)) return SRQ_ERR_INVALID_ARG;   // int32 sums need their matrix
+    if (g.opt.raw_sums && (g.kind != 0 || !g.out || g.acc_out || g.opt.accumulate || g.opt.out_bf16 || g.opt.requant || g.opt.absmax_bits))
+        return SRQ_ERR_UNSUPPORTED;                       // the sums are the only result of such a call
     if (g.M == 0 || g.N == 0) return SRQ_OK;
     DeviceInfo* dev = nullptr;
     if (!device_info(&dev)) return SRQ_ERR_CUDA;
@@ -960,7 +1028,7 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     // (a row must also END on a 16-byte boundary: a store that reaches over the edge of the tensor map
     // was seen to write the whole last 16-byte piece of the row, into the columns of a wider buffer)
     P.tma_out = P.write_out && P.vec_out && g.N % out_vec_elems == 0 && !g.acc_out && g.M < (1ll << 31) && g.N < (1ll << 31) &&
-                encode_output(&map_out, g.out, g.opt.out_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.M, g.N, g.ldo);
+                encode_output(&map_out, g.out, g.opt.out_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : g.opt.raw_sums ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, g.M, g.N, g.ldo);
     if (P.splits > 1 && !encode_output(&map_part, P.part, CU_TENSOR_MAP_DATA_TYPE_INT32, split_tiles * BM * ctas, BN, BN))
         return SRQ_ERR_CUDA;
 
@@ -973,7 +1041,7 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
                                         : launch_kernel<1, 1>(groups, map_a, map_b, map_out, map_part, P, stream);
     else e = ctas == 2 ? launch_kernel<2, 2>(groups, map_a, map_b, map_out, map_part, P, stream)
                        : launch_kernel<1, 2>(groups, map_a, map_b, map_out, map_part, P, stream);
-    ++g_launches;
+    count_launch();
     if (e != cudaSuccess) return SRQ_ERR_CUDA;
     if (P.splits > 1) {
         const int vec = g.ldo % 4 == 0 && (uintptr_t)g.out % 16 == 0;     // 16-byte (binary32) or 8-byte (bfloat16) stores
@@ -982,8 +1050,8 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
         const unsigned grid = (unsigned)(blocks < 8 * (int64_t)dev->sms ? blocks : 8 * (int64_t)dev->sms);
         launch_pdl(dequant_kernel, dim3(grid), dim3(256), 0, stream, P.part, split_tiles, P.full_tiles, P.tiles_n, BM * ctas, g.M, g.N, g.s_row,
                                                  g.row_stride, g.s_col, g.col_stride, g.out, g.ldo, g.acc_out, vec,
-                                                 g.opt.accumulate, g.opt.out_bf16, status);
-        ++g_launches;
+                                                 g.opt.accumulate, g.opt.out_bf16, g.opt.raw_sums, status);
+        count_launch();
         if (cudaGetLastError() != cudaSuccess) return SRQ_ERR_CUDA;
     }
     return SRQ_OK;

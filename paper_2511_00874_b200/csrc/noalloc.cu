@@ -59,11 +59,10 @@ extern "C" srq_status_t sr_quantize_static(const void* x, srq_dtype_t dt, int64_
                                            int8_t* codes_tr, int64_t ld_tr, float* scale_tr, uint32_t* device_status,
                                            void* cuda_stream) {
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (!x || !q || rows < 0 || cols < 0 || ld < cols) return SRQ_ERR_INVALID_ARG;
+    if (!x || rows < 0 || cols < 0 || ld < cols) return SRQ_ERR_INVALID_ARG;
     if (dt != SRQ_F32 && dt != SRQ_BF16) return SRQ_ERR_INVALID_ARG;
-    if (q->bits < 2 || q->bits > 8) return SRQ_ERR_UNSUPPORTED;
-    if (q->scale != SRQ_PER_TENSOR && q->scale != SRQ_PER_ROW) return SRQ_ERR_INVALID_ARG;
-    if (q->round != SRQ_SR && q->round != SRQ_RTN) return SRQ_ERR_INVALID_ARG;
+    const srq_status_t sq = check_qspec(q);            // the same rules as sr_quantize: grid, widths, modes, absmax pointer
+    if (sq != SRQ_OK) return sq;
     if (!codes_rm && !codes_tr) return SRQ_ERR_INVALID_ARG;
     if (codes_rm && (!scale_rm || ld_rm < cols)) return SRQ_ERR_INVALID_ARG;
     if (codes_tr && (!scale_tr || ld_tr < rows)) return SRQ_ERR_INVALID_ARG;
@@ -79,7 +78,7 @@ extern "C" srq_status_t sr_quantize_static(const void* x, srq_dtype_t dt, int64_
         if (cudaMemsetAsync(status, 0, sizeof(uint32_t), st) != cudaSuccess) return SRQ_ERR_CUDA;
     } else {
         clear_static_status<<<1, 1, 0, st>>>();
-        ++g_launches;
+        count_launch();
         if (cudaGetLastError() != cudaSuccess) return SRQ_ERR_CUDA;
     }
 

@@ -23,7 +23,7 @@
 
 namespace srq {
 
-unsigned long long g_launches = 0;
+std::atomic<unsigned long long> g_launches{0};
 
 // ------------------------------------------------------------------------------------------
 // scratch carving
@@ -728,11 +728,12 @@ quantize_rows_warp_kernel(const T* __restrict__ x, const __grid_constant__ Quant
 template <typename T, int MODE, int GW>
 static void launch_rows_warp_one(const T* p, const QuantParams& P, float* delta_out, float qmax, uint32_t* status,
                                  int sms, cudaStream_t st) {
-    static int per_sm = 0;
+    static std::atomic<int> cached{0};              // resident CTAs per SM, asked once (any thread may be first)
+    int per_sm = cached.load(std::memory_order_relaxed);
     if (per_sm == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_rows_warp_kernel<T, MODE, GW>, Q_THREADS, 0) != cudaSuccess || n < 1) n = 1;
-        per_sm = n;
+        cached.store(per_sm = n, std::memory_order_relaxed);
     }
     const int64_t resident = (int64_t)sms * per_sm;
     const int64_t need = (P.rows + Q_THREADS / 32 - 1) / (Q_THREADS / 32);
@@ -756,11 +757,12 @@ static void launch_rows_warp_g(int gw, const void* x, const QuantParams& P, floa
 template <typename T, int MODE, int G>
 static void launch_rows_one(const T* p, const QuantParams& P, float* delta_out, float qmax, uint32_t* status,
                             int sms, cudaStream_t st) {
-    static int per_sm = 0;
+    static std::atomic<int> cached{0};
+    int per_sm = cached.load(std::memory_order_relaxed);
     if (per_sm == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_rows_kernel<T, MODE, G>, Q_THREADS, 0) != cudaSuccess || n < 1) n = 1;
-        per_sm = n;
+        cached.store(per_sm = n, std::memory_order_relaxed);
     }
     const int64_t resident = (int64_t)sms * per_sm;
     const unsigned grid = (unsigned)(P.rows < resident ? P.rows : resident);
@@ -931,7 +933,7 @@ cudaError_t launch_widen_codes(const int8_t* codes, int64_t rows, int64_t cols, 
     const int64_t n = rows * cols;
     const unsigned grid = (unsigned)(n / 256 + 1 < 4096 ? n / 256 + 1 : 4096);
     launch_pdl(widen_codes_kernel, dim3(grid), dim3(256), 0, stream, codes, rows, cols, ld, (uint16_t*)out_bf16, ld_out, one);
-    ++g_launches;
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -941,7 +943,7 @@ cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t c
     const ScaleStep none = {};
     if (dt == SRQ_F32) launch_amax<float>(x, rows, cols, ld, (uint32_t*)absmax, false, nullptr, false, none, stream);
     else launch_amax<__nv_bfloat16>(x, rows, cols, ld, (uint32_t*)absmax, false, nullptr, false, none, stream);
-    ++g_launches;
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -954,20 +956,21 @@ cudaError_t launch_absmax_cols(const void* x, srq_dtype_t dt, int64_t rows, int6
     const ScaleStep none = {};
     if (dt == SRQ_F32) launch_amax<float>(x, rows, cols, ld, nullptr, false, (uint32_t*)absmax_cols, true, none, stream);
     else launch_amax<__nv_bfloat16>(x, rows, cols, ld, nullptr, false, (uint32_t*)absmax_cols, true, none, stream);
-    ++g_launches;
+    count_launch();
     return cudaGetLastError();
 }
 
 // SM count of the current device (asked once per device).
 static int sm_count() {
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];             // zero-initialised; any thread may fill an entry
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-    if (cached[dev] == 0) {
-        int n = 0;
-        cached[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        n = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+        cached[dev].store(n, std::memory_order_relaxed);
     }
-    return cached[dev];
+    return n;
 }
 
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream, bool scratch_zeroed) {
@@ -1020,7 +1023,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     // per-row steps and row-major codes only: one pass (rows of 512 .. 8192 elements)
     if (per_row && want_rm && !want_tr && fast && !sr8 && cols >= 512 && cols <= (int64_t)ROWQ_MAX_G * Q_THREADS * 4) {
         launch_rows(a.dt, P.mode, a.x, P, a.scale_rm, qmax, status, sm_count(), stream);
-        ++g_launches;
+        count_launch();
         return cudaGetLastError();
     }
 
@@ -1034,13 +1037,13 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
             const ScaleStep none = {};
             if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, amax_rm, true, nullptr, false, none, stream);
             else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, amax_rm, true, nullptr, false, none, stream);
-            ++g_launches;
+            count_launch();
         }
         const uint32_t* col_bits = (const uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
         const int64_t n = n0 > n1 ? n0 : n1;
         launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
             amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr, col_bits, n1, inv_tr, a.scale_tr, qmax, status);
-        ++g_launches;
+        count_launch();
     } else if (given) {
         amax_rm = amax_tr = (uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
         const int64_t n = n0 > n1 ? n0 : n1;
@@ -1048,7 +1051,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
             amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
             amax_tr, n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status);
-        ++g_launches;
+        count_launch();
     } else {
         if (!scratch_zeroed) {
             cudaError_t e = cudaMemsetAsync(s.counter, 0, (size_t)((char*)s.inv_rm - (char*)s.counter), stream);
@@ -1062,14 +1065,14 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         const bool want_rows = per_row && want_rm, want_cols = per_row && want_tr;
         if (a.dt == SRQ_F32) launch_amax<float>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, S, stream);
         else launch_amax<__nv_bfloat16>(a.x, rows, cols, a.ld, amax_rm, want_rows, amax_tr, want_cols, S, stream);
-        ++g_launches;
+        count_launch();
         if (!few) {
             const int64_t n = n0 > n1 ? n0 : n1;
             const int threads = 256;
             launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
                 amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
                 amax_tr, n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status);
-            ++g_launches;
+            count_launch();
         }
     }
     {
@@ -1077,7 +1080,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         if (fast) launch_fast(a.dt, P.mode, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);
         else if (a.dt == SRQ_F32) launch_pdl(quantize_kernel<float>, dim3(grid), dim3(Q_THREADS), 0, stream, (const float*)a.x, P);
         else launch_pdl(quantize_kernel<__nv_bfloat16>, dim3(grid), dim3(Q_THREADS), 0, stream, (const __nv_bfloat16*)a.x, P);
-        ++g_launches;
+        count_launch();
     }
     return cudaGetLastError();
 }

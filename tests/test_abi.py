@@ -77,6 +77,57 @@ def test_host_side_argument_checks_need_no_device(L):
     assert r(fake, 0, 8, 8, 8, ctypes.byref(q), fake, 8, fake, None, 0, None, fake, 16, None) == binding.ERR_WORKSPACE
 
 
+def test_the_static_entry_point_applies_the_same_checks_before_anything_is_enqueued(L):
+    fake = 4096
+    f = L.sr_quantize_static
+    r = lambda q, x=fake: int(f(x, 0, 8, 8, 8, ctypes.byref(q), fake, 8, fake, None, 0, None, None, None))
+    assert r(binding.QSpec(format=7).c()) == binding.ERR_INVALID_ARG                 # unknown grid
+    assert r(binding.QSpec(format=binding.GRID_NONE).c()) == binding.ERR_INVALID_ARG  # a quantizer needs a grid
+    assert r(binding.QSpec(bits=4, format=binding.GRID_E4M3).c()) == binding.ERR_UNSUPPORTED   # below E4M0
+    assert r(binding.QSpec(round=binding.SR8, format=binding.GRID_E4M3).c()) == binding.ERR_UNSUPPORTED
+    assert r(binding.QSpec(round=9).c()) == binding.ERR_INVALID_ARG
+    q = binding.QSpec().c()
+    q.absmax = fake + 2                                                               # misaligned known maximum
+    assert r(q) == binding.ERR_INVALID_ARG
+    assert r(binding.QSpec().c(), fake + 4) == binding.ERR_INVALID_ARG                # misaligned input
+    assert int(f(fake, 0, 8, 8, 8, None, fake, 8, fake, None, 0, None, None, None)) == binding.ERR_INVALID_ARG
+
+
+def test_dequant_i32_and_raw_sums_checks(L):
+    fake = 4096
+    d = L.srq_dequant_i32
+    assert int(d(None, 8, 8, 8, fake, 0, fake, 0, fake, 8, 0, None)) == binding.ERR_INVALID_ARG
+    assert int(d(fake, 4, 8, 8, fake, 0, fake, 0, fake, 8, 0, None)) == binding.ERR_INVALID_ARG      # pitch < N
+    assert int(d(fake, 8, 8, 8, fake, 2, fake, 0, fake, 8, 0, None)) == binding.ERR_INVALID_ARG      # stride not 0 / 1
+    assert int(d(fake, 8, 8, 8, fake, 0, fake, 0, fake + 2, 8, 0, None)) == binding.ERR_INVALID_ARG  # fp32 output misaligned
+    assert int(d(fake, 8, 8, 8, fake, 0, fake, 0, fake, 8, 3, None)) == binding.ERR_INVALID_ARG
+    assert int(d(fake, 8, 0, 8, fake, 0, fake, 0, fake, 8, 0, None)) == binding.OK                   # nothing to do
+    o = binding._Output(1, 0, None, None, None, 0, None, 1)                                         # accumulate + raw sums
+    g = L.srq_gemm_i8_ex
+    assert int(g(fake, 32, fake, 32, 8, 8, 24, fake, 0, fake, 0, fake, 8, None, ctypes.byref(o), fake, 4096, None)) == binding.ERR_UNSUPPORTED
+
+
+def test_every_kernel_waits_for_its_predecessor_first():
+    """Kernels are launched as programmatic dependents of the kernel before them, which is only
+    correct if a kernel's first act is the wait (pdl_enter).  Every __global__ function in the
+    sources must therefore start with it, except those only ever launched the ordinary way."""
+    src_dir = os.path.join(ROOT, "paper_2511_00874_b200", "csrc")
+    plain_only = {"bounded_wait_probe_kernel", "clear_static_status"}      # launched with <<< >>>, no attribute
+    seen = 0
+    for name in sorted(os.listdir(src_dir)):
+        text = open(os.path.join(src_dir, name)).read()
+        for m in re.finditer(r"__global__\s+void(?:\s+__launch_bounds__\([^)]*(?:\([^)]*\))?[^)]*\))?\s+(\w+)\s*\(", text):
+            kernel = m.group(1)
+            body = text.index("{", m.end())
+            first = text[body + 1:].lstrip().split("\n", 1)[0].strip()
+            seen += 1
+            if kernel in plain_only:
+                assert ("launch_pdl(" + kernel) not in text, kernel
+                continue
+            assert first == "pdl_enter();", f"{name}: {kernel} starts with {first!r}"
+    assert seen >= 12
+
+
 def test_layer_calls_check_overflow_and_workspace_on_the_host(L):
     q8 = binding.QSpec(bits=8).c()
     q4 = binding.QSpec(bits=4).c()
