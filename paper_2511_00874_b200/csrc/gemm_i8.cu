@@ -5,7 +5,7 @@
 //   acc[i,j] = sum_k a[i,k] * b[j,k]          int8 x int8 -> int32, exact
 //   out[i,j] = float(acc[i,j]) * (s_row[i] * s_col[j])
 //
-// Persistent kernel, one CTA per SM, 6 warps.  Two forms of the same code (template CTAS):
+// Persistent kernel, one CTA per SM, 10 warps.  Two forms of the same code (template CTAS):
 //   CTAS = 2  two CTAs on neighbouring SMs (a cluster) share one 256 x 256 output tile: each stages
 //             its own 128 rows of a and 128 of the 256 rows of b, and the leader CTA issues
 //             tcgen05.mma.cta_group::2 (M256 x N256 x K32), which reads both CTAs' shared memory
@@ -14,15 +14,19 @@
 //   CTAS = 1  one CTA per 128 x 256 tile with tcgen05.mma.cta_group::1 (M128 x N256 x K32).
 // Roles:
 //   warp 0      TMA producer: 128-byte-swizzled tiles of a and b into a shared-memory ring
-//               (6 stages of 32 KB, or 4 of 48 KB), signalled through mbarriers; with CTAS = 2
+//               (5 stages of 32 KB, or 3 of 48 KB), signalled through mbarriers; with CTAS = 2
 //               both CTAs' loads complete on the leader's barrier (no multicast is used)
 //   warp 1      allocates TMEM; in the leader one thread issues the MMAs; accumulators live in
 //               TMEM, two buffers of 256 columns, so the tensor pipe starts the next tile while
 //               the previous one is being drained
-//   warps 2-5   epilogue: tcgen05.ld the accumulator (one TMEM lane quarter per warp), convert,
-//               scale and store (through shared memory and TMA block stores); or, for a split
-//               contraction, add the exact int32 partial sums into a zeroed workspace (TMA block
-//               reductions), which dequant_kernel scales afterwards
+//   warps 2-9   epilogue, two groups of four warps: group g drains accumulator buffer g, i.e. every
+//               other tile of this CTA, so that one group is in the middle of its block stores
+//               while the other is between tiles and the store queue never runs dry (on
+//               output-bound shapes the stores, not the tensor pipe, decide the time).  A warp
+//               takes one TMEM lane quarter: tcgen05.ld, convert, scale and store (through shared
+//               memory and TMA block stores); or, for a split contraction, add the exact int32
+//               partial sums into a zeroed workspace (TMA block reductions), which dequant_kernel
+//               scales afterwards
 // Ragged edges rely on TMA zero fill for loads and on bounds checks for stores.
 // Every wait is bounded by a wall-clock limit; on expiry the CTA records SRQ_ERR_TIMEOUT,
 // stops issuing work, waits (bounded) for what it has in flight, frees its TMEM and returns.
@@ -39,7 +43,8 @@ constexpr int BM = 128, BN = 256, BK = 128;          // per-CTA rows, tile colum
 constexpr int UMMA_K = 32;                             // bytes of K per tcgen05.mma.kind::i8
 constexpr int A_STAGE_BYTES = BM * BK;
 constexpr int TMEM_COLS = 512;                         // two accumulator buffers of BN columns
-constexpr int GEMM_THREADS = 192;
+constexpr int EPI_GROUPS = 2;                          // epilogue warp groups; group g drains accumulator buffer g
+constexpr int GEMM_THREADS = 64 + 128 * EPI_GROUPS;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;      // 2 s
 
 template <int CTAS>
@@ -47,7 +52,7 @@ struct Cfg {
     static constexpr int B_ROWS = BN / CTAS;                         // rows of b staged by each CTA
     static constexpr int B_STAGE_BYTES = B_ROWS * BK;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int STAGES = CTAS == 1 ? 4 : 6;
+    static constexpr int STAGES = CTAS == 1 ? 3 : 5;
 };
 
 template <int STAGES>
@@ -55,12 +60,12 @@ struct SharedTail {                                    // after the stage ring
     uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain;
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
-    alignas(16) float s_col[2][BN];   // read as float4
+    alignas(16) float s_col[2 * EPI_GROUPS][BN];   // read as float4; two per epilogue group, used in turn
 };
 constexpr int OUT_STAGE_BYTES = 32 * 32 * 4;           // one 32 x 32 block of 32-bit results per epilogue warp
 template <int CTAS>
 constexpr size_t gemm_smem() {
-    return 1024 /*alignment slack*/ + (size_t)Cfg<CTAS>::STAGES * Cfg<CTAS>::STAGE_BYTES + 4 * OUT_STAGE_BYTES +
+    return 1024 /*alignment slack*/ + (size_t)Cfg<CTAS>::STAGES * Cfg<CTAS>::STAGE_BYTES + 4 * EPI_GROUPS * OUT_STAGE_BYTES +
            sizeof(SharedTail<Cfg<CTAS>::STAGES>);
 }
 
@@ -370,7 +375,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // the dynamic window starts at the same offset in every CTA, so the aligned layouts coincide
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* out_stage = smem + (size_t)STAGES * STAGE_BYTES;          // 1024-byte aligned, 4 KB per epilogue warp
-    Tail* T = (Tail*)(out_stage + 4 * OUT_STAGE_BYTES);
+    Tail* T = (Tail*)(out_stage + 4 * EPI_GROUPS * OUT_STAGE_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = CTAS == 1 ? 0u : cluster_ctarank();   // position in the CTA pair
     const bool leader = rank == 0;
@@ -479,7 +484,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;                    // TMEM lanes this warp may read
-        const int etid = threadIdx.x - 64;               // 0..127 within the epilogue group
+        const int egrp = (warp - 2) >> 2;                // this warp's group: it takes the units that use accumulator buffer egrp
+        const int etid = (threadIdx.x - 64) & 127;       // 0..127 within the epilogue group
         // the MMA issuer's barriers (in the leader CTA)
         const uint32_t empty_bar0 = CTAS == 1 ? smem_u32(&T->tmem_empty[0]) : map_to_cta(smem_u32(&T->tmem_empty[0]), 0);
         const uint32_t empty_bar1 = CTAS == 1 ? smem_u32(&T->tmem_empty[1]) : map_to_cta(smem_u32(&T->tmem_empty[1]), 0);
@@ -519,28 +525,31 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             sr_next = (row < P.M) ? __ldg(P.s_row + row * P.row_stride) : 0.0f;
         };
-        if (group < units) fetch_steps(group);
-        for (int64_t u = group; u < units && ok; u += groups, ++lt) {
+        // the MMA warp alternates the two accumulators unit by unit, so group g owns this CTA's units g, g + 2, ...
+        const int64_t u_first = group + (int64_t)egrp * groups, u_step = (int64_t)EPI_GROUPS * groups;
+        if (u_first < units) fetch_steps(u_first);
+        for (int64_t u = u_first; u < units && ok; u += u_step, ++lt) {
             const int64_t tile = tile_next;
             const int32_t tn = tn_next, tm = tm_next;
             const bool whole = u < P.full_tiles;              // this unit holds the complete sums of its tile
-            const uint32_t buf = lt & 1u, use = lt >> 1;
+            const uint32_t buf = (uint32_t)egrp, use = lt;
             const int64_t row0 = ((int64_t)tm * CTAS + rank) * BM;      // first row of this CTA's half
             const int64_t row = row0 + quarter * 32 + lane;
             const int64_t col_base = (int64_t)tn * BN;
-            // stage this tile's column step sizes (the other buffer may still be read by slower warps;
-            // this one was last read two tiles ago, which every warp has left)
-            T->s_col[buf][etid] = sc_next[0];
-            T->s_col[buf][etid + 128] = sc_next[1];
+            // stage this tile's column step sizes (the group's other buffer may still be read by slower
+            // warps; this one was last read two of the group's tiles ago, which every warp has left)
+            const uint32_t cbuf = (uint32_t)egrp * 2u + (lt & 1u);
+            T->s_col[cbuf][etid] = sc_next[0];
+            T->s_col[cbuf][etid + 128] = sc_next[1];
             const float sr = sr_next;
-            if (u + groups < units) fetch_steps(u + groups);
+            if (u + u_step < units) fetch_steps(u + u_step);
             bool mine = mbar_wait(&T->tmem_full[buf], use & 1u, &T->abort_flag);
             if (!mine) give_up(T, P.status);
-            // the four warps must leave together (they share named barrier 1): one barrier makes the
+            // the four warps of a group must leave together (they share named barrier 1 + group): one barrier makes the
             // staged step sizes visible and tells every thread whether any of them gave up
             uint32_t any_gave_up;
-            asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.or.pred p, 1, 128, q;\nselp.u32 %0, 1, 0, p;\n}"
-                         : "=r"(any_gave_up) : "r"((uint32_t)(!mine || T->abort_flag != 0u)) : "memory");
+            asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.or.pred p, %2, 128, q;\nselp.u32 %0, 1, 0, p;\n}"
+                         : "=r"(any_gave_up) : "r"((uint32_t)(!mine || T->abort_flag != 0u)), "r"(1 + egrp) : "memory");
             if (any_gave_up) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
@@ -557,7 +566,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         uint32_t v[32];
                         tmem_ld32(taddr + j * 64 + h * 32, v);
                         tmem_ld_wait();
-                        const float* sc = &T->s_col[buf][j * 64 + h * 32];
+                        const float* sc = &T->s_col[cbuf][j * 64 + h * 32];
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             v[i] = __float_as_uint(__fmul_rn(acc_to_float<KIND>(v[i]), __fmul_rn(sr, sc[i])));
@@ -583,7 +592,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     uint32_t v[32];
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
-                    const float* sc = &T->s_col[buf][j * 32];
+                    const float* sc = &T->s_col[cbuf][j * 32];
                     if (!P.opt.raw_sums) {                    // raw sums leave as the int32 words they are
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
@@ -618,7 +627,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     tmem_ld_wait();
                     const int64_t col0 = col_base + j * 32;
                     if (row < P.M && col0 < P.N) {
-                        const float* sc = &T->s_col[buf][j * 32];
+                        const float* sc = &T->s_col[cbuf][j * 32];
                         if (P.acc_out) {
                             int32_t* ad = P.acc_out + row * P.N + col0;
                             if (P.opt.accumulate == 2) {
