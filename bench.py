@@ -450,6 +450,24 @@ def run_ours(args):
         s_clocks = s_sampler.stop()
         s_achieved = ops_per_launch / (s_ms3 / 3.0 * 1e-3) / 1e12
         peak_sus = 2.0 * peaks["bf16_sustained"]
+        # the tensor pipe on its own: the same instruction on operands resident in shared memory, no global
+        # traffic (single launches, then two seconds back to back)
+        mws = srq.new_workspace(256, dev)
+        kb = 2048                                # about the duration of one product launch
+        mma_ops = srq.srq_selftest_mma_rate(mws, kb)
+        torch.cuda.synchronize()
+        time.sleep(1.0)
+        m_evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+        for m0, m1 in m_evs:
+            m0.record()
+            srq.srq_selftest_mma_rate(mws, kb)
+            m1.record()
+        torch.cuda.synchronize()
+        mma_burst = mma_ops / (statistics.mean(m0.elapsed_time(m1) for m0, m1 in m_evs) * 1e-3) / 1e12
+        mm_ms, _ = _timed_loop(lambda _i: srq.srq_selftest_mma_rate(mws, kb), 2.0, mma_ops / (mma_burst * 1e12) * 1e3, torch)
+        mma_sus = mma_ops / (mm_ms * 1e-3) / 1e12
+        if srq.srq_poll_status(mws) != 0:
+            raise SystemExit("tensor-pipe microbenchmark reported a device-side condition")
         result["roofline"] = {
             "bound": "tensor", "kernel": "gemm_i8_kernel", "achieved": achieved, "peak": peak_burst, "unit": "TOPS",
             "frac": achieved / peak_burst, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
@@ -460,8 +478,13 @@ def run_ours(args):
             "frac_of_nominal_4500": achieved / 4500.0,
             "ms_per_launch": {"fwd": gemm_ms[0], "bwd_input": gemm_ms[1], "bwd_weight": gemm_ms[2]},
             "ops_per_launch": ops_per_launch, "clocks": b_clocks,
+            "mma_only": {"burst_tops": mma_burst, "sustained_tops": mma_sus,
+                         "what": "tcgen05.mma.cta_group::2.kind::i8 M256 N256 K32 on operands resident in shared memory, "
+                                 "no global traffic (srq_selftest_mma_rate): the pipe's own ceiling at the clock the power limit allows"},
+            "frac_of_mma_only": achieved / mma_burst,
             "sustained": {"achieved": s_achieved, "peak": peak_sus, "frac": s_achieved / peak_sus,
                           "ms_per_launch": s_ms3 / 3.0, "launches": 3 * s_n, "clocks": s_clocks,
+                          "frac_of_mma_only": s_achieved / mma_sus,
                           "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS TFLOP/s",
                           "regime": "the three products back to back for two seconds (power cap)"}}
         del cA, cAt, cW, cWt, cdY, cdYt

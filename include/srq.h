@@ -370,6 +370,16 @@ void srq_plan_splits(int64_t tiles, int32_t k_blocks, int32_t groups, int32_t *f
  * SRQ_ERR_TIMEOUT (read it with srq_poll_status), the kernel returns and the context stays usable. */
 srq_status_t srq_selftest_bounded_wait(void *ws, size_t ws_bytes, uint32_t limit_us, void *cuda_stream);
 
+/* Measurement aid, not part of the layer: the issue rate of the tensor pipe for the instruction the
+ * products use (tcgen05.mma.cta_group::2.kind::i8, M256 N256 K32).  Every CTA pair of the device
+ * multiplies operand blocks that already sit in its shared memory, k_blocks (1 .. 2^22) blocks of 128
+ * bytes of contraction, into TMEM; nothing moves through global memory.  *ops (host, optional)
+ * receives the integer operations of the launch (2 * 256 * 256 * 128 per pair and block); time the
+ * launch on the stream and divide.  This is the ceiling the main loop of the products is compared
+ * with: the kind::i8 pipe at the clock the power limit allows, with no data movement at all.  The
+ * status word of ws reports a wait that ran out (SRQ_ERR_TIMEOUT), as in the product kernel. */
+srq_status_t srq_selftest_mma_rate(void *ws, size_t ws_bytes, int32_t k_blocks, int64_t *ops, void *cuda_stream);
+
 /* Static, human-readable name of a status. */
 const char *srq_status_string(srq_status_t s);
 

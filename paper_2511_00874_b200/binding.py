@@ -28,7 +28,7 @@ GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
            "sr_quantize", "sr_quantize_static", "srq_absmax", "srq_absmax_cols", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
            "srq_gemm_i8_ex", "qlinear_fwd_ex", "qlinear_bwd_ex", "srq_dequant_i32",
-           "srq_poll_status", "srq_status_string", "srq_launch_count", "srq_selftest_bounded_wait", "srq_plan_splits"]
+           "srq_poll_status", "srq_status_string", "srq_launch_count", "srq_selftest_bounded_wait", "srq_selftest_mma_rate", "srq_plan_splits"]
 
 
 class SrqError(RuntimeError):
@@ -123,6 +123,8 @@ def lib() -> ctypes.CDLL:
     L.srq_dequant_i32.restype = ctypes.c_int
     L.srq_selftest_bounded_wait.argtypes = [vp, sz, ctypes.c_uint32, vp]
     L.srq_selftest_bounded_wait.restype = ctypes.c_int
+    L.srq_selftest_mma_rate.argtypes = [vp, sz, i32, ctypes.POINTER(i64), vp]
+    L.srq_selftest_mma_rate.restype = ctypes.c_int
     L.srq_plan_splits.argtypes = [i64, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.srq_plan_splits.restype = None
     L.srq_poll_status.argtypes = [vp, vp]
@@ -483,6 +485,15 @@ def srq_plan_splits(tiles: int, k_blocks: int, groups: int):
 def srq_selftest_bounded_wait(ws: torch.Tensor, limit_us: int = 1000) -> None:
     """Enqueues the bounded-wait self-test; srq_poll_status(ws) then returns ERR_TIMEOUT."""
     _check(lib().srq_selftest_bounded_wait(ws.data_ptr(), ws.numel(), int(limit_us), _stream()), "srq_selftest_bounded_wait")
+
+
+def srq_selftest_mma_rate(ws: torch.Tensor, k_blocks: int) -> int:
+    """Enqueues the tensor-pipe issue-rate microbenchmark (operands resident in shared memory, no
+    global traffic); returns the integer operations of the launch.  Time it with CUDA events."""
+    ops = ctypes.c_int64(0)
+    _check(lib().srq_selftest_mma_rate(ws.data_ptr(), ws.numel(), int(k_blocks), ctypes.byref(ops), _stream()),
+           "srq_selftest_mma_rate")
+    return int(ops.value)
 
 
 def srq_poll_status(ws: torch.Tensor) -> int:

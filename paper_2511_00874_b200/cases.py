@@ -3,6 +3,7 @@
     python -m paper_2511_00874_b200.cases quantize --rows 16384 --cols 4096 --dtype f32
     python -m paper_2511_00874_b200.cases gemm --M 8192 --N 4096 --K 4096
     python -m paper_2511_00874_b200.cases layer --T 16384 --N 2304 --K 768
+    python -m paper_2511_00874_b200.cases mma-peak --k-blocks 2048 --seconds 2
 
     python -m paper_2511_00874_b200.cases sweep --config 3
 
@@ -91,6 +92,29 @@ def case_gemm(a):
     ops = 2.0 * a.M * a.N * a.K
     return {"op": "srq_gemm_e4m3" if getattr(a, "grid", "int") == "e4m3" else "srq_gemm_i8", "M": a.M, "N": a.N, "K": a.K, "ms": med, "ms_best": best, "TOPS": ops / med / 1e9,
             "out": "bf16" if out_bf16 else "f32", "out_GBps": out.element_size() * a.M * a.N / med / 1e6}
+
+
+def case_mma_peak(a):
+    """The ceiling of the tensor pipe for the products' instruction (kind::i8, CTA pairs, M256 N256 K32):
+    operands resident in shared memory, no global traffic.  `ms` is the median of single launches
+    (burst clocks); with --seconds S the launch is also repeated back to back for S seconds, which
+    is what the power limit sustains."""
+    ws = B.new_workspace(256)
+    ops = B.srq_selftest_mma_rate(ws, a.k_blocks)
+    med, best = _time(lambda: B.srq_selftest_mma_rate(ws, a.k_blocks), a.iters, a.warmup, flush=False)
+    assert B.srq_poll_status(ws) == 0
+    r = {"op": "mma-peak", "k_blocks": a.k_blocks, "ops_per_launch": ops, "ms": med, "ms_best": best, "TOPS": ops / med / 1e9}
+    if a.seconds > 0:
+        n = max(3, int(a.seconds * 1e3 / med))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            B.srq_selftest_mma_rate(ws, a.k_blocks)
+        e1.record()
+        torch.cuda.synchronize()
+        assert B.srq_poll_status(ws) == 0
+        r.update({"sustained_launches": n, "sustained_ms": e0.elapsed_time(e1) / n, "sustained_TOPS": ops * n / e0.elapsed_time(e1) / 1e9})
+    return r
 
 
 def _layer_fn(A, W, dY, q, Y, dA, dW, ws):
@@ -238,7 +262,7 @@ def case_sweep(a):
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     sub = ap.add_subparsers(dest="op", required=True)
-    for name in ("quantize", "gemm", "layer", "sweep"):
+    for name in ("quantize", "gemm", "layer", "sweep", "mma-peak"):
         p = sub.add_parser(name)
         p.add_argument("--iters", type=int, default=20)
         p.add_argument("--warmup", type=int, default=3)
@@ -263,14 +287,17 @@ def main(argv=None):
             p.add_argument("--graph", action="store_true", help="record the step in a CUDA graph and time its replay")
         if name == "sweep":
             p.add_argument("--config", type=int, required=True, choices=[2, 3, 4, 5])
-        if name not in ("gemm", "sweep"):
+        if name == "mma-peak":
+            p.add_argument("--k-blocks", dest="k_blocks", type=int, default=2048, help="128-byte blocks of contraction per CTA pair")
+            p.add_argument("--seconds", type=float, default=0.0, help="also repeat the launch back to back for this long")
+        if name not in ("gemm", "sweep", "mma-peak"):
             p.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
             p.add_argument("--scale", default="tensor", choices=["tensor", "row"])
             p.add_argument("--round", default="sr", choices=["sr", "rtn", "sr8"])
     a = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("a CUDA device is required (there is no CPU fallback)")
-    res = {"quantize": case_quantize, "gemm": case_gemm, "layer": case_layer, "sweep": case_sweep}[a.op](a)
+    res = {"quantize": case_quantize, "gemm": case_gemm, "layer": case_layer, "sweep": case_sweep, "mma-peak": case_mma_peak}[a.op](a)
     if res is not None:
         print(json.dumps(res))
 

@@ -538,6 +538,14 @@ srq_status_t srq_selftest_bounded_wait(void* ws, size_t ws_bytes, uint32_t limit
     return launch_bounded_wait_probe(&((WsHeader*)ws)->status, (uint64_t)limit_us * 1000ull, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
 }
 
+srq_status_t srq_selftest_mma_rate(void* ws, size_t ws_bytes, int32_t k_blocks, int64_t* ops, void* cuda_stream) {
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!ws || !aligned_to(ws, 256) || k_blocks < 1 || k_blocks > (1 << 22)) return SRQ_ERR_INVALID_ARG;
+    if (ws_bytes < sizeof(WsHeader)) return SRQ_ERR_WORKSPACE;
+    if (clear_header(ws, st) != cudaSuccess) return SRQ_ERR_CUDA;
+    return launch_mma_rate(k_blocks, &((WsHeader*)ws)->status, ops, st);
+}
+
 srq_status_t srq_poll_status(void* ws, void* cuda_stream) {
     if (!ws) return SRQ_ERR_INVALID_ARG;
     uint32_t v = 0;

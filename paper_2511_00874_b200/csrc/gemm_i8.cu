@@ -944,6 +944,84 @@ cudaError_t launch_finish_sums(const int32_t* acc, int64_t ld_acc, int64_t M, in
     return cudaGetLastError();
 }
 
+// Issue-rate microbenchmark of the tensor pipe: every CTA pair multiplies operand blocks that already sit
+// in shared memory (pseudo-random bytes, written once by the CTA itself), k_blocks times, with
+// tcgen05.mma.cta_group::2.kind::i8 M256 N256 K32 into its two TMEM accumulators.  Nothing is loaded
+// from or stored to global memory, so the time is what the kind::i8 pipe needs for those operations at
+// the clock the power cap allows: the ceiling the product kernel's main loop is compared with.  The
+// issuing thread stays at most two chunks of eight k-blocks ahead of the pipe (bounded waits).
+__global__ void __launch_bounds__(128, 1) mma_rate_kernel(int32_t k_blocks, uint32_t* status) {
+    pdl_enter();
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);    // a: 128 x 128 bytes, b: 128 x 128 bytes
+    __shared__ uint64_t done[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ volatile uint32_t abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool leader = cluster_ctarank() == 0;
+    for (uint32_t i = threadIdx.x; i < (uint32_t)(A_STAGE_BYTES + Cfg<2>::B_STAGE_BYTES) / 4; i += blockDim.x) {
+        uint32_t h = (i + 1u) * 2654435761u ^ (blockIdx.x * 40503u);     // any byte pattern that toggles the multipliers
+        h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+        reinterpret_cast<uint32_t*>(smem)[i] = h;
+    }
+    fence_async_smem();
+    if (threadIdx.x == 0) {
+        mbar_init(&done[0], 1); mbar_init(&done[1], 1);
+        abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (warp == 1) tmem_alloc<2>(&tmem_base_s, TMEM_COLS);
+    tc_fence_before();
+    cluster_sync();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    if (warp == 0 && lane == 0 && leader) {
+        const uint32_t idesc = make_idesc(0, BM * 2, BN);
+        const uint64_t da = make_smem_desc(smem_u32(smem)), db = make_smem_desc(smem_u32(smem) + A_STAGE_BYTES);
+        bool ok = true;
+        const int32_t chunks = (k_blocks + 7) / 8;
+        for (int32_t c = 0; c < chunks && ok; ++c) {
+            if (c >= 2 && !mbar_wait(&done[c & 1], (uint32_t)((c >> 1) - 1) & 1u, &abort_flag)) { ok = false; break; }
+            const uint32_t d_tmem = tmem_base + (uint32_t)((c >> 2) & 1) * BN;      // both accumulators take turns
+            const int32_t kb_end = min(8, k_blocks - 8 * c);
+            for (int32_t kb = 0; kb < kb_end; ++kb)
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k)
+                    umma<2, 0>(d_tmem, da + (uint64_t)((k * UMMA_K) >> 4), db + (uint64_t)((k * UMMA_K) >> 4), idesc, (c >= 8 || kb > 0 || k > 0) ? 1u : 0u);
+            umma_commit<2>(&done[c & 1], false);
+        }
+        // everything issued must have left the pipe before TMEM is freed
+        for (int32_t c = chunks > 2 ? chunks - 2 : 0; c < chunks && ok; ++c)
+            if (!mbar_wait(&done[c & 1], (uint32_t)(c >> 1) & 1u, &abort_flag)) ok = false;
+        if (!ok) record_status(status, SRQ_ERR_TIMEOUT);
+    }
+    __syncwarp();
+    tc_fence_before();
+    cluster_sync();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc<2>(tmem_base, TMEM_COLS);
+    }
+}
+
+srq_status_t launch_mma_rate(int32_t k_blocks, uint32_t* status, int64_t* ops, cudaStream_t stream) {
+    DeviceInfo* dev = nullptr;
+    if (!device_info(&dev)) return SRQ_ERR_CUDA;
+    if (dev->pairs <= 0) return SRQ_ERR_UNSUPPORTED;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)dev->pairs * 2); cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 1024 + A_STAGE_BYTES + Cfg<2>::B_STAGE_BYTES; cfg.stream = stream;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization; at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = pdl_allowed(stream) ? 2 : 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, mma_rate_kernel, k_blocks, status);
+    count_launch();
+    if (ops) *ops = (int64_t)dev->pairs * k_blocks * (2ll * (BM * 2) * BN * BK);
+    return e == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
+}
+
 // Which tiles are split, and into how many parts.  `groups` tiles run at a time.  Too few tiles to fill
 // the machine: all of them are split.  Several rounds of tiles with a last, partly empty round: only
 // the tiles of that round are split, so that it takes a fraction of a round.  Each part keeps at least

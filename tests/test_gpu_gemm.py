@@ -205,3 +205,16 @@ def test_random_products(case):
         assert np.array_equal(out.cpu().numpy(), ref), tag
     if pad:
         assert bool((full[:, N:] == 7.0).all()), tag + ": pad columns written"
+
+
+def test_tensor_pipe_microbenchmark_runs_and_counts_its_operations():
+    """The issue-rate microbenchmark (no global traffic) finishes with a clean status and reports
+    2 * 256 * 256 * 128 operations per CTA pair and k-block; odd counts take the short last chunk."""
+    ws = srq.new_workspace(256)
+    pairs = torch.cuda.get_device_properties(0).multi_processor_count // 2
+    for kb in (1, 7, 8, 9, 17, 64, 515):
+        ops = srq.srq_selftest_mma_rate(ws, kb)
+        assert srq.srq_poll_status(ws) == 0
+        assert ops > 0 and ops % (kb * 2 * 256 * 256 * 128) == 0 and ops // (kb * 2 * 256 * 256 * 128) <= pairs
+    with pytest.raises(srq.SrqError):
+        srq.srq_selftest_mma_rate(ws, 0)
