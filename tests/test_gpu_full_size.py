@@ -1,4 +1,5 @@
-"""Parity at the benchmark's full size and launch configuration.
+"""Parity at the full size and launch configuration of the benchmark and of every layer shape of the
+GPT-2-small and Llama-style workload families.
 
 Linear layer 4096 -> 4096 with 65536 tokens, fp32 inputs, 8-bit per-tensor SR: the workload
 `bench.py` times, called the way it calls it (no debug copies, so the products run as CTA pairs
@@ -56,6 +57,16 @@ CASES = {
     "bench": (65536, 4096, 4096, torch.float32, srq.PER_TENSOR, 8, 8),
     # the largest Llama-style layer of the per-row configuration: bf16, 8-bit forward, 4-bit backward
     "gate_up": (65536, 5632, 2048, torch.bfloat16, srq.PER_ROW, 8, 4),
+    # every other layer shape the workload families name, at its largest token count: other tile
+    # counts, split plans and tails (2304 = 9 x 256 columns, a 5632-long contraction, 768-wide outputs
+    # whose weight gradient splits the contraction over all CTA pairs)
+    "gpt2_qkv": (65536, 2304, 768, torch.float32, srq.PER_TENSOR, 8, 8),
+    "gpt2_proj": (65536, 768, 768, torch.float32, srq.PER_TENSOR, 8, 8),
+    "gpt2_fc1": (65536, 3072, 768, torch.float32, srq.PER_TENSOR, 8, 8),
+    "gpt2_fc2": (65536, 768, 3072, torch.float32, srq.PER_TENSOR, 8, 8),
+    "llama_qkv": (65536, 2560, 2048, torch.bfloat16, srq.PER_ROW, 8, 4),
+    "llama_o": (65536, 2048, 2048, torch.bfloat16, srq.PER_ROW, 8, 4),
+    "llama_down": (65536, 2048, 5632, torch.bfloat16, srq.PER_ROW, 8, 4),
 }
 
 
