@@ -122,17 +122,20 @@ srq_status_t run_layer(const Operand& a, const Operand& b, srq_dtype_t dt, float
     const Operand* ops[2] = {&a, &b};
     int8_t* codes[2];
     float* scales[2];
+    QuantArgs qargs[2];
+    QuantScratch qscr[2];
     for (int i = 0; i < 2; ++i) {
         const Operand& o = *ops[i];
         codes[i] = (int8_t*)(base + p.off_codes[i]);
         scales[i] = (float*)(base + p.off_scale[i]);
-        QuantArgs qa;
+        QuantArgs& qa = qargs[i];
         qa.x = o.x; qa.dt = dt; qa.rows = o.rows; qa.cols = o.cols; qa.ld = o.cols; qa.q = *o.q;
         qa.codes_rm = o.transposed ? nullptr : codes[i]; qa.ld_rm = p.pitch; qa.scale_rm = o.transposed ? nullptr : scales[i];
         qa.codes_tr = o.transposed ? codes[i] : nullptr; qa.ld_tr = p.pitch; qa.scale_tr = o.transposed ? scales[i] : nullptr;
-        if (Kc > 0 && launch_quantize(qa, carve_quant_scratch(base + p.off_scratch[i], o.rows, o.cols), status, st, true) != cudaSuccess)
-            return SRQ_ERR_CUDA;
+        qscr[i] = carve_quant_scratch(base + p.off_scratch[i], o.rows, o.cols);
     }
+    // both operands: one pair of launches when the problem is small, else operand by operand
+    if (Kc > 0 && launch_quantize_batch(qargs, qscr, 2, status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
     if (Kc == 0) {   // empty contraction: the product is zero
         if (!out || opt.accumulate) return SRQ_OK;
         const size_t eb = opt.out_bf16 ? 2 : 4;
@@ -283,24 +286,29 @@ srq_status_t run_bwd(const void* dY, const void* A, const void* W, srq_dtype_t d
     float* sc[4]; int8_t* cd[4];
     for (int i = 0; i < 4; ++i) { sc[i] = (float*)(base + p.off_scale[i]); cd[i] = (int8_t*)(base + p.off_codes[i]); }
 
+    QuantArgs qargs[3];
+    QuantScratch qscr[3];
+    int nq = 0;
     if (T > 0 && N > 0) {      // dY -> [T,N] codes for dA and [N,T] codes for dW, one read of dY
-        QuantArgs q; q.x = dY; q.dt = dt; q.rows = T; q.cols = N; q.ld = N; q.q = *qdY;
+        QuantArgs& q = qargs[nq]; q.x = dY; q.dt = dt; q.rows = T; q.cols = N; q.ld = N; q.q = *qdY;
         q.codes_rm = cd[0]; q.ld_rm = p.pitch_n; q.scale_rm = sc[0];
         q.codes_tr = cd[1]; q.ld_tr = p.pitch_t; q.scale_tr = sc[1];
-        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[0], T, N), status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
+        qscr[nq++] = carve_quant_scratch(base + p.off_scratch[0], T, N);
     }
     if (N > 0 && K > 0) {      // W -> [K,N]
-        QuantArgs q; q.x = W; q.dt = dt; q.rows = N; q.cols = K; q.ld = K; q.q = *qW;
+        QuantArgs& q = qargs[nq]; q.x = W; q.dt = dt; q.rows = N; q.cols = K; q.ld = K; q.q = *qW;
         q.codes_rm = nullptr; q.ld_rm = 0; q.scale_rm = nullptr;
         q.codes_tr = cd[2]; q.ld_tr = p.pitch_n; q.scale_tr = sc[2];
-        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[1], N, K), status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
+        qscr[nq++] = carve_quant_scratch(base + p.off_scratch[1], N, K);
     }
     if (T > 0 && K > 0) {      // A -> [K,T]
-        QuantArgs q; q.x = A; q.dt = dt; q.rows = T; q.cols = K; q.ld = K; q.q = *qA;
+        QuantArgs& q = qargs[nq]; q.x = A; q.dt = dt; q.rows = T; q.cols = K; q.ld = K; q.q = *qA;
         q.codes_rm = nullptr; q.ld_rm = 0; q.scale_rm = nullptr;
         q.codes_tr = cd[3]; q.ld_tr = p.pitch_t; q.scale_tr = sc[3];
-        if (launch_quantize(q, carve_quant_scratch(base + p.off_scratch[2], T, K), status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
+        qscr[nq++] = carve_quant_scratch(base + p.off_scratch[2], T, K);
     }
+    // all operands: one pair of launches when the problem is small, else operand by operand
+    if (nq > 0 && launch_quantize_batch(qargs, qscr, nq, status, st, true) != cudaSuccess) return SRQ_ERR_CUDA;
 
     // dA[T,K] = Q(dY)[T,N] . Q(W)^T[K,N]
     if (T > 0 && K > 0) {

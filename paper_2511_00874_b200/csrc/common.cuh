@@ -126,6 +126,11 @@ struct QuantArgs {
 cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& scratch, uint32_t* status,
                             cudaStream_t stream, bool scratch_zeroed = false);
 
+// The operands of one layer call (n <= 3, scratch blocks already zeroed): two launches for all of them
+// together where the problem is small, else launch_quantize for each.  Same results either way.
+cudaError_t launch_quantize_batch(const QuantArgs* a, const QuantScratch* s, int n, uint32_t* status, cudaStream_t stream,
+                                  bool scratch_zeroed);
+
 // max |x| of the whole matrix into *absmax (device float, overwritten).
 cudaError_t launch_absmax(const void* x, srq_dtype_t dt, int64_t rows, int64_t cols, int64_t ld, float* absmax, cudaStream_t stream);
 // absmax_cols[c] = max over the rows of |x[r, c]| (device [cols], overwritten).

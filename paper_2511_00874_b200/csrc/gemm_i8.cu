@@ -526,13 +526,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             sr_next = (row < P.M) ? __ldg(P.s_row + row * P.row_stride) : 0.0f;
         };
         // the MMA warp alternates the two accumulators unit by unit, so group g owns this CTA's units g, g + 2, ...
-        const int64_t u_first = group + (int64_t)egrp * groups, u_step = (int64_t)EPI_GROUPS * groups;
+        // A launch in which no CTA has more than one unit is all latency: there both groups drain that
+        // one unit, half of its columns each.
+        const bool share = units <= groups;
+        const int64_t u_first = share ? group : group + (int64_t)egrp * groups, u_step = share ? groups : (int64_t)EPI_GROUPS * groups;
         if (u_first < units) fetch_steps(u_first);
         for (int64_t u = u_first; u < units && ok; u += u_step, ++lt) {
             const int64_t tile = tile_next;
             const int32_t tn = tn_next, tm = tm_next;
             const bool whole = u < P.full_tiles;              // this unit holds the complete sums of its tile
-            const uint32_t buf = (uint32_t)egrp, use = lt;
+            const uint32_t buf = share ? 0u : (uint32_t)egrp, use = lt;
+            const bool releases = !share || egrp == 0;           // one arrival per warp on the accumulator's barrier
+            const int j_lo = share ? egrp * (BN / 64) : 0, j_hi = share ? j_lo + BN / 64 : BN / 32;     // 32-column blocks
             const int64_t row0 = ((int64_t)tm * CTAS + rank) * BM;      // first row of this CTA's half
             const int64_t row = row0 + quarter * 32 + lane;
             const int64_t col_base = (int64_t)tn * BN;
@@ -559,7 +564,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // two 32-column blocks at a time: 64 bfloat16 results per row fill the 128-byte rows
                 // of the staging block, stored as one 32 x 64 box
 #pragma unroll 1
-                for (int j = 0; j < BN / 64; ++j) {
+                for (int j = j_lo / 2; j < j_hi / 2; ++j) {
                     uint32_t w[32];
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
@@ -584,11 +589,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
+                if (lane == 0 && releases) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             } else if (whole && P.tma_out) {
                 // registers -> swizzled shared-memory block -> one TMA store per 32 x 32 block
 #pragma unroll 1
-                for (int j = 0; j < BN / 32; ++j) {
+                for (int j = j_lo; j < j_hi; ++j) {
                     uint32_t v[32];
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
@@ -618,10 +623,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
+                if (lane == 0 && releases) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             } else if (whole) {
 #pragma unroll 1
-                for (int j = 0; j < BN / 32; ++j) {
+                for (int j = j_lo; j < j_hi; ++j) {
                     uint32_t v[32];
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
@@ -690,13 +695,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
+                if (lane == 0 && releases) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             } else {
                 // exact partial sums: integer adds commute, so any arrival order gives the same total.
                 // `part` holds the split tiles one after another, 128 * CTAS rows of 256 sums each.
                 const int32_t prow = (int32_t)((tile - P.full_tiles) * (BM * CTAS) + rank * BM + quarter * 32);
 #pragma unroll 1
-                for (int j = 0; j < BN / 32; ++j) {
+                for (int j = j_lo; j < j_hi; ++j) {
                     uint32_t v[32];
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
@@ -709,7 +714,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
+                if (lane == 0 && releases) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             }
         }
         if (P.opt.absmax_bits) {      // absmax of everything this warp produced: one guarded atomic

@@ -126,17 +126,15 @@ __device__ __forceinline__ uint32_t abs_max16(const uint4& q, __nv_bfloat16) {
 // A CTA covers 64 rows x (32 lanes x 2 groups x 16 bytes); four rows (eight 16-byte loads per thread)
 // are in flight at a time.  vec_ok: base and pitch allow 16-byte loads.
 template <typename T, bool ROWS, bool COLS>
-__global__ void __launch_bounds__(AMAX_THREADS, COLS ? 3 : 4)
-amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok,
-            uint32_t* __restrict__ amax_rm, uint32_t* __restrict__ amax_tr, const ScaleStep S) {
-    pdl_enter();
+__device__ __forceinline__ void amax_tile(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok,
+                                          uint32_t* __restrict__ amax_rm, uint32_t* __restrict__ amax_tr, int64_t blk) {
     constexpr int EPL = 16 / (int)sizeof(T);                   // elements per 16-byte group
     constexpr int TILE_C = 32 * AMAX_GROUPS * EPL;
     __shared__ uint32_t col_max[COLS ? TILE_C : 1];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t n_tc = (cols + TILE_C - 1) / TILE_C;
-    const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * TILE_C;
-    const int64_t r0 = ((int64_t)blockIdx.x / n_tc) * AMAX_TILE_R;
+    const int64_t c0 = (blk % n_tc) * TILE_C;
+    const int64_t r0 = (blk / n_tc) * AMAX_TILE_R;
     if constexpr (COLS) {
         for (int i = threadIdx.x; i < TILE_C; i += AMAX_THREADS) col_max[i] = 0u;
         __syncthreads();
@@ -216,27 +214,82 @@ amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, boo
             if (c < cols && col_max[i]) atomicMax(&amax_tr[c], col_max[i]);
         }
     }
-    if (S.counter == nullptr) return;
-    // the CTA that arrives last sees every maximum and turns them into step sizes
+}
+
+// True in exactly one CTA of the launch: the one that finishes last (`counter` is zero at launch).
+__device__ __forceinline__ bool last_cta_of_launch(uint32_t* counter) {
     __shared__ uint32_t is_last;
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) is_last = atomicAdd(S.counter, 1u) == gridDim.x - 1 ? 1u : 0u;
+    if (threadIdx.x == 0) is_last = atomicAdd(counter, 1u) == gridDim.x - 1 ? 1u : 0u;
     __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    for (int64_t i = threadIdx.x; i < S.n_rm; i += AMAX_THREADS) {
+    if (is_last) __threadfence();
+    return is_last != 0u;
+}
+
+// Step sizes of all groups of one operand from their maxima (one CTA).
+__device__ __forceinline__ void scale_step(const ScaleStep& S, const uint32_t* amax_rm, const uint32_t* amax_tr) {
+    for (int64_t i = threadIdx.x; i < S.n_rm; i += blockDim.x) {
         float d, r;
         scale_from_bits(__ldcg(&amax_rm[i]), S.qmax, &d, &r, S.status);
         S.inv_rm[i] = r;
         if (S.delta_rm) S.delta_rm[i] = d;
     }
-    for (int64_t i = threadIdx.x; i < S.n_tr; i += AMAX_THREADS) {
+    for (int64_t i = threadIdx.x; i < S.n_tr; i += blockDim.x) {
         float d, r;
         scale_from_bits(__ldcg(&amax_tr[i]), S.qmax, &d, &r, S.status);
         S.inv_tr[i] = r;
         if (S.delta_tr) S.delta_tr[i] = d;
     }
+}
+
+template <typename T, bool ROWS, bool COLS>
+__global__ void __launch_bounds__(AMAX_THREADS, COLS ? 3 : 4)
+amax_kernel(const T* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, bool vec_ok,
+            uint32_t* __restrict__ amax_rm, uint32_t* __restrict__ amax_tr, const ScaleStep S) {
+    pdl_enter();
+    amax_tile<T, ROWS, COLS>(x, rows, cols, ld, vec_ok, amax_rm, amax_tr, (int64_t)blockIdx.x);
+    if (S.counter == nullptr) return;
+    // the CTA that arrives last sees every maximum and turns them into step sizes
+    if (last_cta_of_launch(S.counter)) scale_step(S, amax_rm, amax_tr);
+}
+
+// The operands of one layer call in ONE launch (small problems, where the launches themselves are what
+// takes the time): CTAs [first_block[i], first_block[i + 1]) take the tiles of operand i; an operand
+// whose maxima are known contributes no tiles.  The CTA that finishes last derives every operand's
+// step sizes.  Same arithmetic as amax_kernel, flags chosen at run time.
+constexpr int BATCH_MAX = 3;
+struct AmaxOperand {
+    const void* x; int64_t rows, cols, ld;
+    uint32_t* amax_rm; uint32_t* amax_tr;            // where the tiles put their maxima
+    const uint32_t* src_rm; const uint32_t* src_tr;  // what the step sizes are derived from (may be given maxima)
+    int32_t want_rows, want_cols, vec_ok;
+    ScaleStep S;
+};
+struct AmaxBatch {
+    AmaxOperand op[BATCH_MAX];
+    uint32_t first_block[BATCH_MAX + 1];
+    int32_t n;
+    uint32_t* counter;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(AMAX_THREADS, 3)
+amax_batch_kernel(const __grid_constant__ AmaxBatch Bt) {
+    pdl_enter();
+    int i = 0;
+    while (i + 1 < Bt.n && blockIdx.x >= Bt.first_block[i + 1]) ++i;
+    if (blockIdx.x < Bt.first_block[Bt.n]) {
+        const AmaxOperand& o = Bt.op[i];
+        const int64_t blk = (int64_t)(blockIdx.x - Bt.first_block[i]);
+        const T* x = (const T*)o.x;
+        if (o.want_rows && o.want_cols) amax_tile<T, true, true>(x, o.rows, o.cols, o.ld, o.vec_ok != 0, o.amax_rm, o.amax_tr, blk);
+        else if (o.want_rows) amax_tile<T, true, false>(x, o.rows, o.cols, o.ld, o.vec_ok != 0, o.amax_rm, o.amax_tr, blk);
+        else if (o.want_cols) amax_tile<T, false, true>(x, o.rows, o.cols, o.ld, o.vec_ok != 0, o.amax_rm, o.amax_tr, blk);
+        else amax_tile<T, false, false>(x, o.rows, o.cols, o.ld, o.vec_ok != 0, o.amax_rm, o.amax_tr, blk);
+    }
+    if (!last_cta_of_launch(Bt.counter)) return;
+    for (int k = 0; k < Bt.n; ++k) scale_step(Bt.op[k].S, Bt.op[k].src_rm, Bt.op[k].src_tr);
 }
 
 template <typename T>
@@ -807,17 +860,14 @@ static void launch_rows(srq_dtype_t dt, int mode, const void* x, const QuantPara
 // General path: any extent, pitch, alignment and index offset; one Philox block per element
 // when the groups of four do not line up with the flat index.  Same results as the fast path.
 template <typename T>
-__global__ void __launch_bounds__(Q_THREADS)
-quantize_kernel(const T* __restrict__ x, const QuantParams P) {
-    pdl_enter();
+__device__ __forceinline__ void quantize_general_tile(const T* __restrict__ x, const QuantParams& P, uint32_t* tileT, int64_t blk) {
     // transposed tile: column c of the tile holds 128 row codes = 32 words; the word index is
     // XOR-ed with (c >> 2) & 31 so that both the column-wise writes and the row-wise reads
     // touch 32 different banks.
-    __shared__ uint32_t tileT[Q_TILE * (Q_TILE / 4)];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t n_tc = (P.cols + Q_TILE - 1) / Q_TILE;
-    const int64_t c0 = ((int64_t)blockIdx.x % n_tc) * Q_TILE;
-    const int64_t r0 = ((int64_t)blockIdx.x / n_tc) * Q_TILE;
+    const int64_t c0 = (blk % n_tc) * Q_TILE;
+    const int64_t r0 = (blk / n_tc) * Q_TILE;
     const int64_t c = c0 + lane * 4;
     const bool want_rm = P.codes_rm != nullptr, want_tr = P.codes_tr != nullptr;
     const bool sr = P.sr != 0;
@@ -830,8 +880,23 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
     }
     const float inv_tensor = P.per_row ? 0.0f : P.inv_rm[0];
 
+    // the next row quad is requested before the current one is used, so that a tile costs about one
+    // memory round trip instead of four (small inputs are a chain of latencies, not a stream); the loop
+    // itself stays rolled, because the kernel's code must stay small for the same reason
+    float cur[4][4], nxt[4][4];
+    auto load_quad = [&](int it, float (&q)[4][4]) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t r = r0 + (warp + 8 * it) * 4 + i;
+            if (r < P.rows && c < P.cols) load4(x + r * P.ld, c, P.cols, P.vec_in != 0, q[i]);
+            else q[i][0] = q[i][1] = q[i][2] = q[i][3] = 0.0f;
+        }
+    };
+    load_quad(0, cur);
+
 #pragma unroll 1
     for (int it = 0; it < 4; ++it) {
+        if (it + 1 < 4) load_quad(it + 1, nxt);
         const int rq = warp + 8 * it;   // row quad of the tile
         uint32_t wr[4], wt[4];
 #pragma unroll
@@ -839,20 +904,24 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
             const int64_t r = r0 + rq * 4 + i;
             wr[i] = 0u; wt[i] = 0u;
             if (r < P.rows && c < P.cols) {
-                float v[4];
-                load4(x + r * P.ld, c, P.cols, P.vec_in != 0, v);
+                const float (&v)[4] = cur[i];
                 uint32_t rnd[4] = {0u, 0u, 0u, 0u};
                 if (sr || (P.mode & MODE_SR8)) {
                     const bool sr8 = (P.mode & MODE_SR8) != 0;        // 16 elements per block, one byte each
                     const uint64_t i0 = P.index_offset + (uint64_t)r * (uint64_t)P.cols + (uint64_t)c;
+                    if (!sr8 && (i0 & 3u) == 0) {                     // the four elements share one block
+                        const uint64_t jb = i0 >> 2;
+                        philox_rounds((uint32_t)jb, (uint32_t)(jb >> 32), P.keys, rnd);
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const uint64_t ie = i0 + e, jb = sr8 ? ie >> 4 : ie >> 2;
-                        uint32_t o[4];
-                        philox_rounds((uint32_t)jb, (uint32_t)(jb >> 32), P.keys, o);
-                        const uint32_t s = sr8 ? (uint32_t)(ie >> 2) & 3u : (uint32_t)ie & 3u;
-                        const uint32_t w = s == 0 ? o[0] : s == 1 ? o[1] : s == 2 ? o[2] : o[3];
-                        rnd[e] = sr8 ? ((((w >> (8 * ((uint32_t)ie & 3u))) & 0xFFu) << 24) | 0x00800000u) : w;
+                        for (int e = 0; e < 4; ++e) {
+                            const uint64_t ie = i0 + e, jb = sr8 ? ie >> 4 : ie >> 2;
+                            uint32_t o[4];
+                            philox_rounds((uint32_t)jb, (uint32_t)(jb >> 32), P.keys, o);
+                            const uint32_t s = sr8 ? (uint32_t)(ie >> 2) & 3u : (uint32_t)ie & 3u;
+                            const uint32_t w = s == 0 ? o[0] : s == 1 ? o[1] : s == 2 ? o[2] : o[3];
+                            rnd[e] = sr8 ? ((((w >> (8 * ((uint32_t)ie & 3u))) & 0xFFu) << 24) | 0x00800000u) : w;
+                        }
                     }
                 }
                 const float inv_r = P.per_row ? P.inv_rm[want_rm ? r : 0] : inv_tensor;
@@ -880,10 +949,41 @@ quantize_kernel(const T* __restrict__ x, const QuantParams P) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) tileT[(lane * 4 + e) * 32 + (rq ^ lane)] = o[e];
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cur[i][e] = nxt[i][e];
     }
     if (!want_tr) return;
     __syncthreads();
     store_transposed_tile(tileT, P, r0, c0, warp, lane);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(Q_THREADS)
+quantize_kernel(const T* __restrict__ x, const QuantParams P) {
+    pdl_enter();
+    __shared__ uint32_t tileT[Q_TILE * (Q_TILE / 4)];
+    quantize_general_tile<T>(x, P, tileT, (int64_t)blockIdx.x);
+}
+
+// The operands of one layer call in ONE launch (small problems): CTAs [first_block[i], first_block[i + 1])
+// take the tiles of operand i.  The general path's arithmetic, so any extents and alignments; same codes.
+struct QuantBatch {
+    QuantParams P[BATCH_MAX];
+    const void* x[BATCH_MAX];
+    uint32_t first_block[BATCH_MAX + 1];
+    int32_t n;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(Q_THREADS)
+quantize_batch_kernel(const __grid_constant__ QuantBatch Bt) {
+    pdl_enter();
+    __shared__ uint32_t tileT[Q_TILE * (Q_TILE / 4)];
+    int i = 0;
+    while (i + 1 < Bt.n && blockIdx.x >= Bt.first_block[i + 1]) ++i;
+    quantize_general_tile<T>((const T*)Bt.x[i], Bt.P[i], tileT, (int64_t)(blockIdx.x - Bt.first_block[i]));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -973,61 +1073,88 @@ static int sm_count() {
     return n;
 }
 
-cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream, bool scratch_zeroed) {
-    const bool want_rm = a.codes_rm != nullptr, want_tr = a.codes_tr != nullptr;
-    const bool per_row = a.q.scale == SRQ_PER_ROW;
+// Everything launch_quantize derives from its arguments before it launches anything.
+struct QuantPlan {
+    QuantParams P;
+    bool want_rm, want_tr, per_row, given, given_cols, fast, sr8, one_pass;
+    int64_t n0, n1;               // groups whose step sizes are derived (row-major layout / transposed layout)
+    float qmax;
+    uint32_t* amax_rm; uint32_t* amax_tr;     // scratch words the absmax tiles write
+    float* inv_rm; float* inv_tr;
+};
+
+static QuantPlan make_quant_plan(const QuantArgs& a, const QuantScratch& s) {
+    QuantPlan pl;
+    pl.want_rm = a.codes_rm != nullptr; pl.want_tr = a.codes_tr != nullptr;
+    pl.per_row = a.q.scale == SRQ_PER_ROW;
+    const bool want_rm = pl.want_rm, want_tr = pl.want_tr, per_row = pl.per_row;
     const int64_t rows = a.rows, cols = a.cols;
-    if (rows == 0 || cols == 0 || (!want_rm && !want_tr)) return cudaSuccess;
     const bool e4m3 = a.q.format == SRQ_GRID_E4M3;
     // E4Mk grid: bits = 5 + k; the largest value with k mantissa bits is 448 (k = 3, 2), 384 (k = 1), 256 (k = 0)
     const int mant = e4m3 ? a.q.bits - 5 : 3;
-    const float qmax = e4m3 ? (mant >= 2 ? 448.0f : (mant == 1 ? 384.0f : 256.0f)) : (float)((1 << (a.q.bits - 1)) - 1);
+    pl.qmax = e4m3 ? (mant >= 2 ? 448.0f : (mant == 1 ? 384.0f : 256.0f)) : (float)((1 << (a.q.bits - 1)) - 1);
     const size_t esize = a.dt == SRQ_F32 ? 4 : 2;
 
     // group counts and where each layout's absmax lives; per tensor both layouts share word 0
     const int64_t n_rm = want_rm ? (per_row ? rows : 1) : 0;
     const int64_t n_tr = want_tr ? (per_row ? cols : 1) : 0;
-    uint32_t* amax_rm = s.amax_rm;
-    uint32_t* amax_tr = per_row ? s.amax_tr : s.amax_rm;
-    float* inv_rm = s.inv_rm;
-    float* inv_tr = per_row ? s.inv_tr : s.inv_rm;
+    pl.amax_rm = s.amax_rm;
+    pl.amax_tr = per_row ? s.amax_tr : s.amax_rm;
+    pl.inv_rm = s.inv_rm;
+    pl.inv_tr = per_row ? s.inv_tr : s.inv_rm;
 
     const bool vec_in = ((uintptr_t)a.x % (4 * esize) == 0) && (a.ld % 4 == 0);
-    const bool given = a.q.absmax != nullptr && !per_row;   // per tensor: one known maximum for the whole operand
+    pl.given = a.q.absmax != nullptr && !per_row;   // per tensor: one known maximum for the whole operand
     // per row: known column maxima [cols] for the transposed layout (its groups run over the rows, i.e.
     // over the tokens, which other shards may hold); the row-major layout's row maxima are local
-    const bool given_cols = a.q.absmax != nullptr && per_row && want_tr;
+    pl.given_cols = a.q.absmax != nullptr && per_row && want_tr;
     // per tensor: one group feeds both layouts' scale outputs
-    const int64_t n0 = per_row ? n_rm : 1;
-    const int64_t n1 = per_row ? n_tr : ((want_tr && a.scale_tr) ? 1 : 0);
+    pl.n0 = per_row ? n_rm : 1;
+    pl.n1 = per_row ? n_tr : ((want_tr && a.scale_tr) ? 1 : 0);
 
-    QuantParams P;
+    QuantParams& P = pl.P;
     P.rows = rows; P.cols = cols; P.ld = a.ld;
     P.index_offset = a.q.index_offset;
     P.keys = make_philox_keys(a.q.seed, a.q.tensor_id);
     P.sr = a.q.round == SRQ_SR;
-    const bool sr8 = a.q.round == SRQ_SR8;
-    P.mode = sr8 ? MODE_SR8 : ((P.sr ? MODE_SR : 0) | (e4m3 ? MODE_E4M3 : 0));
+    pl.sr8 = a.q.round == SRQ_SR8;
+    P.mode = pl.sr8 ? MODE_SR8 : ((P.sr ? MODE_SR : 0) | (e4m3 ? MODE_E4M3 : 0));
     P.e4m_shift = (uint32_t)(3 - mant);
     P.per_row = per_row;
     P.codes_rm = a.codes_rm; P.ld_rm = a.ld_rm;
     P.codes_tr = a.codes_tr; P.ld_tr = a.ld_tr;
-    P.inv_rm = inv_rm; P.inv_tr = inv_tr;
+    P.inv_rm = pl.inv_rm; P.inv_tr = pl.inv_tr;
     P.vec_in = vec_in;
     P.vec_rm = want_rm && ((uintptr_t)a.codes_rm % 4 == 0) && (a.ld_rm % 4 == 0);
     P.vec_tr = want_tr && ((uintptr_t)a.codes_tr % 4 == 0) && (a.ld_tr % 4 == 0);
     P.vec_tr16 = want_tr && ((uintptr_t)a.codes_tr % 16 == 0) && (a.ld_tr % 16 == 0);
-    const bool fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && (!sr8 || (cols % 16 == 0 && a.q.index_offset % 16 == 0)) && a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) &&
-                      (!want_tr || (P.vec_tr && rows % 4 == 0));
-
+    pl.fast = vec_in && (cols % 4 == 0) && (a.q.index_offset % 4 == 0) && (!pl.sr8 || (cols % 16 == 0 && a.q.index_offset % 16 == 0)) &&
+              a.ld < (1 << 24) && a.ld_rm < (1 << 24) && (!want_rm || P.vec_rm) && (!want_tr || (P.vec_tr && rows % 4 == 0));
     // per-row steps and row-major codes only: one pass (rows of 512 .. 8192 elements)
-    if (per_row && want_rm && !want_tr && fast && !sr8 && cols >= 512 && cols <= (int64_t)ROWQ_MAX_G * Q_THREADS * 4) {
+    pl.one_pass = per_row && want_rm && !want_tr && pl.fast && !pl.sr8 && cols >= 512 && cols <= (int64_t)ROWQ_MAX_G * Q_THREADS * 4;
+    return pl;
+}
+
+cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t* status, cudaStream_t stream, bool scratch_zeroed) {
+    const int64_t rows = a.rows, cols = a.cols;
+    if (rows == 0 || cols == 0 || (!a.codes_rm && !a.codes_tr)) return cudaSuccess;
+    const QuantPlan pl = make_quant_plan(a, s);
+    const QuantParams& P = pl.P;
+    const bool want_rm = pl.want_rm, want_tr = pl.want_tr, per_row = pl.per_row;
+    const int64_t n0 = pl.n0, n1 = pl.n1;
+    const float qmax = pl.qmax;
+    uint32_t* amax_rm = pl.amax_rm;
+    uint32_t* amax_tr = pl.amax_tr;
+    float* inv_rm = pl.inv_rm;
+    float* inv_tr = pl.inv_tr;
+
+    if (pl.one_pass) {
         launch_rows(a.dt, P.mode, a.x, P, a.scale_rm, qmax, status, sm_count(), stream);
         count_launch();
         return cudaGetLastError();
     }
 
-    if (given_cols) {
+    if (pl.given_cols) {
         const int threads = 256;
         if (want_rm) {                                  // row maxima of this shard, then their step sizes
             if (!scratch_zeroed) {
@@ -1041,14 +1168,14 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         }
         const uint32_t* col_bits = (const uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
         const int64_t n = n0 > n1 ? n0 : n1;
-        launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
+        launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream,
             amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr, col_bits, n1, inv_tr, a.scale_tr, qmax, status);
         count_launch();
-    } else if (given) {
+    } else if (pl.given) {
         amax_rm = amax_tr = (uint32_t*)a.q.absmax;     // a non-negative float is its own bit pattern
         const int64_t n = n0 > n1 ? n0 : n1;
         const int threads = 256;
-        launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
+        launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream,
             amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
             amax_tr, n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status);
         count_launch();
@@ -1069,7 +1196,7 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
         if (!few) {
             const int64_t n = n0 > n1 ? n0 : n1;
             const int threads = 256;
-            launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream, 
+            launch_pdl(scales_kernel, dim3((unsigned)((n + threads - 1) / threads)), dim3(threads), 0, stream,
                 amax_rm, n0, inv_rm, want_rm ? a.scale_rm : nullptr,
                 amax_tr, n1, inv_tr, want_tr ? a.scale_tr : nullptr, qmax, status);
             count_launch();
@@ -1077,11 +1204,74 @@ cudaError_t launch_quantize(const QuantArgs& a, const QuantScratch& s, uint32_t*
     }
     {
         const unsigned grid = (unsigned)(((cols + Q_TILE - 1) / Q_TILE) * ((rows + Q_TILE - 1) / Q_TILE));
-        if (fast) launch_fast(a.dt, P.mode, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);
+        if (pl.fast) launch_fast(a.dt, P.mode, (want_rm ? 1 : 0) | (want_tr ? 2 : 0), per_row, a.x, P, grid, stream);
         else if (a.dt == SRQ_F32) launch_pdl(quantize_kernel<float>, dim3(grid), dim3(Q_THREADS), 0, stream, (const float*)a.x, P);
         else launch_pdl(quantize_kernel<__nv_bfloat16>, dim3(grid), dim3(Q_THREADS), 0, stream, (const __nv_bfloat16*)a.x, P);
         count_launch();
     }
+    return cudaGetLastError();
+}
+
+// The operands of one layer call.  Small problems (the launches, not the data, take the time) get two
+// launches for all operands together, one for the maxima and step sizes, one for the codes; anything
+// else, and anything the batched kernels do not cover, goes operand by operand.  Same results.
+cudaError_t launch_quantize_batch(const QuantArgs* a, const QuantScratch* s, int n, uint32_t* status, cudaStream_t stream,
+                                  bool scratch_zeroed) {
+    // measured: below about four million elements per call the saved launches outweigh the general
+    // kernel's lower speed; above, the specialised kernels win
+    constexpr int64_t kBatchMaxElements = 1ll << 22, kBatchMaxGroups = 2048;
+    int64_t elements = 0, groups = 0;
+    bool ok = n >= 2 && n <= BATCH_MAX && scratch_zeroed;
+    QuantPlan pl[BATCH_MAX];
+    for (int i = 0; ok && i < n; ++i) {
+        if (a[i].rows == 0 || a[i].cols == 0 || (!a[i].codes_rm && !a[i].codes_tr) || a[i].dt != a[0].dt) { ok = false; break; }
+        pl[i] = make_quant_plan(a[i], s[i]);
+        elements += a[i].rows * a[i].cols;
+        groups += pl[i].n0 + pl[i].n1;
+        if (a[i].ld >= (1ll << 31) || a[i].rows >= (1ll << 31)) ok = false;
+    }
+    if (!ok || elements > kBatchMaxElements || groups > kBatchMaxGroups) {
+        for (int i = 0; i < n; ++i) {
+            const cudaError_t e = launch_quantize(a[i], s[i], status, stream, scratch_zeroed);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
+    }
+
+    AmaxBatch ab = {};
+    QuantBatch qb = {};
+    ab.n = qb.n = n;
+    ab.counter = s[0].counter;                       // zeroed with the rest of the scratch
+    uint32_t ablocks = 0, qblocks = 0;
+    for (int i = 0; i < n; ++i) {
+        const QuantArgs& A = a[i];
+        const QuantPlan& p = pl[i];
+        const size_t esize = A.dt == SRQ_F32 ? 4 : 2;
+        AmaxOperand& o = ab.op[i];
+        o.x = A.x; o.rows = A.rows; o.cols = A.cols; o.ld = A.ld;
+        o.amax_rm = p.amax_rm; o.amax_tr = p.amax_tr;
+        o.vec_ok = ((uintptr_t)A.x % 16 == 0) && ((A.ld * (int64_t)esize) % 16 == 0);
+        // which maxima the tiles have to find, and which words the step sizes come from
+        bool tiles = true;
+        o.want_rows = p.per_row && p.want_rm; o.want_cols = p.per_row && p.want_tr;
+        o.src_rm = p.amax_rm; o.src_tr = p.amax_tr;
+        if (p.given) { tiles = false; o.src_rm = o.src_tr = (const uint32_t*)A.q.absmax; }
+        else if (p.given_cols) { tiles = p.want_rm; o.want_cols = 0; o.src_tr = (const uint32_t*)A.q.absmax; }
+        o.S = ScaleStep{nullptr, p.n0, p.inv_rm, p.want_rm ? A.scale_rm : nullptr, p.n1, p.inv_tr, p.want_tr ? A.scale_tr : nullptr, p.qmax, status};
+        const int tile_c = 32 * AMAX_GROUPS * (16 / (int)esize);
+        ab.first_block[i] = ablocks;
+        if (tiles) ablocks += (uint32_t)(((A.cols + tile_c - 1) / tile_c) * ((A.rows + AMAX_TILE_R - 1) / AMAX_TILE_R));
+        qb.P[i] = p.P; qb.x[i] = A.x;
+        qb.first_block[i] = qblocks;
+        qblocks += (uint32_t)(((A.cols + Q_TILE - 1) / Q_TILE) * ((A.rows + Q_TILE - 1) / Q_TILE));
+    }
+    ab.first_block[n] = ablocks; qb.first_block[n] = qblocks;
+    if (a[0].dt == SRQ_F32) launch_pdl(amax_batch_kernel<float>, dim3(ablocks ? ablocks : 1u), dim3(AMAX_THREADS), 0, stream, ab);
+    else launch_pdl(amax_batch_kernel<__nv_bfloat16>, dim3(ablocks ? ablocks : 1u), dim3(AMAX_THREADS), 0, stream, ab);
+    count_launch();
+    if (a[0].dt == SRQ_F32) launch_pdl(quantize_batch_kernel<float>, dim3(qblocks), dim3(Q_THREADS), 0, stream, qb);
+    else launch_pdl(quantize_batch_kernel<__nv_bfloat16>, dim3(qblocks), dim3(Q_THREADS), 0, stream, qb);
+    count_launch();
     return cudaGetLastError();
 }
 
