@@ -84,6 +84,28 @@ __device__ __forceinline__ void philox_rounds(uint32_t c0, uint32_t c1, const Ph
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// The same ten rounds, returning the COMPLEMENT of every output word (what the rounding rule adds):
+// in the last round the two words that are low halves of products come complemented from a
+// multiply-add of their own ( ~lo(M c) = lo((-M) c) - 1 ), and the two that end in an exclusive-or
+// absorb the complement into that operation, so that no separate NOT is spent on any of them.
+__device__ __forceinline__ void philox_rounds_not(uint32_t c0, uint32_t c1, const PhiloxKeys& K, uint32_t out[4]) {
+    uint32_t c2 = K.tid0, c3 = K.tid1;
+#pragma unroll
+    for (int r = 0; r < 9; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
+        c3 = (uint32_t)p0;
+    }
+    const uint32_t h0 = __umulhi(0xD2511F53u, c0), h1 = __umulhi(0xCD9E8D57u, c2);
+    out[0] = ~(h1 ^ c1 ^ K.k0[9]);
+    out[1] = c2 * 0x326172A9u + 0xFFFFFFFFu;         // -0xCD9E8D57 mod 2^32
+    out[2] = ~(h0 ^ c3 ^ K.k1[9]);
+    out[3] = c0 * 0x2DAEE0ADu + 0xFFFFFFFFu;         // -0xD2511F53 mod 2^32
+}
+
 // Round keys and upper counter words for one quantization point.
 inline PhiloxKeys make_philox_keys(uint64_t seed, uint64_t tensor_id) {
     PhiloxKeys k;

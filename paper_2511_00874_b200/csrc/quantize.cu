@@ -343,19 +343,20 @@ __global__ void scales_kernel(const uint32_t* amax_rm, int64_t n_rm, float* inv_
 //        (floor(S) + 2^23) >> 24.
 // |t| <= qmax for every element of a group (the reciprocal step is rounded toward zero), so
 // |C| <= qmax 2^24, the sum stays inside int32 and the code inside [-qmax, qmax] without a clamp.
+// NOTTED: the threshold word arrives complemented (philox_rounds_not), which saves the NOT here.
 // MODE: bit 0 = stochastic rounding (else round to nearest), bit 1 = E4M3 grid (else integer grid),
 // bit 2 = stochastic rounding with 8 random bits per element (integer grid only; the thresholds are
 // then handed to the same arithmetic as words (b << 24) | 2^23, whose top 24 bits are (2 b + 1) 2^15).
 constexpr int MODE_SR = 1, MODE_E4M3 = 2, MODE_SR8 = 4;
 
 // Integer grid: returns the 32-bit sum whose top byte is the code (two's complement).
-template <int MODE>
+template <int MODE, bool NOTTED = false>
 __device__ __forceinline__ uint32_t quantize_sum(float x, float inv, uint32_t word) {
     const float s = __fmul_rn(__fmul_rn(x, inv), 16777216.0f);
     if constexpr ((MODE & MODE_SR) != 0) {
         const int c = __float2int_ru(s);
         uint32_t sum;   // (~word >> 8) + c = (2^24 - 1 - u24) + c in one multiply-add (high half)
-        asm("mad.hi.u32 %0, %1, 16777216, %2;" : "=r"(sum) : "r"(~word), "r"((uint32_t)c));
+        asm("mad.hi.u32 %0, %1, 16777216, %2;" : "=r"(sum) : "r"(NOTTED ? word : ~word), "r"((uint32_t)c));
         return sum;
     } else {
         return (uint32_t)__float2int_rd(s) + 0x00800000u;
@@ -368,7 +369,7 @@ __device__ __forceinline__ uint32_t quantize_sum(float x, float inv, uint32_t wo
 // exponent of t, the code is sign | ((E - 120) << 3) + |q| - 8: |q| = 16 carries into the exponent
 // field (next binade), |q| < 8 only occurs for E = 121 and gives the subnormal codes, q = 0 gives +0.
 // Returns the code in the low byte.
-template <int MODE>
+template <int MODE, bool NOTTED = false>
 __device__ __forceinline__ uint32_t quantize_e4m3(float x, float inv, uint32_t word, uint32_t sh) {
     // sh = 3 - k for the E4Mk grid (k mantissa bits; 0 for E4M3 itself): the step of binade e is
     // 2^(e-k), q counts those steps, and q << sh is the same value in the E4M3 code's units of 2^(e-3)
@@ -378,7 +379,7 @@ __device__ __forceinline__ uint32_t quantize_e4m3(float x, float inv, uint32_t w
     uint32_t sum;
     if constexpr ((MODE & MODE_SR) != 0) {
         const int c = __float2int_ru(s);
-        asm("mad.hi.u32 %0, %1, 16777216, %2;" : "=r"(sum) : "r"(~word), "r"((uint32_t)c));
+        asm("mad.hi.u32 %0, %1, 16777216, %2;" : "=r"(sum) : "r"(NOTTED ? word : ~word), "r"((uint32_t)c));
     } else {
         sum = (uint32_t)__float2int_rd(s) + 0x00800000u;
     }
@@ -394,18 +395,18 @@ __device__ __forceinline__ void sr8_words(uint32_t w, uint32_t rnd[4]) {
 }
 
 // Four codes packed into one word, first element in the low byte.
-template <int MODE>
+template <int MODE, bool NOTTED = false>
 __device__ __forceinline__ uint32_t quantize4(const float v[4], float i0, float i1, float i2, float i3,
                                               const uint32_t rnd[4], uint32_t sh) {
     if constexpr ((MODE & MODE_SR8) != 0) {
         return quantize4<MODE_SR>(v, i0, i1, i2, i3, rnd, sh);
     } else if constexpr ((MODE & MODE_E4M3) != 0) {
-        const uint32_t c0 = quantize_e4m3<MODE>(v[0], i0, rnd[0], sh), c1 = quantize_e4m3<MODE>(v[1], i1, rnd[1], sh);
-        const uint32_t c2 = quantize_e4m3<MODE>(v[2], i2, rnd[2], sh), c3 = quantize_e4m3<MODE>(v[3], i3, rnd[3], sh);
+        const uint32_t c0 = quantize_e4m3<MODE, NOTTED>(v[0], i0, rnd[0], sh), c1 = quantize_e4m3<MODE, NOTTED>(v[1], i1, rnd[1], sh);
+        const uint32_t c2 = quantize_e4m3<MODE, NOTTED>(v[2], i2, rnd[2], sh), c3 = quantize_e4m3<MODE, NOTTED>(v[3], i3, rnd[3], sh);
         return __byte_perm(__byte_perm(c0, c1, 0x0040), __byte_perm(c2, c3, 0x0040), 0x5410);
     } else {
-        const uint32_t s0 = quantize_sum<MODE>(v[0], i0, rnd[0]), s1 = quantize_sum<MODE>(v[1], i1, rnd[1]);
-        const uint32_t s2 = quantize_sum<MODE>(v[2], i2, rnd[2]), s3 = quantize_sum<MODE>(v[3], i3, rnd[3]);
+        const uint32_t s0 = quantize_sum<MODE, NOTTED>(v[0], i0, rnd[0]), s1 = quantize_sum<MODE, NOTTED>(v[1], i1, rnd[1]);
+        const uint32_t s2 = quantize_sum<MODE, NOTTED>(v[2], i2, rnd[2]), s3 = quantize_sum<MODE, NOTTED>(v[3], i3, rnd[3]);
         return __byte_perm(__byte_perm(s0, s1, 0x0073), __byte_perm(s2, s3, 0x0073), 0x5410);   // top bytes
     }
 }
@@ -498,6 +499,7 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
     constexpr bool WANT_RM = (LAYOUT & 1) != 0, WANT_TR = (LAYOUT & 2) != 0;
     constexpr bool TWO_STEPS = WANT_TR && PER_ROW;     // transposed layout has its own step sizes
     constexpr bool SRM = (MODE & MODE_SR) != 0, SR8 = (MODE & MODE_SR8) != 0;
+    constexpr bool NT = SRM && !SR8;                  // thresholds arrive complemented
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t c = c0 + lane * 4;
     const bool col_ok = FULL || c < P.cols;             // cols % 4 == 0: a group is all in or all out
@@ -571,17 +573,17 @@ __device__ __forceinline__ void quantize_tile(const T* __restrict__ x, const Qua
             if constexpr (SR8) sr8_words(sw[i], rnd);
             if constexpr (SRM) {
                 if constexpr (FULL) {
-                    philox_rounds(jb_lo + tr * j_row, jb_hi, P.keys, rnd);
+                    philox_rounds_not(jb_lo + tr * j_row, jb_hi, P.keys, rnd);
                 } else {
                     const uint64_t jj = jb + (uint64_t)tr * j_row;
-                    philox_rounds((uint32_t)jj, (uint32_t)(jj >> 32), P.keys, rnd);
+                    philox_rounds_not((uint32_t)jj, (uint32_t)(jj >> 32), P.keys, rnd);
                 }
             }
             if constexpr (WANT_RM || !TWO_STEPS) {
                 const float ir = (PER_ROW && WANT_RM) ? inv_cur[i] : inv_tensor;
-                wr[i] = quantize4<MODE>(v, ir, ir, ir, ir, rnd, P.e4m_shift);
+                wr[i] = quantize4<MODE, NT>(v, ir, ir, ir, ir, rnd, P.e4m_shift);
             }
-            if constexpr (TWO_STEPS) wt[i] = quantize4<MODE>(v, ic[0], ic[1], ic[2], ic[3], rnd, P.e4m_shift);
+            if constexpr (TWO_STEPS) wt[i] = quantize4<MODE, NT>(v, ic[0], ic[1], ic[2], ic[3], rnd, P.e4m_shift);
             else wt[i] = wr[i];
             if constexpr (WANT_RM) {
                 if (FULL || (col_ok && r0 + tr < P.rows)) *reinterpret_cast<uint32_t*>(out_rm + tr * ld_rm) = wr[i];
@@ -719,9 +721,9 @@ quantize_rows_kernel(const T* __restrict__ x, const __grid_constant__ QuantParam
             uint32_t rnd[4] = {0u, 0u, 0u, 0u};
             if constexpr (SRM) {
                 const uint32_t lo = (uint32_t)jb + g;
-                philox_rounds(lo, (uint32_t)(jb >> 32) + (lo < g ? 1u : 0u), P.keys, rnd);
+                philox_rounds_not(lo, (uint32_t)(jb >> 32) + (lo < g ? 1u : 0u), P.keys, rnd);
             }
-            w[k] = quantize4<MODE>(v, inv, inv, inv, inv, rnd, P.e4m_shift);
+            w[k] = quantize4<MODE, SRM>(v, inv, inv, inv, inv, rnd, P.e4m_shift);
         }
 #pragma unroll
         for (int k = 0; k < G; ++k) {
@@ -770,9 +772,9 @@ quantize_rows_warp_kernel(const T* __restrict__ x, const __grid_constant__ Quant
             uint32_t rnd[4] = {0u, 0u, 0u, 0u};
             if constexpr (SRM) {
                 const uint32_t lo = (uint32_t)jb + g;
-                philox_rounds(lo, (uint32_t)(jb >> 32) + (lo < g ? 1u : 0u), P.keys, rnd);
+                philox_rounds_not(lo, (uint32_t)(jb >> 32) + (lo < g ? 1u : 0u), P.keys, rnd);
             }
-            const uint32_t w = quantize4<MODE>(v, inv, inv, inv, inv, rnd, P.e4m_shift);
+            const uint32_t w = quantize4<MODE, SRM>(v, inv, inv, inv, inv, rnd, P.e4m_shift);
             if (g < ngroups) out[g] = w;
         }
     }
