@@ -348,7 +348,7 @@ def run_ours(args):
     barrier()
     if rank == 0:
         sus_sampler.start()
-    sus_ms, sus_n = _timed_loop(lambda i: step(2000 + i), 2.0, ms, torch)
+    sus_ms, sus_n = _timed_loop(lambda i: step(2000 + i), args.sustained_seconds, ms, torch)
     barrier()
     sus_ms = max_over_ranks(sus_ms)
     sus_clocks = sus_sampler.stop() if rank == 0 else None
@@ -446,7 +446,7 @@ def run_ours(args):
         def three(_):
             for a_, b_, o_ in gemms:
                 srq.srq_gemm_i8(a_, b_, one, one, o_, None, gws)
-        s_ms3, s_n = _timed_loop(three, 2.0, 3.0 * launch_ms, torch)
+        s_ms3, s_n = _timed_loop(three, args.sustained_seconds, 3.0 * launch_ms, torch)
         s_clocks = s_sampler.stop()
         s_achieved = ops_per_launch / (s_ms3 / 3.0 * 1e-3) / 1e12
         peak_sus = 2.0 * peaks["bf16_sustained"]
@@ -464,7 +464,7 @@ def run_ours(args):
             m1.record()
         torch.cuda.synchronize()
         mma_burst = mma_ops / (statistics.mean(m0.elapsed_time(m1) for m0, m1 in m_evs) * 1e-3) / 1e12
-        mm_ms, _ = _timed_loop(lambda _i: srq.srq_selftest_mma_rate(mws, kb), 2.0, mma_ops / (mma_burst * 1e12) * 1e3, torch)
+        mm_ms, _ = _timed_loop(lambda _i: srq.srq_selftest_mma_rate(mws, kb), args.sustained_seconds, mma_ops / (mma_burst * 1e12) * 1e3, torch)
         mma_sus = mma_ops / (mm_ms * 1e-3) / 1e12
         if srq.srq_poll_status(mws) != 0:
             raise SystemExit("tensor-pipe microbenchmark reported a device-side condition")
@@ -486,7 +486,7 @@ def run_ours(args):
                           "ms_per_launch": s_ms3 / 3.0, "launches": 3 * s_n, "clocks": s_clocks,
                           "frac_of_mma_only": s_achieved / mma_sus,
                           "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS TFLOP/s",
-                          "regime": "the three products back to back for two seconds (power cap)"}}
+                          "regime": f"the three products back to back for {args.sustained_seconds:g} s (power cap)"}}
         del cA, cAt, cW, cWt, cdY, cdYt
 
         result["quantizer"] = quantizer
@@ -503,6 +503,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the back-to-back loops that give the figures under the power cap")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
