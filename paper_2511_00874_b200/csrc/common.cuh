@@ -39,6 +39,12 @@ __device__ __forceinline__ void pdl_enter() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
+// The two halves on their own, for a kernel whose set-up touches no global memory: it lets its successor
+// be launched at once and waits for its predecessor only when the set-up is done, so that the set-up
+// overlaps the predecessor's tail.  Nothing the predecessor wrote may be read, and nothing it may
+// still read may be written, before pdl_wait().
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 // Not while the stream is being captured: in a replayed graph the ordinary kernel-to-kernel edges were
 // measured faster than the programmatic ones (0.104 against 0.111 ms for a 15-kernel layer).
 static inline bool pdl_allowed(cudaStream_t st) {

@@ -367,7 +367,7 @@ template <int CTAS, int KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_part, const GemmParams P) {
-    pdl_enter();
+    pdl_trigger();                                   // the wait follows the set-up below, which touches only shared memory and TMEM
     using C = Cfg<CTAS>;
     constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES;
     using Tail = SharedTail<STAGES>;
@@ -393,6 +393,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if constexpr (CTAS == 1) __syncthreads(); else cluster_sync();   // the peer's barriers exist from here on
     tc_fence_after();
     const uint32_t tmem_base = T->tmem_base;
+    pdl_wait();                                      // from here on the work before this kernel has finished and is visible
 
     const int64_t groups = gridDim.x / CTAS, group = blockIdx.x / CTAS;   // a group = the CTAs of one tile
     // work units: the first full_tiles tiles whole, then every remaining tile in `splits` parts

@@ -124,6 +124,13 @@ def test_every_kernel_waits_for_its_predecessor_first():
             if kernel in plain_only:
                 assert ("launch_pdl(" + kernel) not in text, kernel
                 continue
+            if first.startswith("pdl_trigger();"):        # set-up first, then the wait, before any global access
+                rest = text[body:text.index("\n}\n", body)]
+                assert "pdl_wait();" in rest, f"{name}: {kernel} triggers but never waits"
+                before = rest[:rest.index("pdl_wait();")]
+                assert not re.search(r"__ldg|__ldc|\bP\.(out|s_row|s_col|acc_out|part|status)\b\s*[\[\+]|tma_load|tma_store|atomic", before), \
+                    f"{name}: {kernel} touches global memory before its wait"
+                continue
             assert first == "pdl_enter();", f"{name}: {kernel} starts with {first!r}"
     assert seen >= 12
 
