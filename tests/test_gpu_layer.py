@@ -182,6 +182,36 @@ def test_layer_with_eight_random_bits_per_element():
     all_passes(A, W, dY, layer_specs(srq.PER_TENSOR, srq.SR8, seed=4, bits_fwd=8, bits_bwd=4))
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_operands_of_one_call_with_different_quantization_points(dtype):
+    """Small layers quantize all operands of a call in one pair of launches; every operand keeps its own
+    point there: per-row steps beside per-tensor steps, round-to-nearest beside 24-bit and 8-bit
+    stochastic rounding, different widths, one operand with a maximum the caller already knows."""
+    T, N, K = 136, 264, 328
+    A, W, dY = synth.layer_inputs(T, N, K, seed=12, dtype=dtype, device="cuda", std_dy=1e-3)
+    q = {"a_fwd": srq.QSpec(8, srq.PER_ROW, srq.SR, 5, 0), "w_fwd": srq.QSpec(5, srq.PER_TENSOR, srq.RTN, 5, 1),
+         "a_bwd": srq.QSpec(6, srq.PER_TENSOR, srq.SR8, 5, 2), "w_bwd": srq.QSpec(8, srq.PER_ROW, srq.RTN, 5, 3),
+         "dy_bwd": srq.QSpec(4, srq.PER_ROW, srq.SR, 5, 4)}
+    all_passes(A, W, dY, q)
+    # the whole backward pass in one call (three operands in the batch), A's maximum handed in
+    m = torch.zeros(1, device="cuda")
+    srq.srq_absmax(A, m)
+    qa = srq.QSpec(6, srq.PER_TENSOR, srq.SR8, 5, 2, absmax=m)
+    dA, dW = torch.empty((T, K), device="cuda"), torch.empty((N, K), device="cuda")
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
+    srq.qlinear_bwd(dY, A, W, q["dy_bwd"], qa, q["w_bwd"], dA, dW, None, None, ws)
+    assert srq.srq_poll_status(ws) == 0
+    oq = lambda s: oracle.QSpec(s.bits, s.scale, s.round, s.seed, s.tensor_id, s.index_offset)
+    f = lambda t: t.float().cpu().numpy()
+    assert np.array_equal(dA.cpu().numpy(), oracle.qlinear_bwd_input(f(dY), f(W), oq(q["dy_bwd"]), oq(q["w_bwd"])).out)
+    assert np.array_equal(dW.cpu().numpy(), oracle.qlinear_bwd_weight(f(dY), f(A), oq(q["dy_bwd"]), oq(q["a_bwd"])).out)
+    # a non-finite input of any operand of the batch reaches the status word
+    W2 = W.clone()
+    W2[3, 5] = float("nan")
+    srq.qlinear_bwd(dY, A, W2, q["dy_bwd"], qa, q["w_bwd"], dA, dW, None, None, ws)
+    assert srq.srq_poll_status(ws) == srq.binding.ERR_NONFINITE
+
+
 @pytest.mark.parametrize("case", range(16))
 def test_random_layers(case):
     """Seeded random layers: extents (aligned and odd, rows long enough for the one-pass per-row
