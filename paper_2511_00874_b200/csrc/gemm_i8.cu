@@ -371,6 +371,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     using C = Cfg<CTAS>;
     constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES;
     using Tail = SharedTail<STAGES>;
+    static_assert(4 * EPI_GROUPS * 4 * OUT_STAGE_BYTES <= STAGES * STAGE_BYTES, "the ring must hold one staging buffer per block of a shared tile");
     extern __shared__ uint8_t smem_raw[];
     // the dynamic window starts at the same offset in every CTA, so the aligned layouts coincide
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -560,6 +561,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
             const uint32_t stage = smem_u32(out_stage + (warp - 2) * OUT_STAGE_BYTES);
+            // A CTA with a single unit has no further use for its operand ring once the accumulator is
+            // complete: its blocks are staged there, one buffer per block, so that no block waits for the
+            // previous block's store to have read the staging buffer (8 warps x 4 blocks x 4 KB).
+            const uint32_t ring_stage = smem_u32(smem) + (uint32_t)((warp - 2) * 4) * (uint32_t)OUT_STAGE_BYTES;
             const int32_t wrow = (int32_t)(row0 + quarter * 32);           // first row of this warp's blocks
             if (whole && P.tma_out && P.opt.out_bf16) {
                 // two 32-column blocks at a time: 64 bfloat16 results per row fill the 128-byte rows
@@ -581,12 +586,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int i = 0; i < 16; ++i) w[h * 16 + i] = pack_bf16(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
                     }
                     const int32_t col0 = (int32_t)col_base + j * 64;
-                    if (lane == 0) bulk_wait_read();
+                    const uint32_t stg = share ? ring_stage + (uint32_t)(j - j_lo / 2) * (uint32_t)OUT_STAGE_BYTES : stage;
+                    if (!share && lane == 0) bulk_wait_read();
                     __syncwarp();
-                    stage_block(stage, lane, w);
+                    stage_block(stg, lane, w);
                     fence_async_smem();
                     __syncwarp();
-                    if (lane == 0 && wrow < P.M && col0 < P.N) { tma_store_2d(&map_out, stage, col0, wrow); bulk_commit(); }
+                    if (lane == 0 && wrow < P.M && col0 < P.N) { tma_store_2d(&map_out, stg, col0, wrow); bulk_commit(); }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -611,14 +617,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                     const int32_t col0 = (int32_t)col_base + j * 32;
                     output_options(P, v, row, col0, rq_inv, amax);
-                    if (lane == 0) bulk_wait_read();          // the previous block has left the staging buffer
+                    const uint32_t stg = share ? ring_stage + (uint32_t)(j - j_lo) * (uint32_t)OUT_STAGE_BYTES : stage;
+                    if (!share && lane == 0) bulk_wait_read();          // the previous block has left the staging buffer
                     __syncwarp();
-                    stage_block(stage, lane, v);
+                    stage_block(stg, lane, v);
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0 && wrow < P.M && col0 < P.N) {
-                        if (P.opt.accumulate == 1) tma_reduce_add_2d(&map_out, stage, col0, wrow);   // binary32 adds in memory
-                        else tma_store_2d(&map_out, stage, col0, wrow);
+                        if (P.opt.accumulate == 1) tma_reduce_add_2d(&map_out, stg, col0, wrow);   // binary32 adds in memory
+                        else tma_store_2d(&map_out, stg, col0, wrow);
                         bulk_commit();
                     }
                 }
@@ -706,12 +713,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     uint32_t v[32];
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
-                    if (lane == 0) bulk_wait_read();
+                    const uint32_t stg = share ? ring_stage + (uint32_t)(j - j_lo) * (uint32_t)OUT_STAGE_BYTES : stage;
+                    if (!share && lane == 0) bulk_wait_read();
                     __syncwarp();
-                    stage_block(stage, lane, v);
+                    stage_block(stg, lane, v);
                     fence_async_smem();
                     __syncwarp();
-                    if (lane == 0) { tma_reduce_add_2d(&map_part, stage, j * 32, prow); bulk_commit(); }
+                    if (lane == 0) { tma_reduce_add_2d(&map_part, stg, j * 32, prow); bulk_commit(); }
                 }
                 tc_fence_before();
                 __syncwarp();

@@ -452,9 +452,11 @@ struct QuantParams {
 };
 
 // Row-wise read of the transposed tile and its stores: one warp per tile column, lane = row quad.
+// Only the row quads [quad_lo, quad_hi) of the tile have been written (a CTA that took a slice of the tile).
 __device__ __forceinline__ void store_transposed_tile(const uint32_t* tileT, const QuantParams& P, int64_t r0, int64_t c0,
-                                                      int warp, int lane) {
+                                                      int warp, int lane, int quad_lo = 0, int quad_hi = 32) {
     const int64_t r = r0 + lane * 4;
+    if (lane < quad_lo || lane >= quad_hi) return;
 #pragma unroll 4
     for (int col = warp; col < Q_TILE; col += 8) {
         const int64_t cc = c0 + col;
@@ -862,7 +864,8 @@ static void launch_rows(srq_dtype_t dt, int mode, const void* x, const QuantPara
 // General path: any extent, pitch, alignment and index offset; one Philox block per element
 // when the groups of four do not line up with the flat index.  Same results as the fast path.
 template <typename T>
-__device__ __forceinline__ void quantize_general_tile(const T* __restrict__ x, const QuantParams& P, uint32_t* tileT, int64_t blk) {
+__device__ __forceinline__ void quantize_general_tile(const T* __restrict__ x, const QuantParams& P, uint32_t* tileT, int64_t blk,
+                                                      int it_lo = 0, int it_hi = 4) {     // 32-row slices of the tile this CTA takes
     // transposed tile: column c of the tile holds 128 row codes = 32 words; the word index is
     // XOR-ed with (c >> 2) & 31 so that both the column-wise writes and the row-wise reads
     // touch 32 different banks.
@@ -894,11 +897,11 @@ __device__ __forceinline__ void quantize_general_tile(const T* __restrict__ x, c
             else q[i][0] = q[i][1] = q[i][2] = q[i][3] = 0.0f;
         }
     };
-    load_quad(0, cur);
+    load_quad(it_lo, cur);
 
 #pragma unroll 1
-    for (int it = 0; it < 4; ++it) {
-        if (it + 1 < 4) load_quad(it + 1, nxt);
+    for (int it = it_lo; it < it_hi; ++it) {
+        if (it + 1 < it_hi) load_quad(it + 1, nxt);
         const int rq = warp + 8 * it;   // row quad of the tile
         uint32_t wr[4], wt[4];
 #pragma unroll
@@ -958,7 +961,7 @@ __device__ __forceinline__ void quantize_general_tile(const T* __restrict__ x, c
     }
     if (!want_tr) return;
     __syncthreads();
-    store_transposed_tile(tileT, P, r0, c0, warp, lane);
+    store_transposed_tile(tileT, P, r0, c0, warp, lane, 8 * it_lo, 8 * it_hi);
 }
 
 template <typename T>
@@ -976,6 +979,7 @@ struct QuantBatch {
     const void* x[BATCH_MAX];
     uint32_t first_block[BATCH_MAX + 1];
     int32_t n;
+    int32_t slices;          // CTAs per 128 x 128 tile (1, 2 or 4): tiny batches are spread over more SMs
 };
 
 template <typename T>
@@ -985,7 +989,9 @@ quantize_batch_kernel(const __grid_constant__ QuantBatch Bt) {
     __shared__ uint32_t tileT[Q_TILE * (Q_TILE / 4)];
     int i = 0;
     while (i + 1 < Bt.n && blockIdx.x >= Bt.first_block[i + 1]) ++i;
-    quantize_general_tile<T>((const T*)Bt.x[i], Bt.P[i], tileT, (int64_t)(blockIdx.x - Bt.first_block[i]));
+    const uint32_t local = blockIdx.x - Bt.first_block[i];
+    const int per = 4 / Bt.slices, it_lo = (int)(local % (uint32_t)Bt.slices) * per;
+    quantize_general_tile<T>((const T*)Bt.x[i], Bt.P[i], tileT, (int64_t)(local / (uint32_t)Bt.slices), it_lo, it_lo + per);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1243,6 +1249,12 @@ cudaError_t launch_quantize_batch(const QuantArgs* a, const QuantScratch* s, int
     AmaxBatch ab = {};
     QuantBatch qb = {};
     ab.n = qb.n = n;
+    {   // a handful of tiles would leave most SMs idle and each CTA with a long serial loop: slice the tiles
+        int64_t tiles = 0;
+        for (int i = 0; i < n; ++i) tiles += ((a[i].cols + Q_TILE - 1) / Q_TILE) * ((a[i].rows + Q_TILE - 1) / Q_TILE);
+        const int sms = sm_count();
+        qb.slices = tiles * 4 <= 2 * sms ? 4 : (tiles * 2 <= 2 * sms ? 2 : 1);
+    }
     ab.counter = s[0].counter;                       // zeroed with the rest of the scratch
     uint32_t ablocks = 0, qblocks = 0;
     for (int i = 0; i < n; ++i) {
@@ -1265,7 +1277,7 @@ cudaError_t launch_quantize_batch(const QuantArgs* a, const QuantScratch* s, int
         if (tiles) ablocks += (uint32_t)(((A.cols + tile_c - 1) / tile_c) * ((A.rows + AMAX_TILE_R - 1) / AMAX_TILE_R));
         qb.P[i] = p.P; qb.x[i] = A.x;
         qb.first_block[i] = qblocks;
-        qblocks += (uint32_t)(((A.cols + Q_TILE - 1) / Q_TILE) * ((A.rows + Q_TILE - 1) / Q_TILE));
+        qblocks += (uint32_t)(((A.cols + Q_TILE - 1) / Q_TILE) * ((A.rows + Q_TILE - 1) / Q_TILE)) * (uint32_t)qb.slices;
     }
     ab.first_block[n] = ablocks; qb.first_block[n] = qblocks;
     if (a[0].dt == SRQ_F32) launch_pdl(amax_batch_kernel<float>, dim3(ablocks ? ablocks : 1u), dim3(AMAX_THREADS), 0, stream, ab);
