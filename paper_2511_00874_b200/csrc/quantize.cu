@@ -1253,7 +1253,7 @@ cudaError_t launch_quantize_batch(const QuantArgs* a, const QuantScratch* s, int
         int64_t tiles = 0;
         for (int i = 0; i < n; ++i) tiles += ((a[i].cols + Q_TILE - 1) / Q_TILE) * ((a[i].rows + Q_TILE - 1) / Q_TILE);
         const int sms = sm_count();
-        qb.slices = tiles * 4 <= 2 * sms ? 4 : (tiles * 2 <= 2 * sms ? 2 : 1);
+        qb.slices = tiles * 4 <= 8 * sms ? 4 : (tiles * 2 <= 8 * sms ? 2 : 1);
     }
     ab.counter = s[0].counter;                       // zeroed with the rest of the scratch
     uint32_t ablocks = 0, qblocks = 0;
