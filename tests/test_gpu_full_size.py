@@ -130,3 +130,57 @@ def test_layer_at_full_size(case):
         assert torch.equal(out2, out), name + ": block-store path differs from the element-wise path"
         _freivalds(acc, qa, qb, rng)
         del acc, out2
+
+
+@pytest.mark.parametrize("scale,dtype", [(srq.PER_TENSOR, torch.float32), (srq.PER_ROW, torch.bfloat16)])
+def test_layer_on_the_floating_point_grid_over_many_tiles(scale, dtype):
+    """The E4M3 grid at a size that runs many rounds of CTA-pair tiles (16384 tokens, 4096 -> 4096):
+    every code and step size of all five quantization points against the oracle (bit for bit), and
+    sampled rows of Y, dA and dW against the oracle's exact binary64 products of those codes within
+    1e-5 * |row| * |col| (the summation order of the binary32 accumulators is the hardware's)."""
+    T, N, K = 16384, 4096, 4096
+    A = synth.normal((T, K), 1.0, 2000, dtype, "cuda")
+    dY = synth.normal((T, N), 1e-3, 2001, dtype, "cuda")
+    W = synth.normal((N, K), 0.02, 2002, dtype, "cuda")
+    q = {k: srq.QSpec(8, scale, srq.SR, 4, i, 0, srq.GRID_E4M3) for i, k in enumerate(["a_f", "w_f", "a_b", "w_b", "dy"])}
+    oq = lambda s: oracle.QSpec(s.bits, s.scale, s.round, s.seed, s.tensor_id, s.index_offset)
+    ws = srq.new_workspace(srq.srq_workspace_bytes(T, N, K))
+    Y, dA, dW = torch.empty((T, N), device="cuda"), torch.empty((T, K), device="cuda"), torch.empty((N, K), device="cuda")
+    srq.qlinear_fwd(A, W, q["a_f"], q["w_f"], Y, None, ws)
+    srq.qlinear_bwd(dY, A, W, q["dy"], q["a_b"], q["w_b"], dA, dW, None, None, ws)
+    assert srq.srq_poll_status(ws) == 0
+    hA, hW, hdY = A.float().cpu().numpy(), W.float().cpu().numpy(), dY.float().cpu().numpy()
+    o_af = oracle.sr_quantize_e4m3(hA, oq(q["a_f"]), True, False)
+    o_wf = oracle.sr_quantize_e4m3(hW, oq(q["w_f"]), True, False)
+    o_dy = oracle.sr_quantize_e4m3(hdY, oq(q["dy"]), True, True)
+    o_wb = oracle.sr_quantize_e4m3(hW, oq(q["w_b"]), False, True)
+    o_ab = oracle.sr_quantize_e4m3(hA, oq(q["a_b"]), False, True)
+    g_af = _codes(A, q["a_f"], True, False)
+    g_wf = _codes(W, q["w_f"], True, False)
+    g_dy = _codes(dY, q["dy"], True, True)
+    g_wb = _codes(W, q["w_b"], False, True)
+    g_ab = _codes(A, q["a_b"], False, True)
+    u8 = lambda t: t.view(torch.uint8).cpu().numpy()
+    for name, g, o in (("A fwd", g_af[0], o_af[0]), ("W fwd", g_wf[0], o_wf[0]), ("dY", g_dy[0], o_dy[0]), ("dY^T", g_dy[1], o_dy[2]),
+                       ("W^T bwd", g_wb[1], o_wb[2]), ("A^T bwd", g_ab[1], o_ab[2])):
+        assert np.array_equal(u8(g), o), name + ": codes"
+    for name, g, o in (("A fwd", g_af[2], o_af[1]), ("W fwd", g_wf[2], o_wf[1]), ("dY", g_dy[2], o_dy[1]), ("dY^T", g_dy[3], o_dy[3]),
+                       ("W bwd", g_wb[3], o_wb[3]), ("A bwd", g_ab[3], o_ab[3])):
+        assert np.array_equal(g.cpu().numpy(), o), name + ": step size"
+    rng = np.random.default_rng(1)
+    rows_t = np.sort(rng.choice(T, 24, replace=False))
+    rows_n = np.sort(rng.choice(N, 8, replace=False))
+    pick = lambda sc, rows: sc if sc.size == 1 else sc[rows]
+
+    def check(name, out, rows, ca, sa, cb, sb):
+        _, ref = oracle.gemm_e4m3_nt(ca[rows], cb, pick(sa, rows), sb)
+        na = np.linalg.norm(oracle.e4m3_decode(ca[rows]), axis=1)
+        nb = np.linalg.norm(oracle.e4m3_decode(cb), axis=1)
+        sc = np.broadcast_to(pick(sa, rows), (len(rows),))[:, None].astype(np.float64) * np.broadcast_to(sb, (cb.shape[0],))[None, :]
+        bound = 1e-5 * na[:, None] * nb[None, :] * sc + 1e-30
+        got = out[torch.from_numpy(rows).cuda()].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref) <= bound * 1.001 + np.abs(ref) * 2e-7), name
+
+    check("Y rows", Y, rows_t, o_af[0], o_af[1], o_wf[0], o_wf[1])
+    check("dA rows", dA, rows_t, o_dy[0], o_dy[1], o_wb[2], o_wb[3])
+    check("dW rows", dW, rows_n, o_dy[2], o_dy[3], o_ab[2], o_ab[3])
