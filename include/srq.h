@@ -370,6 +370,17 @@ void srq_plan_splits(int64_t tiles, int32_t k_blocks, int32_t groups, int32_t *f
  * SRQ_ERR_TIMEOUT (read it with srq_poll_status), the kernel returns and the context stays usable. */
 srq_status_t srq_selftest_bounded_wait(void *ws, size_t ws_bytes, uint32_t limit_us, void *cuda_stream);
 
+/* Measurement aid, not part of the layer: device-side timing of the product kernel inside whatever
+ * sequence of calls the caller runs (a whole layer step), which stream events around a call cannot
+ * give because a call enqueues several kernels.  slots is a caller-owned DEVICE array of 2 * n
+ * 64-bit words that the caller has initialised to (all ones, zero) pairs: the i-th product launch
+ * after this call lowers slots[2 i] to the nanosecond time (%globaltimer) at which its first CTA
+ * starts work, after the kernel before it has finished, and raises slots[2 i + 1] to the time its
+ * last CTA ends; launches beyond n are not timed.  Two atomics per CTA, nothing else changes.
+ * srq_set_product_timer(NULL, 0) switches it off.  The setting is process-wide (all streams and
+ * devices): time one stream at a time. */
+srq_status_t srq_set_product_timer(uint64_t *slots, int64_t n);
+
 /* Measurement aid, not part of the layer: the issue rate of the tensor pipe for the instruction the
  * products use (tcgen05.mma.cta_group::2.kind::i8, M256 N256 K32).  Every CTA pair of the device
  * multiplies operand blocks that already sit in its shared memory, k_blocks (1 .. 2^22) blocks of 128

@@ -28,7 +28,7 @@ GRID_INT, GRID_E4M3, GRID_NONE = 0, 1, 2
 EXPORTS = ["srq_quantize_workspace_bytes", "srq_gemm_workspace_bytes", "srq_workspace_bytes",
            "sr_quantize", "sr_quantize_static", "srq_absmax", "srq_absmax_cols", "srq_gemm_i8", "srq_gemm_e4m3", "qlinear_fwd", "qlinear_bwd_input", "qlinear_bwd_weight", "qlinear_bwd",
            "srq_gemm_i8_ex", "qlinear_fwd_ex", "qlinear_bwd_ex", "srq_dequant_i32",
-           "srq_poll_status", "srq_status_string", "srq_launch_count", "srq_selftest_bounded_wait", "srq_selftest_mma_rate", "srq_plan_splits"]
+           "srq_poll_status", "srq_status_string", "srq_launch_count", "srq_selftest_bounded_wait", "srq_selftest_mma_rate", "srq_set_product_timer", "srq_plan_splits"]
 
 
 class SrqError(RuntimeError):
@@ -125,6 +125,8 @@ def lib() -> ctypes.CDLL:
     L.srq_selftest_bounded_wait.restype = ctypes.c_int
     L.srq_selftest_mma_rate.argtypes = [vp, sz, i32, ctypes.POINTER(i64), vp]
     L.srq_selftest_mma_rate.restype = ctypes.c_int
+    L.srq_set_product_timer.argtypes = [vp, i64]
+    L.srq_set_product_timer.restype = ctypes.c_int
     L.srq_plan_splits.argtypes = [i64, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.srq_plan_splits.restype = None
     L.srq_poll_status.argtypes = [vp, vp]
@@ -494,6 +496,24 @@ def srq_selftest_mma_rate(ws: torch.Tensor, k_blocks: int) -> int:
     _check(lib().srq_selftest_mma_rate(ws.data_ptr(), ws.numel(), int(k_blocks), ctypes.byref(ops), _stream()),
            "srq_selftest_mma_rate")
     return int(ops.value)
+
+
+def srq_set_product_timer(slots: Optional[torch.Tensor]) -> None:
+    """Device-side start / end times (ns) of the next product launches into ``slots``, an int64 CUDA
+    tensor of shape [n, 2] initialised with ``new_product_timer``; None switches the timing off."""
+    if slots is None:
+        _check(lib().srq_set_product_timer(None, 0), "srq_set_product_timer")
+        return
+    if slots.dtype != torch.int64 or slots.dim() != 2 or slots.shape[1] != 2 or not slots.is_contiguous():
+        raise TypeError("slots must be a contiguous int64 CUDA tensor of shape [n, 2]")
+    _check(lib().srq_set_product_timer(slots.data_ptr(), slots.shape[0]), "srq_set_product_timer")
+
+
+def new_product_timer(n: int, device="cuda") -> torch.Tensor:
+    """[n, 2] slots holding (all ones, zero): what srq_set_product_timer expects."""
+    t = torch.zeros((n, 2), dtype=torch.int64, device=device)
+    t[:, 0] = -1
+    return t
 
 
 def srq_poll_status(ws: torch.Tensor) -> int:

@@ -546,6 +546,12 @@ srq_status_t srq_selftest_bounded_wait(void* ws, size_t ws_bytes, uint32_t limit
     return launch_bounded_wait_probe(&((WsHeader*)ws)->status, (uint64_t)limit_us * 1000ull, st) == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
 }
 
+srq_status_t srq_set_product_timer(uint64_t* slots, int64_t n) {
+    if (n < 0 || (n > 0 && (!slots || !aligned_to(slots, 8)))) return SRQ_ERR_INVALID_ARG;
+    set_product_timer((unsigned long long*)slots, n);
+    return SRQ_OK;
+}
+
 srq_status_t srq_selftest_mma_rate(void* ws, size_t ws_bytes, int32_t k_blocks, int64_t* ops, void* cuda_stream) {
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (!ws || !aligned_to(ws, 256) || k_blocks < 1 || k_blocks > (1 << 22)) return SRQ_ERR_INVALID_ARG;

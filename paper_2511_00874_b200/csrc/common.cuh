@@ -206,6 +206,8 @@ cudaError_t launch_bounded_wait_probe(uint32_t* status, uint64_t limit_ns, cudaS
 cudaError_t launch_finish_sums(const int32_t* acc, int64_t ld_acc, int64_t M, int64_t N, const float* s_row, int32_t row_stride,
                                const float* s_col, int32_t col_stride, float* out, int64_t ldo, int out_bf16, cudaStream_t stream);
 srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t stream);
+// Device-side timing of the next n product launches into slots[2 * i] (start) / slots[2 * i + 1] (end).
+void set_product_timer(unsigned long long* slots, int64_t n);
 // Tensor-pipe issue-rate microbenchmark: every CTA pair issues k_blocks x 4 kind::i8 MMAs (M256 N256 K32)
 // on operands resident in shared memory; *ops receives the integer operations of the launch.
 srq_status_t launch_mma_rate(int32_t k_blocks, uint32_t* status, int64_t* ops, cudaStream_t stream);

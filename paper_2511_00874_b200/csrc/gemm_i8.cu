@@ -292,6 +292,7 @@ struct GemmParams {
     int32_t* acc_out;          // optional raw sums [M, N]
     int32_t* part;             // split tiles: zeroed int32 [(tiles - full_tiles) * 128 * CTAS, 256], tile after tile
     uint32_t* status;
+    unsigned long long* timer; // optional: [0] lowered to the time the first CTA starts its work, [1] raised to the time the last one ends
     int32_t vec_out;           // 16-byte stores to out allowed
     int32_t tma_out;           // out is written with TMA stores (map_out valid, no acc_out)
     int32_t write_out;         // out is wanted (it may be left out when only codes are)
@@ -395,6 +396,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = T->tmem_base;
     pdl_wait();                                      // from here on the work before this kernel has finished and is visible
+    if (P.timer && threadIdx.x == 0) atomicMin(&P.timer[0], (unsigned long long)global_ns());
 
     const int64_t groups = gridDim.x / CTAS, group = blockIdx.x / CTAS;   // a group = the CTAs of one tile
     // work units: the first full_tiles tiles whole, then every remaining tile in `splits` parts
@@ -743,6 +745,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tc_fence_after();
         tmem_dealloc<CTAS>(tmem_base, TMEM_COLS);
     }
+    if (P.timer && threadIdx.x == 0) atomicMax(&P.timer[1], (unsigned long long)global_ns());
 }
 
 // Second step of a split contraction: out = float(sum) * (s_row * s_col) over the finished sums of the
@@ -1036,6 +1039,22 @@ srq_status_t launch_mma_rate(int32_t k_blocks, uint32_t* status, int64_t* ops, c
     return e == cudaSuccess ? SRQ_OK : SRQ_ERR_CUDA;
 }
 
+// Optional device-side timing of the product launches (srq_set_product_timer): launch i of the calls
+// that follow writes its start and end times into slot i of a caller-owned device array.
+static std::mutex g_timer_mu;
+static unsigned long long* g_timer_slots = nullptr;
+static int64_t g_timer_n = 0, g_timer_next = 0;
+
+void set_product_timer(unsigned long long* slots, int64_t n) {
+    std::lock_guard<std::mutex> lock(g_timer_mu);
+    g_timer_slots = n > 0 ? slots : nullptr; g_timer_n = n > 0 ? n : 0; g_timer_next = 0;
+}
+static unsigned long long* next_timer_slot() {
+    std::lock_guard<std::mutex> lock(g_timer_mu);
+    if (!g_timer_slots || g_timer_next >= g_timer_n) return nullptr;
+    return g_timer_slots + 2 * g_timer_next++;
+}
+
 // Which tiles are split, and into how many parts.  `groups` tiles run at a time.  Too few tiles to fill
 // the machine: all of them are split.  Several rounds of tiles with a last, partly empty round: only
 // the tiles of that round are split, so that it takes a fraction of a round.  Each part keeps at least
@@ -1118,6 +1137,7 @@ srq_status_t launch_gemm_i8(const GemmArgs& g, uint32_t* status, cudaStream_t st
     P.s_col = g.s_col; P.col_stride = g.col_stride;
     P.out = g.out; P.ldo = g.ldo; P.acc_out = g.acc_out;
     P.status = status;
+    P.timer = next_timer_slot();
     const int out_vec_elems = g.opt.out_bf16 ? 8 : 4;      // elements per 16 bytes of output
     P.vec_out = g.out && ((uintptr_t)g.out % 16 == 0) && (g.ldo % out_vec_elems == 0);
 

@@ -218,3 +218,31 @@ def test_tensor_pipe_microbenchmark_runs_and_counts_its_operations():
         assert ops > 0 and ops % (kb * 2 * 256 * 256 * 128) == 0 and ops // (kb * 2 * 256 * 256 * 128) <= pairs
     with pytest.raises(srq.SrqError):
         srq.srq_selftest_mma_rate(ws, 0)
+
+
+def test_product_timer_brackets_the_launches_and_changes_no_result():
+    """srq_set_product_timer: the next launches write their device-side start and end times into the
+    caller's slots, in order; launches beyond the slots and launches after it is switched off are not
+    timed; results stay those of the untimed call."""
+    a, b = _codes(512, 1024, 1), _codes(512, 1024, 2)
+    one = torch.ones(1, device="cuda")
+    want, _ = _run(a, b, one, one, want_acc=False)
+    slots = srq.new_product_timer(2)
+    srq.srq_set_product_timer(slots)
+    try:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        outs = [_run(a, b, one, one, want_acc=False)[0] for _ in range(3)]      # the third finds no slot
+        e1.record()
+        torch.cuda.synchronize()
+    finally:
+        srq.srq_set_product_timer(None)
+    t = slots.cpu().numpy()
+    dur = t[:, 1] - t[:, 0]
+    assert (t[:, 0] > 0).all() and (dur > 0).all() and (dur < e0.elapsed_time(e1) * 1e6).all()
+    assert t[1, 0] >= t[0, 1]                                   # the second launch starts after the first has ended
+    for o in outs:
+        assert np.array_equal(o, want)
+    again = srq.new_product_timer(1)
+    _run(a, b, one, one, want_acc=False)                        # switched off: nothing is written
+    assert again[0, 1].item() == 0
