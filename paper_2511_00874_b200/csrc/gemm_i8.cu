@@ -127,8 +127,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
     return r;
 }
+// Arrival on a barrier of the pair (possibly the other CTA's).  What it orders here are TMEM reads
+// against the MMAs that overwrite the accumulator, which the tcgen05 fences on both sides of the
+// barrier take care of; a cluster-scope release on top of that made the arriving thread wait for its
+// outstanding memory traffic (about 2 800 cycles per tile at the end of a tile's stores).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
 // Tile load into this CTA's shared memory.  CTAS = 2: the completion bytes are counted on the
@@ -568,6 +572,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // previous block's store to have read the staging buffer (8 warps x 4 blocks x 4 KB).
             const uint32_t ring_stage = smem_u32(smem) + (uint32_t)((warp - 2) * 4) * (uint32_t)OUT_STAGE_BYTES;
             const int32_t wrow = (int32_t)(row0 + quarter * 32);           // first row of this warp's blocks
+            // The accumulator is free as soon as this warp's last TMEM load has completed: the MMAs of the
+            // tile after next start while the last block is still being scaled, staged and stored.
+            auto release_acc = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0 && releases) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
+            };
             if (whole && P.tma_out && P.opt.out_bf16) {
                 // two 32-column blocks at a time: 64 bfloat16 results per row fill the 128-byte rows
                 // of the staging block, stored as one 32 x 64 box
@@ -579,6 +590,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         uint32_t v[32];
                         tmem_ld32(taddr + j * 64 + h * 32, v);
                         tmem_ld_wait();
+                        if (h == 1 && j == j_hi / 2 - 1) release_acc();
                         const float* sc = &T->s_col[cbuf][j * 64 + h * 32];
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
@@ -596,9 +608,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     __syncwarp();
                     if (lane == 0 && wrow < P.M && col0 < P.N) { tma_store_2d(&map_out, stg, col0, wrow); bulk_commit(); }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0 && releases) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             } else if (whole && P.tma_out) {
                 // registers -> swizzled shared-memory block -> one TMA store per 32 x 32 block
 #pragma unroll 1
@@ -606,6 +615,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     uint32_t v[32];
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
+                    if (j == j_hi - 1) release_acc();
                     const float* sc = &T->s_col[cbuf][j * 32];
                     if (!P.opt.raw_sums) {                    // raw sums leave as the int32 words they are
 #pragma unroll
@@ -631,9 +641,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         bulk_commit();
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0 && releases) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             } else if (whole) {
 #pragma unroll 1
                 for (int j = j_lo; j < j_hi; ++j) {
@@ -715,6 +722,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     uint32_t v[32];
                     tmem_ld32(taddr + j * 32, v);
                     tmem_ld_wait();
+                    if (j == j_hi - 1) release_acc();
                     const uint32_t stg = share ? ring_stage + (uint32_t)(j - j_lo) * (uint32_t)OUT_STAGE_BYTES : stage;
                     if (!share && lane == 0) bulk_wait_read();
                     __syncwarp();
@@ -723,9 +731,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) { tma_reduce_add_2d(&map_part, stg, j * 32, prow); bulk_commit(); }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0 && releases) mbar_arrive_cluster(buf ? empty_bar1 : empty_bar0);
             }
         }
         if (P.opt.absmax_bits) {      // absmax of everything this warp produced: one guarded atomic
